@@ -1,0 +1,228 @@
+/*
+ * agx - prefix-cached block attention and greedy speculative acceptance for NVIDIA B200 (sm_100a).
+ *
+ * One GPU hot path, shared by the two halves of the Agent-X method:
+ *   prefill with prefix caching  : attention of the q uncached suffix tokens of a prompt over a
+ *                                  KV cache that already holds the cached prefix (Sec. 2.3,
+ *                                  "Prefix caching"; Sec. 4.2 makes the prefix long and the suffix short);
+ *   speculative-decoding verify  : attention of the most recent token followed by N draft tokens
+ *                                  (q = N + 1) over the whole cached context, then acceptance
+ *                                  (Sec. 2.3, "Speculative decoding"; Sec. 4.3 supplies the drafts
+ *                                  from an n-gram table and falls back to q = 1 on a table miss).
+ *
+ * Conventions shared by every call
+ *   - All functions are extern "C", return an agx_status (0 = AGX_OK, negative = error) unless
+ *     stated otherwise, never throw and never abort.  Work is enqueued on the caller's stream and
+ *     the call returns without synchronising (except agx_get_status and the *_host call).
+ *   - "device" pointers are device memory owned by the caller; "host" pointers are ordinary host
+ *     memory read during the call only (the caller may reuse it as soon as the call returns).
+ *     The library never frees or retains caller memory.  The handle owns a few hundred bytes of
+ *     device state (a status word and a ticket counter).
+ *   - A handle must be used from one stream at a time: calls on the same handle that overlap on
+ *     the GPU share that state and race.
+ *   - Ragged batches: B sequences; sequence s has a cached prefix of prefix_len[s] tokens and a
+ *     block of q_len[s] >= 1 new tokens; cu_q[B+1] is the exclusive prefix sum of q_len and
+ *     total_q = cu_q[B].  Rows of q_block, k_new, v_new, out and logits are sequence-major,
+ *     position-minor: row cu_q[s] + i is block position i of sequence s.
+ *   - Element type: AGX_BF16 (bfloat16) or AGX_F32 (float), fixed per handle.  Accumulation and
+ *     softmax are always fp32; outputs are rounded to the element type (nearest-even).
+ *   - KV pool layout (library-defined): k_pool and v_pool are [num_pages][num_kv_heads][16][head_dim],
+ *     256-byte aligned.  Token t of sequence s lives in page page_table[s*page_table_stride + t/16],
+ *     slot t%16.  prefix_len need not be a multiple of 16 (a reused prefix may be cut anywhere).
+ *     Pages may be shared between sequences for reading; pages that a call appends into must be
+ *     private to that sequence.
+ *   - Query head h reads KV head h / (num_q_heads / num_kv_heads).
+ */
+#ifndef AGX_H_
+#define AGX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define AGX_API __attribute__((visibility("default")))
+#else
+#define AGX_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct agx_handle agx_handle;
+typedef int32_t agx_status;
+
+enum {
+    AGX_OK = 0,
+    AGX_E_INVAL = -1,       /* null / misaligned pointer, bad shape, q_len < 1, workspace too small */
+    AGX_E_RANGE = -2,       /* lengths exceed the page table, or too many sequences/rows */
+    AGX_E_UNSUPPORTED = -3, /* head_dim, page size or dtype combination not built */
+    AGX_E_CUDA = -4,        /* a CUDA runtime call or launch failed; see agx_last_error */
+    AGX_E_DEVICE = -5,      /* the device status word is non-zero (see agx_get_status) */
+    AGX_E_NOMEM = -6
+};
+
+enum { AGX_BF16 = 0, AGX_F32 = 1 };
+
+/* Bits of the device status word (sticky until agx_get_status clears them). */
+enum {
+    AGX_DEV_BAD_PAGE = 1,    /* a page id outside [0, num_pages) was met; the access was skipped */
+    AGX_DEV_WAIT_TIMEOUT = 2 /* a bounded in-kernel wait gave up; results of that launch are invalid */
+};
+
+typedef struct agx_config {
+    int32_t num_q_heads;  /* Hq */
+    int32_t num_kv_heads; /* Hkv, divides Hq */
+    int32_t head_dim;     /* d: 64 or 128 for AGX_F32, 128 for AGX_BF16 */
+    int32_t page_size;    /* must be 16 */
+    int32_t dtype;        /* AGX_BF16 or AGX_F32 */
+    float scale;          /* softmax scale; 0 selects 1/sqrt(head_dim) */
+} agx_config;
+
+/* Create / destroy a handle on the current CUDA device.  No paper counterpart (plumbing). */
+AGX_API agx_status agx_create(const agx_config* config, agx_handle** out_handle);
+AGX_API agx_status agx_destroy(agx_handle* handle);
+
+/* Text for a status code; and the detail message of the last failing call on this handle
+ * (valid until the next call on the handle).  Never NULL. */
+AGX_API const char* agx_status_string(agx_status status);
+AGX_API const char* agx_last_error(const agx_handle* handle);
+
+/*
+ * agx_kv_append - write the block's K and V rows into the sequences' pages.
+ * Sec. 2.3: prefill fills the KV cache; with prefix caching only the uncached suffix is
+ * written, after the cached prefix.  In a verify step the rows are speculative: acceptance later
+ * commits a length and moves no data; dead slots are overwritten by the next append.
+ *   k_pool, v_pool : device, pools as laid out above (written)
+ *   k_new, v_new   : device, [total_q][num_kv_heads][head_dim], 16-byte aligned
+ *   page_table     : device int32, [B][page_table_stride]
+ *   prefix_len     : device int32 [B]; row i of sequence s goes to token slot prefix_len[s] + i
+ *   cu_q           : device int32 [B+1]
+ * Errors: AGX_E_INVAL on null/misaligned pointers or B/total_q < 0; a page id outside
+ * [0, num_pages) sets AGX_DEV_BAD_PAGE and that row is not written.  B == 0 or total_q == 0 is a no-op.
+ */
+AGX_API agx_status agx_kv_append(agx_handle* handle, void* k_pool, void* v_pool, int64_t num_pages,
+                         const void* k_new, const void* v_new, const int32_t* page_table,
+                         int32_t page_table_stride, const int32_t* prefix_len, const int32_t* cu_q,
+                         int32_t B, int32_t total_q, void* stream);
+
+/*
+ * agx_attn_workspace_bytes - scratch bytes agx_attn_prefixed needs for this batch (host lengths).
+ * Returns a negative agx_status on bad arguments.  The figure depends only on the config, the
+ * lengths and the device's SM count.
+ */
+AGX_API int64_t agx_attn_workspace_bytes(agx_handle* handle, int32_t B, const int32_t* h_prefix_len,
+                                 const int32_t* h_q_len);
+
+/*
+ * agx_attn_prefixed - attention of each sequence's block over its cached prefix plus the block.
+ * Sec. 2.3 (prefix caching): a token looks only at the tokens up to itself, so row i of the block
+ * (absolute position P + i) attends to tokens 0 .. P + i of the sequence: all of the cached prefix, and the
+ * block rows up to and including itself.  The same call serves the verify block of speculative
+ * decoding (q = N + 1) and plain decode (q = 1).  agx_kv_append for the same block must have
+ * been enqueued before, so the pages already hold tokens P .. P + q - 1.
+ *   out[r][h][:] = sum_j softmax_j(scale * <q_block[r][h], K[j][h/G]>) V[j][h/G],  j in [0, P + i]
+ *   q_block      : device, [total_q][num_q_heads][head_dim], 16-byte aligned
+ *   k_pool,v_pool: device pools (read only); page_table: device int32 [B][page_table_stride]
+ *   h_prefix_len, h_q_len : HOST int32 [B].  They size the launch and are copied into kernel
+ *                  arguments, so the values in force are the ones passed here.
+ *   out          : device, [total_q][num_q_heads][head_dim], element type of the handle
+ *   lse          : device float [total_q][num_q_heads] or NULL; natural-log sum of exp of the
+ *                  scaled scores
+ *   workspace    : device, >= agx_attn_workspace_bytes(...) bytes, 256-byte aligned (may be NULL
+ *                  when that figure is 0)
+ * Dispatch: a sequence whose q_len * G rows fit one 64-row tile runs the split-KV kernel
+ * (bandwidth-bound); longer blocks run the tensor-core tile kernel.  Sequences of both kinds may
+ * share a batch.
+ * Errors: AGX_E_INVAL (null/misaligned, q_len < 1, prefix_len < 0, workspace too small),
+ * AGX_E_RANGE ((P + q) exceeds 16 * page_table_stride), AGX_E_CUDA.  Page ids outside
+ * [0, num_pages) set AGX_DEV_BAD_PAGE and read as zeros.
+ */
+AGX_API agx_status agx_attn_prefixed(agx_handle* handle, const void* q_block, const void* k_pool,
+                             const void* v_pool, int64_t num_pages, const int32_t* page_table,
+                             int32_t page_table_stride, const int32_t* h_prefix_len,
+                             const int32_t* h_q_len, int32_t B, void* out, float* lse,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Scratch bytes agx_accept_greedy needs for total_q logits rows. */
+AGX_API int64_t agx_accept_workspace_bytes(agx_handle* handle, int32_t total_q, int32_t vocab);
+
+/*
+ * agx_accept_greedy - per-row vocabulary argmax, longest matching draft prefix, commit.
+ * Sec. 2.3 (speculative decoding, steps 2-3): drafts are kept up to the first one the target
+ * disagrees with; that draft and every later one are dropped, and the kept drafts plus the
+ * target's own next token start the next round.  With
+ * an n-gram draft source (Sec. 4.3) there are no draft logits, so a draft is accepted iff it
+ * equals the target's greedy token.
+ * For sequence s with k = q_len[s] - 1 drafts d_1..d_k, logits row 0 belongs to the most recent
+ * token and row i to draft d_i:
+ *   t_r        = lowest index attaining max_v logits[r][v]   (NaN never beats a number; a row of
+ *                only NaN gives 0; -0 and +0 tie)
+ *   accept_len = number of leading i in 1..k with d_i == t_{i-1}
+ *   next_token = t_{accept_len};   seq_lens[s] <- seq_lens[s] + accept_len + 1
+ *   logits     : device, [total_q][row_stride] of logits_dtype (AGX_BF16 / AGX_F32); only the
+ *                first vocab entries of a row are read; rows 16-byte aligned
+ *   drafts     : device int32 [total_q - B]; sequence s owns entries cu_q[s]-s .. (any int32 is
+ *                legal; values outside [0, vocab) never match)
+ *   cu_q       : device int32 [B+1]
+ *   accept_len, next_token : device int32 [B] (written)
+ *   argmax     : device int32 [total_q] or NULL (written)
+ *   seq_lens   : device int32 [B] or NULL; in: committed length before the block (the prefix
+ *                length), out: prefix + accept_len + 1
+ * Prefill uses the same call with no drafts (q_len = 1 per sequence, the last row's logits).
+ * Errors: AGX_E_INVAL, AGX_E_RANGE (vocab < 1, row_stride < vocab), AGX_E_CUDA.
+ */
+AGX_API agx_status agx_accept_greedy(agx_handle* handle, const void* logits, int32_t logits_dtype,
+                             int64_t row_stride, int32_t vocab, const int32_t* drafts,
+                             const int32_t* cu_q, int32_t B, int32_t total_q, int32_t* accept_len,
+                             int32_t* next_token, int32_t* argmax, int32_t* seq_lens,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * agx_get_status - synchronise the stream, read and clear the device status word.
+ * *device_status receives the AGX_DEV_* bits (0 = clean).  Returns AGX_E_DEVICE when non-zero.
+ */
+AGX_API agx_status agx_get_status(agx_handle* handle, void* stream, int32_t* device_status);
+
+/*
+ * agx_verify_step_host - one whole step (append, attention, acceptance) for callers whose
+ * activations live in HOST memory.  Same operations as the three calls above (Sec. 2.3), plus the
+ * host<->device copies: q_block, k_new, v_new, logits, drafts and the lengths go to the device,
+ * out, accept_len, next_token and seq_lens come back, and the stream is synchronised before the
+ * call returns.  The KV pools and the page table stay on the device: they are the cache.
+ *   k_pool, v_pool, page_table : device (as in agx_kv_append)
+ *   h_prefix_len, h_q_len      : host int32 [B]
+ *   h_q_block, h_k_new, h_v_new: host, element type of the handle (pinned memory makes the
+ *                                copies asynchronous; pageable memory works but serialises)
+ *   h_logits                   : host, [total_q][row_stride] of logits_dtype
+ *   h_drafts                   : host int32 [total_q - B] (may be NULL when total_q == B)
+ *   h_out                      : host, [total_q][num_q_heads][head_dim]
+ *   h_accept_len, h_next_token, h_seq_lens : host int32 [B]; h_seq_lens receives
+ *                                prefix_len + accept_len + 1
+ *   workspace                  : device, >= agx_verify_step_host_workspace_bytes(...) bytes,
+ *                                256-byte aligned; holds the staged copies and both scratch areas
+ * Errors: as the three calls; nothing is launched when a check fails.
+ */
+AGX_API int64_t agx_verify_step_host_workspace_bytes(agx_handle* handle, int32_t B,
+                                                     const int32_t* h_prefix_len,
+                                                     const int32_t* h_q_len, int32_t logits_dtype,
+                                                     int64_t row_stride, int32_t vocab);
+AGX_API agx_status agx_verify_step_host(agx_handle* handle, void* k_pool, void* v_pool,
+                                        int64_t num_pages, const int32_t* page_table,
+                                        int32_t page_table_stride, const int32_t* h_prefix_len,
+                                        const int32_t* h_q_len, int32_t B, const void* h_q_block,
+                                        const void* h_k_new, const void* h_v_new,
+                                        const void* h_logits, int32_t logits_dtype,
+                                        int64_t row_stride, int32_t vocab, const int32_t* h_drafts,
+                                        void* h_out, int32_t* h_accept_len, int32_t* h_next_token,
+                                        int32_t* h_seq_lens, void* workspace,
+                                        size_t workspace_bytes, void* stream);
+
+/* Number of kernels the last agx_attn_prefixed / agx_accept_greedy / agx_kv_append call on this
+ * handle launched (for launch accounting in benchmarks). */
+AGX_API int32_t agx_last_launch_count(const agx_handle* handle);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AGX_H_ */

@@ -1,0 +1,172 @@
+// Greedy acceptance: per-row vocabulary argmax fused with the draft comparison and the length
+// commit, in ONE launch (Sec. 2.3, speculative decoding: the first mismatching draft and all
+// drafts after it are discarded; the accepted drafts plus the target's own token continue).
+//
+// HBM-bound scan: rows * vocab * elem bytes, read once with 128-bit loads.  Grid = (chunks, rows);
+// every block reduces its slice of one row to a packed 64-bit (ordered value, inverted index) key
+// whose unsigned maximum is "largest value, lowest index on ties".  The last block to finish
+// (ticket counter) folds the per-chunk keys, compares drafts and writes the results, so no second
+// launch and no host round trip is needed.
+#include "agx_internal.cuh"
+
+namespace agx {
+
+// Monotone map float -> uint32 with: NaN -> 0 (below everything), -0 == +0.
+__device__ __forceinline__ unsigned int ordered_key(float x) {
+    if (x != x) return 0u;
+    unsigned int b = __float_as_uint(x);
+    if (b == 0x80000000u) b = 0u;
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+__device__ __forceinline__ unsigned long long pack_key(unsigned int key, unsigned int idx) {
+    return ((unsigned long long)key << 32) | (unsigned long long)(0xFFFFFFFFu - idx);
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(unsigned int lo16) { return __uint_as_float(lo16 << 16); }
+
+template <bool kBf16>
+__device__ __forceinline__ void scan_vec(const uint4 v, unsigned int base, unsigned int& best_key,
+                                         unsigned int& best_idx) {
+    const unsigned int w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (kBf16) {
+            const unsigned int k0 = ordered_key(bf16_bits_to_float(w[i] & 0xFFFFu));
+            const unsigned int k1 = ordered_key(__uint_as_float(w[i] & 0xFFFF0000u));
+            if (k0 > best_key) { best_key = k0; best_idx = base + 2 * i; }
+            if (k1 > best_key) { best_key = k1; best_idx = base + 2 * i + 1; }
+        } else {
+            const unsigned int k0 = ordered_key(__uint_as_float(w[i]));
+            if (k0 > best_key) { best_key = k0; best_idx = base + i; }
+        }
+    }
+}
+
+template <bool kBf16, bool kVec>
+__global__ void __launch_bounds__(256)
+accept_kernel(const void* __restrict__ logits, long long row_stride, int vocab, int chunk_elems, int chunks,
+              const int* __restrict__ drafts, const int* __restrict__ cu_q, int B, int total_q,
+              int* __restrict__ accept_len, int* __restrict__ next_token, int* __restrict__ argmax,
+              int* __restrict__ seq_lens, unsigned long long* partials, int* tokens, unsigned int* ticket) {
+    constexpr int kVecElems = kBf16 ? 8 : 4;
+    const int row = blockIdx.y;
+    const int chunk = blockIdx.x;
+    const unsigned int begin = (unsigned int)chunk * (unsigned int)chunk_elems;
+    const unsigned int end = min((unsigned int)vocab, begin + (unsigned int)chunk_elems);
+
+    unsigned long long best = 0ull;  // "no element": loses to every real element
+    if (kVec) {
+        const char* row_ptr = (const char*)logits + (size_t)row * row_stride * (kBf16 ? 2 : 4);
+        unsigned int best_key = 0u, best_idx = 0u;
+        bool any = false;
+        // two independent 16-byte loads in flight per thread per trip
+        unsigned int i = begin + threadIdx.x * kVecElems;
+        const unsigned int stride = 256 * kVecElems;
+        for (; i + stride + kVecElems <= end; i += 2 * stride) {
+            const uint4 a = __ldg((const uint4*)(row_ptr + (size_t)i * (kBf16 ? 2 : 4)));
+            const uint4 b = __ldg((const uint4*)(row_ptr + (size_t)(i + stride) * (kBf16 ? 2 : 4)));
+            if (!any) { best_idx = i; any = true; }
+            scan_vec<kBf16>(a, i, best_key, best_idx);
+            scan_vec<kBf16>(b, i + stride, best_key, best_idx);
+        }
+        for (; i < end; i += stride) {
+            if (i + kVecElems <= end) {
+                const uint4 a = __ldg((const uint4*)(row_ptr + (size_t)i * (kBf16 ? 2 : 4)));
+                if (!any) { best_idx = i; any = true; }
+                scan_vec<kBf16>(a, i, best_key, best_idx);
+            } else {
+                for (unsigned int e = i; e < end; ++e) {
+                    float x;
+                    if (kBf16) x = bf16_bits_to_float(((const unsigned short*)row_ptr)[e]);
+                    else x = ((const float*)row_ptr)[e];
+                    const unsigned int k = ordered_key(x);
+                    if (!any) { best_idx = e; any = true; }
+                    if (k > best_key) { best_key = k; best_idx = e; }
+                }
+            }
+        }
+        if (any) best = pack_key(best_key, best_idx);
+    } else {
+        for (unsigned int e = begin + threadIdx.x; e < end; e += 256) {
+            float x;
+            if (kBf16) x = bf16_bits_to_float(((const unsigned short*)logits)[(size_t)row * row_stride + e]);
+            else x = ((const float*)logits)[(size_t)row * row_stride + e];
+            const unsigned long long k = pack_key(ordered_key(x), e);
+            best = k > best ? k : best;
+        }
+    }
+
+    // block reduce (unsigned 64-bit max)
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, best, off);
+        best = o > best ? o : best;
+    }
+    __shared__ unsigned long long warp_best[8];
+    __shared__ bool is_last;
+    if ((threadIdx.x & 31) == 0) warp_best[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long b = warp_best[0];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) b = warp_best[w] > b ? warp_best[w] : b;
+        partials[(size_t)row * chunks + chunk] = b;
+        __threadfence();
+        const unsigned int total = gridDim.x * gridDim.y;
+        const unsigned int t = atomicAdd(ticket, 1u);
+        is_last = (t == total - 1);
+        if (is_last) *ticket = 0u;  // leave the counter ready for the next launch
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+
+    // final fold: one thread per row
+    for (int r = threadIdx.x; r < total_q; r += 256) {
+        unsigned long long b = 0ull;
+        for (int c = 0; c < chunks; ++c) {
+            const unsigned long long v = __ldcg(partials + (size_t)r * chunks + c);
+            b = v > b ? v : b;
+        }
+        const int t = (int)(0xFFFFFFFFu - (unsigned int)(b & 0xFFFFFFFFull));
+        tokens[r] = t;
+        if (argmax) argmax[r] = t;
+    }
+    __syncthreads();
+    // draft comparison and commit: one thread per sequence
+    for (int s = threadIdx.x; s < B; s += 256) {
+        const int r0 = cu_q[s];
+        const int k = cu_q[s + 1] - r0 - 1;
+        const int* dr = drafts + (r0 - s);
+        int a = 0;
+        while (a < k && dr[a] == tokens[r0 + a]) ++a;
+        accept_len[s] = a;
+        next_token[s] = tokens[r0 + a];
+        if (seq_lens) seq_lens[s] = seq_lens[s] + a + 1;
+    }
+}
+
+cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_stride, int vocab, const int* drafts,
+                          const int* cu_q, int B, int total_q, int* accept_len, int* next_token, int* argmax,
+                          int* seq_lens, unsigned long long* partials, int chunks, unsigned int* ticket,
+                          cudaStream_t stream) {
+    const bool bf16 = logits_dtype == AGX_BF16;
+    const int esz = bf16 ? 2 : 4;
+    const int vec_elems = 16 / esz;
+    int chunk_elems = (vocab + chunks - 1) / chunks;
+    chunk_elems = (chunk_elems + vec_elems - 1) / vec_elems * vec_elems;  // chunk starts stay 16-byte aligned
+    const bool vec = ((uintptr_t)logits % 16 == 0) && ((row_stride * esz) % 16 == 0);
+    int* tokens = (int*)(partials + (size_t)total_q * chunks);
+    dim3 grid(chunks, total_q);
+#define AGX_LAUNCH_ACCEPT(BF, VEC)                                                                              \
+    accept_kernel<BF, VEC><<<grid, 256, 0, stream>>>(logits, row_stride, vocab, chunk_elems, chunks, drafts,    \
+                                                     cu_q, B, total_q, accept_len, next_token, argmax, seq_lens, \
+                                                     partials, tokens, ticket)
+    if (bf16) { if (vec) AGX_LAUNCH_ACCEPT(true, true); else AGX_LAUNCH_ACCEPT(true, false); }
+    else      { if (vec) AGX_LAUNCH_ACCEPT(false, true); else AGX_LAUNCH_ACCEPT(false, false); }
+#undef AGX_LAUNCH_ACCEPT
+    return cudaGetLastError();
+}
+
+}  // namespace agx

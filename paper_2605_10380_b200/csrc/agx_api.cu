@@ -1,0 +1,481 @@
+// C ABI of the agx library: argument checks, launch planning, dispatch.  No kernel lives here.
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "agx_internal.cuh"
+
+struct agx_handle {
+    agx_config cfg;
+    float scale;
+    int device;
+    int sm_count;
+    int* d_status;          // device status word
+    unsigned int* d_ticket; // ticket counter of the accept kernel (self-resetting)
+    int last_launches;
+    int small_min_split;    // tokens; tuning knob (env AGX_SMALL_MIN_SPLIT)
+    int force_mma_sync;     // route large q through the mma.sync kernel (env AGX_FORCE_MMA_SYNC)
+    std::vector<int32_t> cu_host;  // staging for agx_verify_step_host (lives until its final sync)
+    char err[512];
+};
+
+namespace {
+
+using namespace agx;
+
+agx_status fail(agx_handle* h, agx_status code, const char* fmt, ...) {
+    if (h) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(h->err, sizeof h->err, fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+
+agx_status cuda_fail(agx_handle* h, cudaError_t e, const char* what) {
+    return fail(h, AGX_E_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+inline bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+inline int round_up(long long v, int m) { return (int)((v + m - 1) / m * m); }
+inline int elem_size(int dtype) { return dtype == AGX_BF16 ? 2 : 4; }
+
+enum Kind { KIND_SMALL1 = 0, KIND_SMALL2, KIND_SMALL4, KIND_TILE, KIND_SIMT, KIND_COUNT };
+
+struct Launch {
+    Kind kind;
+    int total_rows;  // sum of q_len over the launch's sequences
+    int num_items;
+    std::vector<SeqPlan> seqs;
+};
+
+struct Plan {
+    std::vector<Launch> launches;
+    long long part_entries = 0;  // (row, head, split) partial slots
+    bool any_split = false;
+};
+
+// Decide kernel kind, KV splits and partial slots for every sequence (host lengths only).
+agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, int pt_stride, Plan& plan) {
+    const agx_config& c = h->cfg;
+    const int G = c.num_q_heads / c.num_kv_heads;
+    std::vector<int> row0(B + 1, 0);
+    for (int s = 0; s < B; ++s) {
+        if (Q[s] < 1) return fail(h, AGX_E_INVAL, "q_len[%d] = %d < 1", s, Q[s]);
+        if (P[s] < 0) return fail(h, AGX_E_INVAL, "prefix_len[%d] = %d < 0", s, P[s]);
+        if (pt_stride >= 0 && (long long)P[s] + Q[s] > (long long)pt_stride * kPage)
+            return fail(h, AGX_E_RANGE, "sequence %d: %d + %d tokens exceed the page table (%d pages)", s, P[s], Q[s], pt_stride);
+        if ((long long)row0[s] + Q[s] > (1 << 30)) return fail(h, AGX_E_RANGE, "too many rows");
+        row0[s + 1] = row0[s] + Q[s];
+    }
+    std::vector<int> groups[KIND_COUNT];
+    for (int s = 0; s < B; ++s) {
+        Kind k;
+        if (c.dtype == AGX_F32) k = KIND_SIMT;
+        else {
+            const int rows = Q[s] * G;
+            if (rows <= 16) k = KIND_SMALL1;
+            else if (rows <= 32) k = KIND_SMALL2;
+            else if (rows <= kSmallRowsMax || h->force_mma_sync || !attn_tile_available()) k = KIND_SMALL4;
+            else k = KIND_TILE;
+        }
+        groups[k].push_back(s);
+    }
+    for (int k = 0; k < KIND_COUNT; ++k) {
+        const std::vector<int>& seqs = groups[k];
+        if (seqs.empty()) continue;
+        // ---- choose the split length C (tokens) so that one wave of CTAs covers the group
+        int unit, min_split, target;
+        long long base_items = 0;  // items per split, summed over sequences
+        std::vector<long long> per_seq_items(seqs.size());
+        if (k == KIND_SIMT) { unit = 64; min_split = 256; target = h->sm_count * 16; }
+        else if (k == KIND_TILE) { unit = 128; min_split = 512; target = h->sm_count; }
+        else { unit = 64; min_split = h->small_min_split; target = h->sm_count * (k == KIND_SMALL4 ? 1 : 2); }
+        const int rows_per_chunk = (k == KIND_SMALL1) ? 16 : (k == KIND_SMALL2) ? 32 : (k == KIND_SMALL4) ? 64 : 256;
+        long long work = 0;
+        for (size_t n = 0; n < seqs.size(); ++n) {
+            const int s = seqs[n];
+            long long items;
+            if (k == KIND_SIMT) items = (long long)Q[s] * c.num_q_heads;
+            else items = (long long)c.num_kv_heads * ((Q[s] * G + rows_per_chunk - 1) / rows_per_chunk);
+            per_seq_items[n] = items;
+            base_items += items;
+            work += items * (P[s] + Q[s]);
+        }
+        int C = std::max(min_split, round_up((work + target - 1) / target, unit));
+        for (;;) {
+            long long items = 0;
+            for (size_t n = 0; n < seqs.size(); ++n) {
+                const int L = P[seqs[n]] + Q[seqs[n]];
+                items += per_seq_items[n] * ((L + C - 1) / C);
+            }
+            if (items <= std::max<long long>(target, base_items)) break;
+            C += unit;
+        }
+        // ---- emit launches of at most kMaxSeqs sequences
+        for (size_t a = 0; a < seqs.size(); a += kMaxSeqs) {
+            Launch ln;
+            ln.kind = (Kind)k;
+            ln.total_rows = 0;
+            ln.num_items = 0;
+            for (size_t n = a; n < std::min(seqs.size(), a + kMaxSeqs); ++n) {
+                const int s = seqs[n];
+                const int L = P[s] + Q[s];
+                SeqPlan sp;
+                sp.prefix_len = P[s];
+                sp.q_len = Q[s];
+                sp.q_row0 = row0[s];
+                sp.seq_index = s;
+                sp.nsplit = (L + C - 1) / C;
+                sp.split_tokens = round_up((L + sp.nsplit - 1) / sp.nsplit, unit);
+                sp.nsplit = (L + sp.split_tokens - 1) / sp.split_tokens;
+                sp.row_chunks = (k == KIND_SIMT) ? 1 : (Q[s] * G + rows_per_chunk - 1) / rows_per_chunk;
+                sp.item0 = ln.num_items;
+                sp.part_base = 0;
+                if (sp.nsplit > 1) {
+                    if (plan.part_entries + (long long)Q[s] * c.num_q_heads * sp.nsplit > 0x7FFFFFFFll)
+                        return fail(h, AGX_E_RANGE, "split partials exceed 2^31 entries");
+                    sp.part_base = (int)plan.part_entries;
+                    plan.part_entries += (long long)Q[s] * c.num_q_heads * sp.nsplit;
+                    plan.any_split = true;
+                }
+                const long long items = per_seq_items[n] * sp.nsplit;
+                if (ln.num_items + items > 0x7FFFFFFFll) return fail(h, AGX_E_RANGE, "too many work items");
+                ln.num_items += (int)items;
+                ln.total_rows += Q[s];
+                ln.seqs.push_back(sp);
+            }
+            plan.launches.push_back(std::move(ln));
+        }
+    }
+    return AGX_OK;
+}
+
+inline size_t part_ml_bytes(long long entries) { return (size_t)((entries * sizeof(float2) + 255) / 256 * 256); }
+
+}  // namespace
+
+extern "C" {
+
+const char* agx_status_string(agx_status s) {
+    switch (s) {
+        case AGX_OK: return "ok";
+        case AGX_E_INVAL: return "invalid argument";
+        case AGX_E_RANGE: return "argument out of range";
+        case AGX_E_UNSUPPORTED: return "unsupported configuration";
+        case AGX_E_CUDA: return "CUDA error";
+        case AGX_E_DEVICE: return "device status word set";
+        case AGX_E_NOMEM: return "out of memory";
+        default: return "unknown status";
+    }
+}
+
+const char* agx_last_error(const agx_handle* h) { return h ? h->err : "null handle"; }
+
+agx_status agx_create(const agx_config* cfg, agx_handle** out) {
+    if (!cfg || !out) return AGX_E_INVAL;
+    *out = nullptr;
+    if (cfg->num_q_heads < 1 || cfg->num_kv_heads < 1 || cfg->num_q_heads % cfg->num_kv_heads != 0) return AGX_E_INVAL;
+    if (cfg->page_size != kPage) return AGX_E_UNSUPPORTED;
+    if (cfg->dtype != AGX_BF16 && cfg->dtype != AGX_F32) return AGX_E_UNSUPPORTED;
+    if (cfg->dtype == AGX_BF16 && cfg->head_dim != 128) return AGX_E_UNSUPPORTED;
+    if (cfg->dtype == AGX_F32 && cfg->head_dim != 64 && cfg->head_dim != 128) return AGX_E_UNSUPPORTED;
+    if (!(cfg->scale >= 0.f)) return AGX_E_INVAL;
+    agx_handle* h = new (std::nothrow) agx_handle();
+    if (!h) return AGX_E_NOMEM;
+    h->cfg = *cfg;
+    h->scale = cfg->scale > 0.f ? cfg->scale : 1.0f / sqrtf((float)cfg->head_dim);
+    h->err[0] = 0;
+    h->last_launches = 0;
+    const char* env = getenv("AGX_SMALL_MIN_SPLIT");
+    h->small_min_split = env ? std::max(64, atoi(env) / 64 * 64) : 256;
+    env = getenv("AGX_FORCE_MMA_SYNC");
+    h->force_mma_sync = env ? atoi(env) : 0;
+    cudaError_t e = cudaGetDevice(&h->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
+    int major = 0;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, h->device);
+    if (e == cudaSuccess && major != 10) { delete h; return AGX_E_UNSUPPORTED; }
+    if (e == cudaSuccess) e = cudaMalloc((void**)&h->d_status, 256);
+    if (e != cudaSuccess) { delete h; return e == cudaErrorMemoryAllocation ? AGX_E_NOMEM : AGX_E_CUDA; }
+    e = cudaMemset(h->d_status, 0, 256);
+    if (e != cudaSuccess) { cudaFree(h->d_status); delete h; return AGX_E_CUDA; }
+    h->d_ticket = (unsigned int*)(h->d_status + 16);
+    *out = h;
+    return AGX_OK;
+}
+
+agx_status agx_destroy(agx_handle* h) {
+    if (!h) return AGX_E_INVAL;
+    cudaFree(h->d_status);
+    delete h;
+    return AGX_OK;
+}
+
+agx_status agx_kv_append(agx_handle* h, void* k_pool, void* v_pool, int64_t num_pages, const void* k_new,
+                         const void* v_new, const int32_t* page_table, int32_t pt_stride, const int32_t* prefix_len,
+                         const int32_t* cu_q, int32_t B, int32_t total_q, void* stream) {
+    if (!h) return AGX_E_INVAL;
+    h->last_launches = 0;
+    if (B < 0 || total_q < 0) return fail(h, AGX_E_INVAL, "negative B or total_q");
+    if (B == 0 || total_q == 0) return AGX_OK;
+    if (!k_pool || !v_pool || !k_new || !v_new || !page_table || !prefix_len || !cu_q)
+        return fail(h, AGX_E_INVAL, "null pointer");
+    if (!aligned(k_pool, 16) || !aligned(v_pool, 16) || !aligned(k_new, 16) || !aligned(v_new, 16))
+        return fail(h, AGX_E_INVAL, "K/V buffers must be 16-byte aligned");
+    if (num_pages < 1 || pt_stride < 1) return fail(h, AGX_E_INVAL, "num_pages and page_table_stride must be >= 1");
+    cudaError_t e = launch_kv_append(h->cfg.dtype, k_pool, v_pool, num_pages, k_new, v_new, page_table, pt_stride,
+                                     prefix_len, cu_q, B, total_q, h->cfg.num_kv_heads, h->cfg.head_dim, h->d_status,
+                                     (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "kv_append launch");
+    h->last_launches = 1;
+    return AGX_OK;
+}
+
+int64_t agx_attn_workspace_bytes(agx_handle* h, int32_t B, const int32_t* P, const int32_t* Q) {
+    if (!h) return AGX_E_INVAL;
+    if (B < 0) return fail(h, AGX_E_INVAL, "negative B");
+    if (B == 0) return 0;
+    if (!P || !Q) return fail(h, AGX_E_INVAL, "null pointer");
+    Plan plan;
+    agx_status st = make_plan(h, B, P, Q, -1, plan);
+    if (st != AGX_OK) return st;
+    if (plan.part_entries == 0) return 0;
+    return (int64_t)(part_ml_bytes(plan.part_entries) + (size_t)plan.part_entries * h->cfg.head_dim * sizeof(float));
+}
+
+agx_status agx_attn_prefixed(agx_handle* h, const void* q_block, const void* k_pool, const void* v_pool,
+                             int64_t num_pages, const int32_t* page_table, int32_t pt_stride, const int32_t* P,
+                             const int32_t* Q, int32_t B, void* out, float* lse, void* workspace,
+                             size_t workspace_bytes, void* stream_v) {
+    if (!h) return AGX_E_INVAL;
+    h->last_launches = 0;
+    if (B < 0) return fail(h, AGX_E_INVAL, "negative B");
+    if (B == 0) return AGX_OK;
+    if (!q_block || !k_pool || !v_pool || !page_table || !P || !Q || !out) return fail(h, AGX_E_INVAL, "null pointer");
+    if (!aligned(q_block, 16) || !aligned(out, 16) || !aligned(k_pool, 256) || !aligned(v_pool, 256))
+        return fail(h, AGX_E_INVAL, "q_block/out must be 16-byte and pools 256-byte aligned");
+    if (num_pages < 1 || pt_stride < 1) return fail(h, AGX_E_INVAL, "num_pages and page_table_stride must be >= 1");
+    Plan plan;
+    agx_status st = make_plan(h, B, P, Q, pt_stride, plan);
+    if (st != AGX_OK) return st;
+    const size_t need = plan.part_entries == 0 ? 0
+        : part_ml_bytes(plan.part_entries) + (size_t)plan.part_entries * h->cfg.head_dim * sizeof(float);
+    if (need > 0) {
+        if (!workspace || !aligned(workspace, 256)) return fail(h, AGX_E_INVAL, "workspace missing or not 256-byte aligned");
+        if (workspace_bytes < need) return fail(h, AGX_E_INVAL, "workspace too small: %zu < %zu", workspace_bytes, need);
+    }
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    AttnParams p;
+    memset(&p, 0, sizeof p);
+    p.q = q_block; p.k_pool = k_pool; p.v_pool = v_pool; p.page_table = page_table;
+    p.out = out; p.lse = lse;
+    p.part_ml = (float2*)workspace;
+    p.part_o = need ? (float*)((char*)workspace + part_ml_bytes(plan.part_entries)) : nullptr;
+    p.status = h->d_status;
+    p.num_pages = num_pages;
+    p.pt_stride = pt_stride;
+    p.hq = h->cfg.num_q_heads; p.hkv = h->cfg.num_kv_heads; p.head_dim = h->cfg.head_dim;
+    p.scale_log2 = h->scale * 1.4426950408889634f;
+    for (const Launch& ln : plan.launches) {
+        p.num_seqs = (int)ln.seqs.size();
+        p.num_items = ln.num_items;
+        bool split = false;
+        for (int i = 0; i < p.num_seqs; ++i) { p.seq[i] = ln.seqs[i]; split |= ln.seqs[i].nsplit > 1; }
+        cudaError_t e;
+        switch (ln.kind) {
+            case KIND_SMALL1: e = launch_attn_small_bf16(p, 1, stream); break;
+            case KIND_SMALL2: e = launch_attn_small_bf16(p, 2, stream); break;
+            case KIND_SMALL4: e = launch_attn_small_bf16(p, 4, stream); break;
+            case KIND_SIMT: e = launch_attn_simt_f32(p, stream); break;
+            default: return fail(h, AGX_E_UNSUPPORTED, "tile kernel not built");
+        }
+        if (e != cudaSuccess) return cuda_fail(h, e, "attention launch");
+        h->last_launches++;
+        if (split) {
+            e = launch_attn_combine(p, h->cfg.dtype, ln.total_rows, stream);
+            if (e != cudaSuccess) return cuda_fail(h, e, "combine launch");
+            h->last_launches++;
+        }
+    }
+    return AGX_OK;
+}
+
+static int accept_chunks(const agx_handle* h, int total_q, int vocab, int dtype) {
+    const int vec = 16 / elem_size(dtype);
+    const int target = 2 * h->sm_count;
+    int want = std::max(1, (target + total_q - 1) / total_q);
+    const int max_chunks = std::max(1, (vocab + 256 * vec * 2 - 1) / (256 * vec * 2));  // >= 2 vectors per thread
+    want = std::min(want, max_chunks);
+    int chunk_elems = (vocab + want - 1) / want;
+    chunk_elems = (chunk_elems + vec - 1) / vec * vec;
+    return (vocab + chunk_elems - 1) / chunk_elems;
+}
+
+int64_t agx_accept_workspace_bytes(agx_handle* h, int32_t total_q, int32_t vocab) {
+    if (!h) return AGX_E_INVAL;
+    if (total_q < 0 || vocab < 1) return fail(h, AGX_E_RANGE, "total_q < 0 or vocab < 1");
+    // chunk count depends on the logits dtype; size for the larger of the two
+    const int chunks = std::max(accept_chunks(h, std::max(total_q, 1), vocab, AGX_BF16),
+                                accept_chunks(h, std::max(total_q, 1), vocab, AGX_F32));
+    return (int64_t)total_q * chunks * 8 + (int64_t)total_q * 4 + 256;
+}
+
+agx_status agx_accept_greedy(agx_handle* h, const void* logits, int32_t logits_dtype, int64_t row_stride,
+                             int32_t vocab, const int32_t* drafts, const int32_t* cu_q, int32_t B, int32_t total_q,
+                             int32_t* accept_len, int32_t* next_token, int32_t* argmax, int32_t* seq_lens,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+    if (!h) return AGX_E_INVAL;
+    h->last_launches = 0;
+    if (B < 0 || total_q < 0) return fail(h, AGX_E_INVAL, "negative B or total_q");
+    if (B == 0) return AGX_OK;
+    if (total_q < B) return fail(h, AGX_E_INVAL, "total_q < B (every sequence has at least one row)");
+    if (logits_dtype != AGX_BF16 && logits_dtype != AGX_F32) return fail(h, AGX_E_UNSUPPORTED, "logits dtype");
+    if (vocab < 1 || row_stride < vocab) return fail(h, AGX_E_RANGE, "vocab < 1 or row_stride < vocab");
+    if (total_q > 65535) return fail(h, AGX_E_RANGE, "more than 65535 logits rows in one call");
+    if (!logits || !cu_q || !accept_len || !next_token || (!drafts && total_q > B)) return fail(h, AGX_E_INVAL, "null pointer");
+    if (!aligned(logits, elem_size(logits_dtype))) return fail(h, AGX_E_INVAL, "logits misaligned");
+    const int64_t need = agx_accept_workspace_bytes(h, total_q, vocab);
+    if (!workspace || !aligned(workspace, 8) || (int64_t)workspace_bytes < need)
+        return fail(h, AGX_E_INVAL, "accept workspace missing, misaligned or too small (%lld needed)", (long long)need);
+    const int chunks = accept_chunks(h, total_q, vocab, logits_dtype);
+    cudaError_t e = launch_accept(logits, logits_dtype, row_stride, vocab, drafts, cu_q, B, total_q, accept_len,
+                                  next_token, argmax, seq_lens, (unsigned long long*)workspace, chunks, h->d_ticket,
+                                  (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "accept launch");
+    h->last_launches = 1;
+    return AGX_OK;
+}
+
+agx_status agx_get_status(agx_handle* h, void* stream, int32_t* device_status) {
+    if (!h || !device_status) return AGX_E_INVAL;
+    int v = 0;
+    cudaError_t e = cudaMemcpyAsync(&v, h->d_status, sizeof v, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "status read");
+    *device_status = v;
+    if (v != 0) {
+        e = cudaMemsetAsync(h->d_status, 0, sizeof(int), (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(h, e, "status clear");
+        return fail(h, AGX_E_DEVICE, "device status 0x%x", v);
+    }
+    return AGX_OK;
+}
+
+int32_t agx_last_launch_count(const agx_handle* h) { return h ? h->last_launches : 0; }
+
+}  // extern "C"
+
+namespace {
+struct HostStepLayout {
+    size_t q, k, v, out, logits, drafts, prefix, cu, acc, next, seqlen, attn_ws, accept_ws, total;
+    size_t q_bytes, kv_bytes, logits_bytes, attn_ws_bytes, accept_ws_bytes;
+    int total_q;
+};
+agx_status host_step_layout(agx_handle* h, int B, const int32_t* P, const int32_t* Q, int logits_dtype,
+                            int64_t row_stride, int vocab, HostStepLayout& L) {
+    if (B < 1 || !P || !Q) return fail(h, AGX_E_INVAL, "B < 1 or null lengths");
+    if (logits_dtype != AGX_BF16 && logits_dtype != AGX_F32) return fail(h, AGX_E_UNSUPPORTED, "logits dtype");
+    if (vocab < 1 || row_stride < vocab) return fail(h, AGX_E_RANGE, "vocab < 1 or row_stride < vocab");
+    long long tq = 0;
+    for (int s = 0; s < B; ++s) {
+        if (Q[s] < 1) return fail(h, AGX_E_INVAL, "q_len[%d] = %d < 1", s, Q[s]);
+        tq += Q[s];
+    }
+    if (tq > 65535) return fail(h, AGX_E_RANGE, "more than 65535 rows in one host step");
+    const int64_t aws = agx_attn_workspace_bytes(h, B, P, Q);
+    if (aws < 0) return (agx_status)aws;
+    const int64_t cws = agx_accept_workspace_bytes(h, (int)tq, vocab);
+    if (cws < 0) return (agx_status)cws;
+    const size_t es = elem_size(h->cfg.dtype);
+    L.total_q = (int)tq;
+    L.q_bytes = (size_t)tq * h->cfg.num_q_heads * h->cfg.head_dim * es;
+    L.kv_bytes = (size_t)tq * h->cfg.num_kv_heads * h->cfg.head_dim * es;
+    L.logits_bytes = (size_t)tq * row_stride * elem_size(logits_dtype);
+    L.attn_ws_bytes = (size_t)aws;
+    L.accept_ws_bytes = (size_t)cws;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 255) / 256 * 256; return o; };
+    L.q = take(L.q_bytes); L.k = take(L.kv_bytes); L.v = take(L.kv_bytes); L.out = take(L.q_bytes);
+    L.logits = take(L.logits_bytes); L.drafts = take((size_t)(tq - B) * 4 + 4);
+    L.prefix = take((size_t)B * 4); L.cu = take((size_t)(B + 1) * 4);
+    L.acc = take((size_t)B * 4); L.next = take((size_t)B * 4); L.seqlen = take((size_t)B * 4);
+    L.attn_ws = take(L.attn_ws_bytes); L.accept_ws = take(L.accept_ws_bytes);
+    L.total = off;
+    return AGX_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int64_t agx_verify_step_host_workspace_bytes(agx_handle* h, int32_t B, const int32_t* P, const int32_t* Q,
+                                             int32_t logits_dtype, int64_t row_stride, int32_t vocab) {
+    if (!h) return AGX_E_INVAL;
+    HostStepLayout L;
+    agx_status st = host_step_layout(h, B, P, Q, logits_dtype, row_stride, vocab, L);
+    return st != AGX_OK ? (int64_t)st : (int64_t)L.total;
+}
+
+agx_status agx_verify_step_host(agx_handle* h, void* k_pool, void* v_pool, int64_t num_pages,
+                                const int32_t* page_table, int32_t pt_stride, const int32_t* P, const int32_t* Q,
+                                int32_t B, const void* h_q, const void* h_k, const void* h_v, const void* h_logits,
+                                int32_t logits_dtype, int64_t row_stride, int32_t vocab, const int32_t* h_drafts,
+                                void* h_out, int32_t* h_accept, int32_t* h_next, int32_t* h_seq_lens, void* workspace,
+                                size_t workspace_bytes, void* stream_v) {
+    if (!h) return AGX_E_INVAL;
+    HostStepLayout L;
+    agx_status st = host_step_layout(h, B, P, Q, logits_dtype, row_stride, vocab, L);
+    if (st != AGX_OK) return st;
+    if (!k_pool || !v_pool || !page_table || !h_q || !h_k || !h_v || !h_logits || !h_out || !h_accept || !h_next ||
+        !h_seq_lens || (!h_drafts && L.total_q > B))
+        return fail(h, AGX_E_INVAL, "null pointer");
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < L.total)
+        return fail(h, AGX_E_INVAL, "host-step workspace missing, misaligned or too small (%zu needed)", L.total);
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    char* ws = (char*)workspace;
+    std::vector<int32_t>& cu = h->cu_host;  // outlives the asynchronous copy (the call ends with a sync)
+    cu.assign(B + 1, 0);
+    for (int s = 0; s < B; ++s) cu[s + 1] = cu[s] + Q[s];
+    cudaError_t e = cudaSuccess;
+    auto h2d = [&](size_t off, const void* src, size_t bytes) {
+        if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(ws + off, src, bytes, cudaMemcpyHostToDevice, stream);
+    };
+    h2d(L.q, h_q, L.q_bytes); h2d(L.k, h_k, L.kv_bytes); h2d(L.v, h_v, L.kv_bytes);
+    h2d(L.logits, h_logits, L.logits_bytes);
+    h2d(L.drafts, h_drafts, (size_t)(L.total_q - B) * 4);
+    h2d(L.prefix, P, (size_t)B * 4);
+    h2d(L.seqlen, P, (size_t)B * 4);
+    h2d(L.cu, cu.data(), (size_t)(B + 1) * 4);
+    if (e != cudaSuccess) return cuda_fail(h, e, "host step: upload");
+    int launches = 0;
+    st = agx_kv_append(h, k_pool, v_pool, num_pages, ws + L.k, ws + L.v, page_table, pt_stride,
+                       (const int32_t*)(ws + L.prefix), (const int32_t*)(ws + L.cu), B, L.total_q, stream);
+    if (st != AGX_OK) return st;
+    launches += h->last_launches;
+    st = agx_attn_prefixed(h, ws + L.q, k_pool, v_pool, num_pages, page_table, pt_stride, P, Q, B, ws + L.out, nullptr,
+                           L.attn_ws_bytes ? ws + L.attn_ws : nullptr, L.attn_ws_bytes, stream);
+    if (st != AGX_OK) return st;
+    launches += h->last_launches;
+    st = agx_accept_greedy(h, ws + L.logits, logits_dtype, row_stride, vocab, (const int32_t*)(ws + L.drafts),
+                           (const int32_t*)(ws + L.cu), B, L.total_q, (int32_t*)(ws + L.acc), (int32_t*)(ws + L.next),
+                           nullptr, (int32_t*)(ws + L.seqlen), ws + L.accept_ws, L.accept_ws_bytes, stream);
+    if (st != AGX_OK) return st;
+    launches += h->last_launches;
+    auto d2h = [&](void* dst, size_t off, size_t bytes) {
+        if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, ws + off, bytes, cudaMemcpyDeviceToHost, stream);
+    };
+    d2h(h_out, L.out, L.q_bytes);
+    d2h(h_accept, L.acc, (size_t)B * 4); d2h(h_next, L.next, (size_t)B * 4); d2h(h_seq_lens, L.seqlen, (size_t)B * 4);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "host step: download");
+    h->last_launches = launches;
+    return AGX_OK;
+}
+
+}  // extern "C"

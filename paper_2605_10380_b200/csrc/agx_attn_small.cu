@@ -1,0 +1,502 @@
+// Small-q attention over a paged KV cache: the verify block of speculative decoding (q = N + 1
+// rows, Sec. 2.3) and plain decode (q = 1, the selective fallback of Sec. 4.3).
+//
+// The step is HBM-bound: every K and V byte of the sequence is read once and meets only q * G
+// query rows (G = Hq / Hkv), i.e. q * G flop per KV byte.  That is above what the fp32 FMA pipes
+// sustain at HBM speed once q * G > ~8, so the q * G rows of one KV head are packed into the M
+// dimension of warp-level bf16 tensor-core MMAs (m16n8k16, fp32 accumulate): the kernel stays
+// bandwidth-bound and verifying 8 tokens costs the same bytes as decoding 1.
+//
+// Work item = (sequence, KV head, KV split).  A CTA of 4 * MT warps: warp (mt, kg) owns query rows
+// [16 mt, 16 mt + 16) and, in every 64-token stage, page kg.  K/V pages stream through a
+// multi-stage cp.async ring (16-byte chunks, XOR-swizzled rows so ldmatrix is conflict-free); the
+// four KV groups keep private online-softmax states that are merged through shared memory at the
+// end.  Splits write fp32 (m, l, O) partials; a combine kernel merges them in fixed order, so
+// results are bit-reproducible run to run.
+#include <math.h>
+
+#include "agx_internal.cuh"
+
+namespace agx {
+
+namespace {
+
+constexpr int kD = 128;                    // head dim of the bf16 kernels
+constexpr int kRowBytes = kD * 2;          // one (token, head) row
+constexpr int kKW = 4;                     // KV groups (pages per stage)
+constexpr int kStageTokens = kKW * kPage;  // 64
+constexpr int kStageBytes = 2 * kStageTokens * kRowBytes;  // K + V = 32 KB
+constexpr int kMergeStride = 136;          // floats per merged row (conflict-free float2 stores)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+// D(16x8, f32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// byte offset of 16-byte chunk `ch` (0..15) of row `r` in a [rows][256 B] tile, XOR-swizzled
+__device__ __forceinline__ uint32_t swz(int r, int ch) { return (uint32_t)(r * kRowBytes + ((ch ^ (r & 7)) << 4)); }
+
+// Locate the work item: sequence plan + (kv head, split).
+__device__ __forceinline__ int find_seq(const AttnParams& p, int item) {
+    int s = 0;
+#pragma unroll 1
+    for (int i = 1; i < p.num_seqs; ++i)
+        if (p.seq[i].item0 <= item) s = i;
+    return s;
+}
+
+}  // namespace
+
+template <int MT, int NS>
+__global__ void __launch_bounds__(128 * MT, (MT <= 2) ? 2 : 1)
+attn_small_bf16_kernel(const __grid_constant__ AttnParams p) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    constexpr int kThreads = 128 * MT;
+    constexpr int kQBytes = MT * 16 * kRowBytes;
+    unsigned char* q_smem = smem;
+    unsigned char* ring = smem + kQBytes;
+
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    const int mt = warp % MT;
+    const int kg = warp / MT;
+
+    const int si = find_seq(p, blockIdx.x);
+    const SeqPlan sp = p.seq[si];
+    int local = blockIdx.x - sp.item0;  // ((g * row_chunks) + rc) * nsplit + split
+    const int split = local % sp.nsplit;
+    local /= sp.nsplit;
+    const int rc = local % sp.row_chunks;
+    const int g = local / sp.row_chunks;
+    const int G = p.hq / p.hkv;
+    const int P = sp.prefix_len;
+    const int q = sp.q_len;
+    const int rows = q * G;          // query rows of this KV head, r = i * G + (h % G)
+    const int row0 = rc * 16 * MT;   // first row of this CTA's chunk
+    // the chunk's last row sees tokens 0 .. P + i_last
+    const int vis_end = P + min(q - 1, (row0 + 16 * MT - 1) / G) + 1;
+    const int tok_begin = split * sp.split_tokens;
+    const int tok_end = min(vis_end, tok_begin + sp.split_tokens);
+    const int n_stages = max(0, (tok_end - tok_begin + kStageTokens - 1) / kStageTokens);
+    const int* pt_row = p.page_table + (long long)sp.seq_index * p.pt_stride;
+    const unsigned char* k_pool = (const unsigned char*)p.k_pool;
+    const unsigned char* v_pool = (const unsigned char*)p.v_pool;
+
+    // ---- stage loader: 2048 16-byte chunks (K then V), each thread 2048 / kThreads of them
+    auto load_stage = [&](int stage) {
+        if (stage < n_stages) {
+            unsigned char* buf = ring + (stage % NS) * kStageBytes;
+            const int tok0 = tok_begin + stage * kStageTokens;
+#pragma unroll
+            for (int it = 0; it < 2048 / kThreads; ++it) {
+                const int c = it * kThreads + tid;
+                const int kv = c >> 10;
+                const int pg = (c >> 8) & 3;
+                const int r = (c >> 4) & 15;
+                const int ch = c & 15;
+                const int tok = tok0 + pg * kPage + r;
+                bool valid = tok < tok_end;
+                long long page = 0;
+                if (valid) {
+                    page = __ldg(pt_row + (tok >> 4));
+                    if (page < 0 || page >= p.num_pages) {
+                        valid = false;
+                        page = 0;
+                        atomicOr(p.status, AGX_DEV_BAD_PAGE);
+                    }
+                }
+                const unsigned char* src = (kv ? v_pool : k_pool) +
+                                           (((page * p.hkv + g) * kPage + r) * (long long)kRowBytes + ch * 16);
+                const uint32_t dst = smem_u32(buf + kv * (kStageTokens * kRowBytes) + pg * (kPage * kRowBytes)) + swz(r, ch);
+                cp_async16(dst, src, valid ? 16 : 0);
+            }
+        }
+        cp_async_commit();
+    };
+
+    // ---- Q tile -> shared (rows beyond q*G are zero), then A fragments in registers
+    for (int c = tid; c < MT * 16 * 16; c += kThreads) {
+        const int r = c >> 4, ch = c & 15;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (row0 + r < rows) {
+            const int i = (row0 + r) / G, hg = (row0 + r) - i * G;
+            const long long off = ((long long)(sp.q_row0 + i) * p.hq + g * G + hg) * kRowBytes + ch * 16;
+            v = __ldg((const uint4*)((const unsigned char*)p.q + off));
+        }
+        *(uint4*)(q_smem + swz(r, ch)) = v;
+    }
+#pragma unroll
+    for (int s = 0; s < NS - 1; ++s) load_stage(s);
+    __syncthreads();  // Q tile visible
+
+    uint32_t qa[8][4];
+    {
+        const int r = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const int ch = ks * 2 + (lane >> 4);
+            ldmatrix_x4(qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], smem_u32(q_smem) + swz(r, ch));
+        }
+    }
+
+    float o[16][4];
+#pragma unroll
+    for (int n = 0; n < 16; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+    float m_run[2] = {-INFINITY, -INFINITY};
+    float l_run[2] = {0.f, 0.f};
+
+    // row limits (last visible token) for the two rows this thread holds
+    int limit[2];
+    {
+        const int rA = row0 + mt * 16 + (lane >> 2);
+        limit[0] = P + min(rA / G, q - 1);
+        limit[1] = P + min((rA + 8) / G, q - 1);
+    }
+
+    for (int stage = 0; stage < n_stages; ++stage) {
+        cp_async_wait<NS - 2>();
+        __syncthreads();             // stage data visible to all; ring slot (stage-1) % NS is free
+        load_stage(stage + NS - 1);  // refill it
+
+        const int tok0 = tok_begin + stage * kStageTokens + kg * kPage;
+        if (tok0 < tok_end) {
+            const unsigned char* buf = ring + (stage % NS) * kStageBytes;
+            const uint32_t k_base = smem_u32(buf + kg * (kPage * kRowBytes));
+            const uint32_t v_base = k_base + kStageTokens * kRowBytes;
+
+            // S = Q K^T for 16 tokens: two n-tiles of 8 tokens
+            float s[2][4];
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) { s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f; }
+#pragma unroll
+            for (int kp = 0; kp < 4; ++kp) {
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) {
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4(b0, b1, b2, b3, k_base + swz(nt * 8 + (lane & 7), kp * 4 + (lane >> 3)));
+                    mma_bf16(s[nt], qa[2 * kp], b0, b1);
+                    mma_bf16(s[nt], qa[2 * kp + 1], b2, b3);
+                }
+            }
+            // scale to log2 units, mask the causal edge / the end of the split
+            const bool need_mask = (tok0 + kPage - 1 > P) || (tok0 + kPage > tok_end);
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float v = s[nt][e] * p.scale_log2;
+                    if (need_mask) {
+                        const int tok = tok0 + nt * 8 + 2 * (lane & 3) + (e & 1);
+                        if (tok > limit[e >> 1] || tok >= tok_end) v = -INFINITY;
+                    }
+                    s[nt][e] = v;
+                }
+            }
+            // online softmax for rows A (e = 0,1) and B (e = 2,3)
+            float corr[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                float mx = fmaxf(fmaxf(s[0][2 * h], s[0][2 * h + 1]), fmaxf(s[1][2 * h], s[1][2 * h + 1]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
+                const float m_new = fmaxf(m_run[h], mx);
+                const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
+                corr[h] = exp2f(m_run[h] - m_ref);
+                m_run[h] = m_new;
+                float sum = 0.f;
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) {
+                    s[nt][2 * h] = exp2f(s[nt][2 * h] - m_ref);
+                    s[nt][2 * h + 1] = exp2f(s[nt][2 * h + 1] - m_ref);
+                    sum += s[nt][2 * h] + s[nt][2 * h + 1];
+                }
+                l_run[h] = l_run[h] * corr[h] + sum;
+            }
+            if (__any_sync(0xFFFFFFFFu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+                for (int n = 0; n < 16; ++n) {
+                    o[n][0] *= corr[0]; o[n][1] *= corr[0];
+                    o[n][2] *= corr[1]; o[n][3] *= corr[1];
+                }
+            }
+            // O += P V
+            uint32_t pa[4];
+            pa[0] = pack_bf16(s[0][0], s[0][1]);
+            pa[1] = pack_bf16(s[0][2], s[0][3]);
+            pa[2] = pack_bf16(s[1][0], s[1][1]);
+            pa[3] = pack_bf16(s[1][2], s[1][3]);
+#pragma unroll
+            for (int cp = 0; cp < 8; ++cp) {
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4_trans(b0, b1, b2, b3,
+                                  v_base + swz((lane & 7) + ((lane >> 3) & 1) * 8, cp * 2 + (lane >> 4)));
+                mma_bf16(o[2 * cp], pa, b0, b1);
+                mma_bf16(o[2 * cp + 1], pa, b2, b3);
+            }
+        }
+    }
+    cp_async_wait<0>();
+    __syncthreads();  // ring is dead: reuse it for the cross-group merge
+
+    // ---- merge the 4 KV groups of each m-tile through shared memory
+    float* merge_o = (float*)ring;                                    // [MT*4][16][kMergeStride]
+    float2* merge_ml = (float2*)(ring + MT * kKW * 16 * kMergeStride * 4);  // [MT*4][16]
+    {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 1);
+            l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 2);
+        }
+        float* mo = merge_o + (size_t)(mt * kKW + kg) * 16 * kMergeStride;
+        const int rA = lane >> 2;
+#pragma unroll
+        for (int n = 0; n < 16; ++n) {
+            const int col = n * 8 + 2 * (lane & 3);
+            *(float2*)(mo + rA * kMergeStride + col) = make_float2(o[n][0], o[n][1]);
+            *(float2*)(mo + (rA + 8) * kMergeStride + col) = make_float2(o[n][2], o[n][3]);
+        }
+        if ((lane & 3) == 0) {
+            merge_ml[(mt * kKW + kg) * 16 + rA] = make_float2(m_run[0], l_run[0]);
+            merge_ml[(mt * kKW + kg) * 16 + rA + 8] = make_float2(m_run[1], l_run[1]);
+        }
+    }
+    __syncthreads();
+
+    // each thread finishes 4 consecutive columns of one row at a time
+    for (int idx = tid; idx < MT * 16 * (kD / 4); idx += kThreads) {
+        const int r = idx / (kD / 4);
+        const int c4 = (idx - r * (kD / 4)) * 4;
+        if (row0 + r >= rows) continue;
+        const int rm = r >> 4, rr = r & 15;
+        float m_all = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < kKW; ++k) m_all = fmaxf(m_all, merge_ml[(rm * kKW + k) * 16 + rr].x);
+        float l_all = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < kKW; ++k) {
+            const float2 ml = merge_ml[(rm * kKW + k) * 16 + rr];
+            const float w = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m_all);
+            l_all += ml.y * w;
+            const float4 v = *(const float4*)(merge_o + ((size_t)(rm * kKW + k) * 16 + rr) * kMergeStride + c4);
+            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+        }
+        const int i = (row0 + r) / G, hg = (row0 + r) - i * G;
+        const int h = g * G + hg;
+        if (sp.nsplit == 1) {
+            const float inv = 1.f / l_all;
+            const long long off = ((long long)(sp.q_row0 + i) * p.hq + h) * kD + c4;
+            uint2 packed;
+            packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+            packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+            *(uint2*)((__nv_bfloat16*)p.out + off) = packed;
+            if (p.lse && c4 == 0) p.lse[(long long)(sp.q_row0 + i) * p.hq + h] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+        } else {
+            const long long e = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit + split;
+            *(float4*)(p.part_o + e * kD + c4) = acc;
+            if (c4 == 0) p.part_ml[e] = make_float2(m_all, l_all);
+        }
+    }
+}
+
+// --------------------------------------------------------------------------------------------
+// Scalar kernel for fp32 pools (any q; d = 64 or 128).  CTA = 4 warps on one (sequence, row, head,
+// split); a warp takes every 4th token, lanes split the head dim, dot products reduce by shuffle.
+template <int D>
+__global__ void __launch_bounds__(128)
+attn_simt_f32_kernel(const __grid_constant__ AttnParams p) {
+    constexpr int kPer = D / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int si = find_seq(p, blockIdx.x);
+    const SeqPlan sp = p.seq[si];
+    int local = blockIdx.x - sp.item0;  // ((i * Hq) + h) * nsplit + split
+    const int split = local % sp.nsplit;
+    local /= sp.nsplit;
+    const int h = local % p.hq;
+    const int i = local / p.hq;
+    const int G = p.hq / p.hkv;
+    const int g = h / G;
+    const int tok_begin = split * sp.split_tokens;
+    const int tok_end = min(sp.prefix_len + i + 1, tok_begin + sp.split_tokens);  // causal limit for row i
+    const int* pt_row = p.page_table + (long long)sp.seq_index * p.pt_stride;
+    const float* kp = (const float*)p.k_pool;
+    const float* vp = (const float*)p.v_pool;
+
+    float qv[kPer], acc[kPer];
+    const float* qrow = (const float*)p.q + ((long long)(sp.q_row0 + i) * p.hq + h) * D;
+#pragma unroll
+    for (int c = 0; c < kPer; ++c) { qv[c] = qrow[lane + 32 * c] * p.scale_log2; acc[c] = 0.f; }
+    float m = -INFINITY, l = 0.f;
+    for (int tok = tok_begin + warp; tok < tok_end; tok += 4) {
+        long long page = __ldg(pt_row + (tok >> 4));
+        if (page < 0 || page >= p.num_pages) {
+            if (lane == 0) atomicOr(p.status, AGX_DEV_BAD_PAGE);
+            continue;
+        }
+        const long long base = ((page * p.hkv + g) * kPage + (tok & 15)) * (long long)D;
+        float dot = 0.f;
+#pragma unroll
+        for (int c = 0; c < kPer; ++c) dot += qv[c] * kp[base + lane + 32 * c];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, off);
+        const float m_new = fmaxf(m, dot);
+        const float corr = exp2f(m - m_new);
+        const float w = exp2f(dot - m_new);
+        l = l * corr + w;
+#pragma unroll
+        for (int c = 0; c < kPer; ++c) acc[c] = acc[c] * corr + w * vp[base + lane + 32 * c];
+        m = m_new;
+    }
+    __shared__ float sm_o[4][D];
+    __shared__ float2 sm_ml[4];
+#pragma unroll
+    for (int c = 0; c < kPer; ++c) sm_o[warp][lane + 32 * c] = acc[c];
+    if (lane == 0) sm_ml[warp] = make_float2(m, l);
+    __syncthreads();
+    for (int c = threadIdx.x; c < D; c += 128) {
+        float m_all = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) m_all = fmaxf(m_all, sm_ml[k].x);
+        float l_all = 0.f, a = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float w = (sm_ml[k].x == -INFINITY) ? 0.f : exp2f(sm_ml[k].x - m_all);
+            l_all += sm_ml[k].y * w;
+            a += sm_o[k][c] * w;
+        }
+        if (sp.nsplit == 1) {
+            ((float*)p.out)[((long long)(sp.q_row0 + i) * p.hq + h) * D + c] = a / l_all;
+            if (p.lse && c == 0) p.lse[(long long)(sp.q_row0 + i) * p.hq + h] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+        } else {
+            const long long e = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit + split;
+            p.part_o[e * D + c] = a;
+            if (c == 0) p.part_ml[e] = make_float2(m_all, l_all);
+        }
+    }
+}
+
+// --------------------------------------------------------------------------------------------
+// Combine: out[row, h] = sum_k O_k 2^(m_k - m) / sum_k l_k 2^(m_k - m), splits in index order.
+// One warp per (row, head); lanes own 4 consecutive floats of each 128-wide chunk.
+template <bool kBf16Out>
+__global__ void __launch_bounds__(128)
+attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
+    const int lane = threadIdx.x & 31;
+    const int rh = blockIdx.x * 4 + (threadIdx.x >> 5);  // index over (local row, head) of the launch's sequences
+    if (rh >= total_rows * p.hq) return;
+    const int lrow = rh / p.hq, h = rh - lrow * p.hq;
+    // sequences are laid out back to back in launch-local row order
+    int si = 0, acc_rows = 0;
+#pragma unroll 1
+    for (int s = 0; s < p.num_seqs; ++s) {
+        if (lrow >= acc_rows && lrow < acc_rows + p.seq[s].q_len) { si = s; break; }
+        acc_rows += p.seq[s].q_len;
+    }
+    const SeqPlan sp = p.seq[si];
+    if (sp.nsplit == 1) return;  // written directly by the attention kernel
+    const int i = lrow - acc_rows;
+    const long long e0 = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit;
+    float m_all = -INFINITY;
+    for (int k = 0; k < sp.nsplit; ++k) m_all = fmaxf(m_all, p.part_ml[e0 + k].x);
+    const int D = p.head_dim;
+    float l_all = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int c4 = lane * 4;
+    for (int k = 0; k < sp.nsplit; ++k) {
+        const float2 ml = p.part_ml[e0 + k];
+        const float w = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m_all);
+        l_all += ml.y * w;
+        if (c4 < D) {
+            const float4 v = *(const float4*)(p.part_o + (e0 + k) * D + c4);
+            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+        }
+    }
+    const float inv = 1.f / l_all;
+    const long long off = ((long long)(sp.q_row0 + i) * p.hq + h) * D + c4;
+    if (c4 < D) {
+        if (kBf16Out) {
+            uint2 packed;
+            packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+            packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+            *(uint2*)((__nv_bfloat16*)p.out + off) = packed;
+        } else {
+            *(float4*)((float*)p.out + off) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+        }
+    }
+    if (p.lse && lane == 0) p.lse[(long long)(sp.q_row0 + i) * p.hq + h] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+}
+
+// --------------------------------------------------------------------------------------------
+namespace {
+template <int MT, int NS>
+cudaError_t launch_small(const AttnParams& p, cudaStream_t stream) {
+    constexpr int kQBytes = MT * 16 * kRowBytes;
+    constexpr int kMergeBytes = MT * kKW * 16 * (kMergeStride * 4 + 8);
+    constexpr int kRing = NS * kStageBytes;
+    constexpr int kSmem = kQBytes + (kRing > kMergeBytes ? kRing : kMergeBytes);
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(attn_small_bf16_kernel<MT, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    attn_small_bf16_kernel<MT, NS><<<p.num_items, 128 * MT, kSmem, stream>>>(p);
+    return cudaGetLastError();
+}
+}  // namespace
+
+int attn_small_bf16_kv_tile() { return kStageTokens; }
+bool attn_tile_available() { return false; }
+
+cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, cudaStream_t stream) {
+    if (p.num_items == 0) return cudaSuccess;
+    switch (mt) {
+        case 1: return launch_small<1, 3>(p, stream);
+        case 2: return launch_small<2, 3>(p, stream);
+        case 4: return launch_small<4, 5>(p, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+cudaError_t launch_attn_simt_f32(const AttnParams& p, cudaStream_t stream) {
+    if (p.num_items == 0) return cudaSuccess;
+    if (p.head_dim == 64) attn_simt_f32_kernel<64><<<p.num_items, 128, 0, stream>>>(p);
+    else if (p.head_dim == 128) attn_simt_f32_kernel<128><<<p.num_items, 128, 0, stream>>>(p);
+    else return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, cudaStream_t stream) {
+    const long long n = (long long)total_rows * p.hq;
+    if (n == 0) return cudaSuccess;
+    const int blocks = (int)((n + 3) / 4);
+    if (dtype == AGX_BF16) attn_combine_kernel<true><<<blocks, 128, 0, stream>>>(p, total_rows);
+    else attn_combine_kernel<false><<<blocks, 128, 0, stream>>>(p, total_rows);
+    return cudaGetLastError();
+}
+
+}  // namespace agx

@@ -1,0 +1,72 @@
+// Internal declarations shared by the agx CUDA sources (not part of the C ABI).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "agx.h"
+
+namespace agx {
+
+constexpr int kPage = 16;          // tokens per KV page
+constexpr int kMaxSeqs = 48;       // sequences per attention launch (plans travel as kernel arguments)
+constexpr int kSmallRowsMax = 64;  // q_len * G above this goes to the tile kernel
+
+// Per-sequence launch plan, built on the host from the host lengths.
+struct SeqPlan {
+    int prefix_len;    // P
+    int q_len;         // q
+    int q_row0;        // first row of the sequence in q_block / out
+    int seq_index;     // row of the page table
+    int nsplit;        // KV splits
+    int row_chunks;    // query-row chunks per KV head (1 for verify blocks)
+    int split_tokens;  // tokens per split (multiple of the kernel's KV tile)
+    int item0;         // first work item of this sequence in the launch
+    int part_base;     // first partial entry; entry = part_base + (i*Hq + h)*nsplit + split
+};
+
+struct AttnParams {
+    const void* q;
+    const void* k_pool;
+    const void* v_pool;
+    const int* page_table;
+    void* out;
+    float* lse;
+    float* part_o;   // [entries][head_dim] fp32, un-normalised, relative to part_ml.x
+    float2* part_ml; // [entries] (running max in log2 units, sum)
+    int* status;
+    long long num_pages;
+    int pt_stride;
+    int hq, hkv, head_dim;
+    int num_seqs;
+    int num_items;
+    float scale_log2;  // scale * log2(e)
+    SeqPlan seq[kMaxSeqs];
+};
+
+// Launchers (each returns the cudaError_t of its launch).
+cudaError_t launch_kv_append(int dtype, void* k_pool, void* v_pool, long long num_pages, const void* k_new,
+                             const void* v_new, const int* page_table, int pt_stride, const int* prefix_len,
+                             const int* cu_q, int B, int total_q, int hkv, int head_dim, int* status,
+                             cudaStream_t stream);
+
+// Small-q split-KV kernel (bf16, d = 128, tensor-core mma.sync); mt = m-tiles of 16 rows (1, 2, 4).
+cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, cudaStream_t stream);
+int attn_small_bf16_kv_tile();  // tokens per pipeline stage
+// Scalar fp32-math kernel for AGX_F32 pools (any q, d in {64, 128}).
+cudaError_t launch_attn_simt_f32(const AttnParams& p, cudaStream_t stream);
+// Merge of split partials into out / lse.
+cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, cudaStream_t stream);
+
+bool attn_tile_available();
+// Large-q tensor-core tile kernel (bf16, d = 128, tcgen05 + TMEM + TMA).
+struct TileLaunch;  // opaque to other translation units
+cudaError_t launch_attn_tile_bf16(const AttnParams& p, const void* tmap_k, const void* tmap_v, int sm_count,
+                                  cudaStream_t stream);
+
+cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_stride, int vocab, const int* drafts,
+                          const int* cu_q, int B, int total_q, int* accept_len, int* next_token, int* argmax,
+                          int* seq_lens, unsigned long long* partials, int chunks, unsigned int* ticket,
+                          cudaStream_t stream);
+
+}  // namespace agx

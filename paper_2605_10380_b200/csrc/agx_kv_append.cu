@@ -1,0 +1,60 @@
+// KV append: scatter the block's K/V rows into the sequences' pages (Sec. 2.3: prefill fills the
+// KV cache; with prefix caching only the uncached suffix is written, behind the cached prefix).
+//
+// HBM-bound copy: 2 * 2 * rows * Hkv * d * elem bytes (read + write, K and V).  One thread moves
+// 16 bytes of K and 16 bytes of V; a (token, kv head) row is `vec_per_row` consecutive threads, so
+// loads and stores are fully coalesced 128-bit accesses.
+#include "agx_internal.cuh"
+
+namespace agx {
+
+__global__ void __launch_bounds__(256)
+kv_append_kernel(uint4* __restrict__ k_pool, uint4* __restrict__ v_pool, long long num_pages,
+                 const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                 const int* __restrict__ page_table, int pt_stride, const int* __restrict__ prefix_len,
+                 const int* __restrict__ cu_q, int B, int total_q, int hkv, int vec_per_row, int* status) {
+    const long long n_vec = (long long)total_q * hkv * vec_per_row;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < n_vec;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(idx % vec_per_row);
+        const long long row = idx / vec_per_row;  // (token, kv head)
+        const int g = (int)(row % hkv);
+        const int r = (int)(row / hkv);           // row of k_new
+        // sequence of row r: last s with cu_q[s] <= r
+        int lo = 0, hi = B;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (__ldg(cu_q + mid) <= r) lo = mid; else hi = mid;
+        }
+        const int s = lo;
+        const int tok = __ldg(prefix_len + s) + (r - __ldg(cu_q + s));
+        const int page_slot = tok / kPage;
+        long long page = -1;
+        if (tok >= 0 && page_slot < pt_stride) page = __ldg(page_table + (long long)s * pt_stride + page_slot);
+        if (page < 0 || page >= num_pages) {
+            if (c == 0 && g == 0) atomicOr(status, AGX_DEV_BAD_PAGE);
+            continue;
+        }
+        const long long dst = (((page * hkv + g) * kPage) + (tok % kPage)) * vec_per_row + c;
+        k_pool[dst] = k_new[idx];
+        v_pool[dst] = v_new[idx];
+    }
+}
+
+cudaError_t launch_kv_append(int dtype, void* k_pool, void* v_pool, long long num_pages, const void* k_new,
+                             const void* v_new, const int* page_table, int pt_stride, const int* prefix_len,
+                             const int* cu_q, int B, int total_q, int hkv, int head_dim, int* status,
+                             cudaStream_t stream) {
+    const int esz = dtype == AGX_BF16 ? 2 : 4;
+    const int vec_per_row = head_dim * esz / 16;
+    const long long n_vec = (long long)total_q * hkv * vec_per_row;
+    if (n_vec == 0) return cudaSuccess;
+    long long blocks = (n_vec + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    kv_append_kernel<<<(int)blocks, 256, 0, stream>>>((uint4*)k_pool, (uint4*)v_pool, num_pages, (const uint4*)k_new,
+                                                      (const uint4*)v_new, page_table, pt_stride, prefix_len, cu_q,
+                                                      B, total_q, hkv, vec_per_row, status);
+    return cudaGetLastError();
+}
+
+}  // namespace agx

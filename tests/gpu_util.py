@@ -1,0 +1,100 @@
+"""Helpers for the GPU parity tests: move a workload to the device, run the CUDA path through the
+C ABI binding, bring results back as float64 numpy, and compare with the oracle."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2605_10380_b200 import agx
+from paper_2605_10380_b200 import workloads as W
+
+ATOL = 1e-2   # max-abs bound on attention outputs (unit-variance inputs, fp32 accumulation)
+RTOL = 2e-2   # bound on the per-(row, head) normwise relative error  ||gpu - ref||_inf / ||ref||_inf
+
+
+def dev(arr: np.ndarray, dtype: str | None = None) -> torch.Tensor:
+    t = torch.from_numpy(np.ascontiguousarray(arr)).cuda()
+    if dtype == "bf16":
+        t = t.view(torch.bfloat16)
+    return t
+
+
+def host_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to(torch.float64).cpu().numpy()
+
+
+def host_storage(t: torch.Tensor, dtype: str) -> np.ndarray:
+    if dtype == "bf16":
+        return t.detach().view(torch.uint16).cpu().numpy()
+    return t.detach().cpu().numpy()
+
+
+class DeviceBatch:
+    def __init__(self, w: W.AttnWorkload, poison_tail: bool = False):
+        self.w = w
+        self.h = agx.Handle(w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype)
+        self.k_pool = dev(w.k_pool, w.dtype)
+        self.v_pool = dev(w.v_pool, w.dtype)
+        self.q_block = dev(w.q_block, w.dtype)
+        self.k_new = dev(w.k_new, w.dtype)
+        self.v_new = dev(w.v_new, w.dtype)
+        self.page_table = dev(w.page_table)
+        self.prefix_len = dev(w.prefix_len)
+        self.cu_q = dev(w.cu_q)
+        tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+        self.out = torch.zeros((w.total_q, w.num_q_heads, w.head_dim), dtype=tdt, device="cuda")
+        self.lse = torch.zeros((w.total_q, w.num_q_heads), dtype=torch.float32, device="cuda")
+        n = self.h.attn_workspace_bytes(w.prefix_len, w.q_len)
+        self.ws_bytes = n
+        self.ws = torch.empty(max(n, 256), dtype=torch.uint8, device="cuda") if n else None
+
+    def append(self):
+        self.h.kv_append(self.k_pool, self.v_pool, self.k_new, self.v_new, self.page_table, self.prefix_len, self.cu_q)
+
+    def attend(self):
+        w = self.w
+        self.h.attn_prefixed(self.q_block, self.k_pool, self.v_pool, self.page_table, w.prefix_len, w.q_len,
+                             self.out, self.lse, self.ws)
+        self.launches = self.h.last_launch_count()
+        torch.cuda.synchronize()
+        return host_f64(self.out), host_f64(self.lse)
+
+    def status(self):
+        return self.h.get_status()
+
+
+def oracle_pools_after_append(w: W.AttnWorkload):
+    kp, vp = w.k_pool.copy(), w.v_pool.copy()
+    oracle.kv_append(kp, vp, w.k_new, w.v_new, w.dtype, w.page_table, w.prefix_len, w.cu_q)
+    return kp, vp
+
+
+def check_attention(gpu: np.ndarray, ref: np.ndarray, what: str = ""):
+    """gpu, ref: [..., d].  Gate: max-abs <= 1e-2 AND per-row normwise relative error <= 2e-2."""
+    assert gpu.shape == ref.shape
+    assert np.all(np.isfinite(gpu)), f"{what}: non-finite output"
+    err = np.abs(gpu - ref)
+    max_abs = float(err.max()) if err.size else 0.0
+    row_err = err.max(axis=-1)
+    row_ref = np.abs(ref).max(axis=-1)
+    rel = float((row_err / np.maximum(row_ref, 1e-30)).max()) if err.size else 0.0
+    assert max_abs <= ATOL, f"{what}: max-abs {max_abs:.3e} > {ATOL}"
+    assert rel <= RTOL, f"{what}: normwise relative {rel:.3e} > {RTOL}"
+    return max_abs, rel
+
+
+def run_accept(h: agx.Handle, aw: W.AcceptWorkload, with_seq_lens=True):
+    logits = dev(aw.logits, aw.dtype)
+    drafts = dev(aw.drafts) if aw.drafts.size else torch.zeros(1, dtype=torch.int32, device="cuda")
+    cu_q = dev(aw.cu_q)
+    B = len(aw.cu_q) - 1
+    rows = int(aw.cu_q[-1])
+    acc = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    nxt = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    am = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
+    sl = dev(aw.prefix_len.copy()) if with_seq_lens else None
+    ws = torch.empty(h.accept_workspace_bytes(rows, aw.vocab), dtype=torch.uint8, device="cuda")
+    h.accept_greedy(logits[:rows], aw.dtype, aw.vocab, drafts, cu_q, acc, nxt, am, sl, ws)
+    torch.cuda.synchronize()
+    return (am.cpu().numpy(), acc.cpu().numpy(), nxt.cpu().numpy(), None if sl is None else sl.cpu().numpy())

@@ -1,0 +1,239 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
+
+Attention: max-abs error <= 1e-2 and per-(row, head) normwise relative error <= 2e-2.
+KV append, argmax, accept lengths, next tokens, committed lengths: bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_10380_b200 import agx
+from paper_2605_10380_b200 import workloads as W
+from tests.gpu_util import (DeviceBatch, check_attention, dev, host_storage, oracle_pools_after_append,
+                            run_accept)
+
+pytestmark = pytest.mark.gpu
+
+
+def run_and_check(w, sample=None, poison=False):
+    b = DeviceBatch(w)
+    if poison:  # slots past P + q in every sequence's last page hold NaN: they must never be read
+        nanbits = 0x7FC0 if w.dtype == "bf16" else np.float32(np.nan)
+        for s in range(w.batch):
+            L = int(w.prefix_len[s] + w.q_len[s])
+            if L % 16:
+                pg = int(w.page_table[s, L // 16])
+                kp = host_storage(b.k_pool, w.dtype); vp = host_storage(b.v_pool, w.dtype)
+                kp[pg, :, L % 16:, :] = nanbits; vp[pg, :, L % 16:, :] = nanbits
+                b.k_pool.copy_(dev(kp, w.dtype)); b.v_pool.copy_(dev(vp, w.dtype))
+    b.append()
+    out, lse = b.attend()
+    assert b.status() == 0
+    kp, vp = oracle_pools_after_append(w)
+    # append parity, bit-exact on the touched pages
+    gk = host_storage(b.k_pool, w.dtype); gv = host_storage(b.v_pool, w.dtype)
+    if not poison:
+        assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
+    if sample is None:
+        ref, ref_lse = oracle.attn_paged_batch(w.q_block, kp, vp, w.page_table, w.dtype, w.prefix_len, w.q_len, w.cu_q)
+        stats = check_attention(out, ref, w.name)
+        assert np.max(np.abs(lse - ref_lse)) <= 2e-3, "lse"
+    else:
+        rng = np.random.default_rng(sample[0])
+        stats = (0.0, 0.0)
+        for s in range(w.batch):
+            q = int(w.q_len[s]); r0 = int(w.cu_q[s])
+            n = min(sample[1], q * w.num_q_heads)
+            si = np.concatenate([[0, q - 1], rng.integers(0, q, n)]).astype(np.int32)
+            sh = np.concatenate([[0, w.num_q_heads - 1], rng.integers(0, w.num_q_heads, n)]).astype(np.int32)
+            ref, ref_lse, _ = oracle.attn_paged(w.q_block[r0:r0 + q], kp, vp, w.page_table[s], w.dtype,
+                                                int(w.prefix_len[s]), select=(si, sh))
+            st = check_attention(out[r0 + si, sh], ref, f"{w.name} seq {s}")
+            stats = (max(stats[0], st[0]), max(stats[1], st[1]))
+            assert np.max(np.abs(lse[r0 + si, sh] - ref_lse)) <= 2e-3
+    return b, stats
+
+
+# ------------------------------------------------------------------ named configurations
+def test_c1_tiny_verify_fp32():
+    b, _ = run_and_check(W.c1_tiny_verify())
+    assert b.launches >= 1
+
+
+def test_c1_tiny_verify_bf16_rounded_inputs_d128():
+    w = W.make_attn_workload("c1_bf16", 1, "bf16", 4, 2, 128, [256], [4], spare_pages=47)
+    run_and_check(w)
+
+
+def test_c2_decode_verify():
+    b, stats = run_and_check(W.c2_decode_verify())
+    assert b.ws_bytes > 0  # the context is split over many CTAs
+
+
+def test_c2_accept_bf16_uniform_accept_lengths():
+    h = agx.Handle(32, 8, 128, "bf16")
+    for a in range(8):
+        aw = W.make_planted_accept("c2_accept", 200 + a, "bf16", 128256, [8], [4096], planned_accept=[a])
+        ref = oracle.accept_greedy(aw.logits, "bf16", aw.vocab, aw.drafts, aw.cu_q, aw.prefix_len)
+        got = run_accept(h, aw)
+        for g, r in zip(got, ref):
+            assert np.array_equal(g, r)
+        assert got[1][0] == a and got[3][0] == 4096 + a + 1
+
+
+def test_c1_accept_fp32_first_two_of_three_match():
+    logits = W.natural_logits(1, 4, 1024, "f32")
+    am, _, _, _ = oracle.accept_greedy(logits, "f32", 1024, np.zeros(0, np.int32), np.arange(5, dtype=np.int32),
+                                       np.zeros(4, np.int32))
+    drafts = np.array([am[0], am[1], (am[2] + 1) % 1024], dtype=np.int32)  # first 2 of 3 match
+    aw = W.AcceptWorkload("c1_accept", "f32", 1024, 1024, logits, drafts, np.array([0, 4], np.int32),
+                          np.array([256], np.int32))
+    h = agx.Handle(4, 2, 64, "f32")
+    got = run_accept(h, aw)
+    ref = oracle.accept_greedy(logits, "f32", 1024, drafts, aw.cu_q, aw.prefix_len)
+    for g, r in zip(got, ref):
+        assert np.array_equal(g, r)
+    assert got[1][0] == 2 and got[2][0] == am[2] and got[3][0] == 259
+
+
+# ------------------------------------------------------------------ small-q kernel: shapes and edges
+@pytest.mark.parametrize("P,q,hq,hkv", [
+    (0, 1, 32, 8), (1, 1, 32, 8), (15, 1, 8, 8), (16, 2, 32, 8), (17, 4, 32, 8), (63, 8, 32, 8), (64, 8, 32, 8),
+    (65, 16, 32, 8), (1000, 3, 24, 8), (2049, 5, 32, 8), (5000, 8, 32, 8), (777, 16, 32, 8), (300, 7, 4, 1),
+    (130, 1, 4, 4), (4095, 2, 16, 2),
+])
+def test_small_q_shapes(P, q, hq, hkv):
+    w = W.make_attn_workload(f"small_{P}_{q}", 1000 + P + q, "bf16", hq, hkv, 128, [P], [q], spare_pages=3)
+    run_and_check(w, poison=True)
+
+
+def test_small_q_ragged_batch_with_shared_prefix():
+    P = [2048, 2100, 4000, 2048 + 15, 9000, 2500, 3001, 2048]
+    q = [1, 2, 4, 8, 16, 3, 5, 8]
+    w = W.make_attn_workload("ragged_small", 42, "bf16", 32, 8, 128, P, q, shared_prefix_tokens=2048)
+    run_and_check(w, sample=(7, 12))
+
+
+def test_q1_equals_plain_decode_on_gpu():
+    w = W.make_attn_workload("decode", 9, "bf16", 32, 8, 128, [1234], [1])
+    b = DeviceBatch(w); b.append(); out, _ = b.attend()
+    kp, vp = oracle_pools_after_append(w)
+    K = W.gather_contiguous(kp, w.page_table[0], 1235); V = W.gather_contiguous(vp, w.page_table[0], 1235)
+    ref = oracle.decode_plain(w.q_block[0], K, V, "bf16")
+    check_attention(out[0], ref, "decode")
+
+
+def test_split_results_are_bit_reproducible():
+    w = W.c2_decode_verify(seed=12)
+    b = DeviceBatch(w); b.append()
+    a, _ = b.attend()
+    b.out.zero_()
+    c, _ = b.attend()
+    assert np.array_equal(a, c)
+
+
+def test_fp32_path_shapes():
+    for (P, q, hq, hkv, d) in [(0, 1, 4, 2, 64), (100, 5, 4, 2, 64), (700, 3, 8, 2, 128), (31, 20, 4, 4, 64)]:
+        w = W.make_attn_workload(f"f32_{P}_{q}", 5 + P, "f32", hq, hkv, d, [P, P + 3], [q, 1], spare_pages=2)
+        run_and_check(w, poison=True)
+
+
+def test_mma_sync_kernel_handles_large_q(monkeypatch):
+    """The warp-MMA kernel also serves long blocks (row chunks); it is the baseline the tensor-core
+    tile kernel is measured against."""
+    monkeypatch.setenv("AGX_FORCE_MMA_SYNC", "1")
+    w = W.make_attn_workload("mma_large", 77, "bf16", 24, 8, 128, [500, 37], [200, 130])
+    run_and_check(w, sample=(3, 40))
+
+
+# ------------------------------------------------------------------ KV append alone
+def test_kv_append_ragged_bit_exact_and_untouched_elsewhere():
+    w = W.make_attn_workload("append", 5, "bf16", 32, 8, 128, [5, 30, 16, 0, 4095], [3, 1, 20, 17, 600], spare_pages=5)
+    b = DeviceBatch(w); b.append(); torch.cuda.synchronize()
+    kp, vp = oracle_pools_after_append(w)
+    assert np.array_equal(host_storage(b.k_pool, "bf16"), kp)
+    assert np.array_equal(host_storage(b.v_pool, "bf16"), vp)
+
+
+def test_bad_page_id_sets_status_and_does_not_fault():
+    w = W.make_attn_workload("badpage", 6, "bf16", 32, 8, 128, [100], [4])
+    w.page_table[0, 2] = w.num_pages + 1000
+    b = DeviceBatch(w); b.append(); b.attend()
+    assert b.status() & agx.AGX_DEV_BAD_PAGE
+    assert b.status() == 0  # cleared by the read
+
+
+# ------------------------------------------------------------------ accept
+def test_accept_natural_ties_and_special_values():
+    h = agx.Handle(32, 8, 128, "bf16")
+    x = W.natural_logits(5, 40, 128256, "bf16")
+    am_ref, _, _, _ = oracle.accept_greedy(x, "bf16", 128256, np.zeros(0, np.int32), np.arange(41, dtype=np.int32),
+                                           np.zeros(40, np.int32))
+    q_len = [8, 1, 16, 4, 2, 9]
+    cu = W.cu_from_q(q_len)
+    rng = np.random.default_rng(0)
+    plan = np.array([int(rng.integers(0, q)) for q in q_len], dtype=np.int32)
+    drafts = W.make_drafts(3, am_ref, cu, plan, 128256)
+    aw = W.AcceptWorkload("ties", "bf16", 128256, 128256, x, drafts, cu, np.arange(6, dtype=np.int32) * 100)
+    got = run_accept(h, aw)
+    ref = oracle.accept_greedy(x, "bf16", 128256, drafts, cu, aw.prefix_len)
+    for g, r in zip(got, ref):
+        assert np.array_equal(g, r)
+    assert np.array_equal(got[1], plan)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_accept_special_values_padding_and_odd_vocab(dtype):
+    V, stride = 1001, 1008
+    x = np.full((6, stride), 9.0, dtype=np.float32)
+    x[:, :V] = -1.0
+    x[0, [3, 700]] = 2.0
+    x[1, :V] = -0.0; x[1, 5] = 0.0
+    x[2, :V] = np.nan; x[2, 999] = -50.0
+    x[3, :V] = np.nan
+    x[4, :V] = -np.inf
+    x[5, 1000] = np.inf; x[5, 1] = 1e30
+    xs = W.to_storage(x, dtype)
+    cu = np.arange(7, dtype=np.int32)
+    aw = W.AcceptWorkload("special", dtype, V, stride, xs, np.zeros(0, np.int32), cu, np.zeros(6, np.int32))
+    h = agx.Handle(4, 2, 64, "f32")
+    got = run_accept(h, aw)
+    ref = oracle.accept_greedy(xs, dtype, V, aw.drafts, cu, aw.prefix_len)
+    assert got[0].tolist() == [3, 0, 999, 0, 0, 1000]
+    for g, r in zip(got, ref):
+        assert np.array_equal(g, r)
+
+
+def test_accept_many_rows_and_unaligned_rows():
+    h = agx.Handle(4, 2, 64, "f32")
+    aw = W.make_planted_accept("many", 31, "bf16", 3001, [5] * 60 + [1] * 40, np.arange(100), row_stride=3001)
+    got = run_accept(h, aw)
+    ref = oracle.accept_greedy(aw.logits, "bf16", aw.vocab, aw.drafts, aw.cu_q, aw.prefix_len)
+    for g, r in zip(got, ref):
+        assert np.array_equal(g, r)
+    # twice in a row on the same handle: the ticket counter resets itself
+    got2 = run_accept(h, aw)
+    for g, r in zip(got2, ref):
+        assert np.array_equal(g, r)
+
+
+# ------------------------------------------------------------------ argument errors (host side)
+def test_argument_errors_are_reported_not_faulted():
+    w = W.make_attn_workload("err", 6, "bf16", 32, 8, 128, [100], [4])
+    b = DeviceBatch(w)
+    with pytest.raises(agx.AgxError) as e:
+        b.h.attn_prefixed(b.q_block, b.k_pool, b.v_pool, b.page_table, [100], [0], b.out)
+    assert e.value.status == -1
+    with pytest.raises(agx.AgxError) as e:
+        b.h.attn_prefixed(b.q_block, b.k_pool, b.v_pool, b.page_table, [100000], [4], b.out)
+    assert e.value.status == -2
+    with pytest.raises(agx.AgxError):
+        agx.Handle(32, 5, 128, "bf16")
+    with pytest.raises(agx.AgxError):
+        agx.Handle(32, 8, 96, "bf16")
+    w2 = W.c2_decode_verify()
+    b2 = DeviceBatch(w2)
+    with pytest.raises(agx.AgxError) as e:  # split launch without workspace
+        b2.h.attn_prefixed(b2.q_block, b2.k_pool, b2.v_pool, b2.page_table, w2.prefix_len, w2.q_len, b2.out)
+    assert e.value.status == -1
