@@ -1,0 +1,482 @@
+#!/usr/bin/env python
+"""Benchmark of the prefix-cached block-attention / greedy-accept hot path on B200.
+
+One JSON line on stdout (rank 0).  A *step* is one pass of the whole hot path over one batch:
+for every layer ``agx_kv_append`` + ``agx_attn_prefixed``, then one ``agx_accept_greedy``.
+
+Default workload = "decode verification": batch 1, cached context 4096, q = 8 (7 drafts + the last
+emitted token), GQA 32/8, head_dim 128, bf16, page size 16 with shuffled pages, 32 independent
+per-layer KV pools (553 MB, larger than L2, so every layer's KV is read from HBM), accept on bf16
+logits [8, 128256].  ``value`` counts query tokens per second per attention-layer call
+(``layers * q / step time``).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl agx|reference] [--no-extra]
+
+N > 1 (under torchrun) runs one independent replica per GPU (the path shards by sequence with no
+exchange step): weak scaling, value = all ranks' units / max-over-ranks time.
+``--impl reference`` times the CPU oracle (the only reference there is) on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "prefix-cached attn query tok/s"
+UNIT = "query tok/s (per attention-layer call)"
+C2 = dict(P=4096, q=8, hq=32, hkv=8, d=128, vocab=128256, layers=32)
+
+
+# --------------------------------------------------------------------------- peaks / clocks
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- distributed helpers
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def aggregate_over_ranks(ms_local: float, units_local: float, backend_device=None):
+    """Weak scaling over independent replicas: time = max over ranks, units = sum over ranks."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return ms_local, units_local
+    dev = backend_device if backend_device is not None else "cpu"
+    t = torch.tensor([ms_local], dtype=torch.float64, device=dev)
+    u = torch.tensor([units_local], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# --------------------------------------------------------------------------- workload on the device
+def alg_bytes_attn(P, q, hq, hkv, d, esz=2):
+    return 2 * hkv * d * esz * (P + q) + 2 * q * hq * d * esz
+
+
+def alg_flops_attn(P, q, hq, d):
+    return 4 * d * hq * (q * P + q * (q + 1) // 2)
+
+
+class LayeredVerify:
+    """`layers` independent KV pools for one (or more) sequences, plus logits for the accept step."""
+
+    def __init__(self, torch, agx, W, P_list, q_list, hq, hkv, d, layers, vocab, seed):
+        self.torch, self.W = torch, W
+        self.P = np.asarray(P_list, np.int32); self.Q = np.asarray(q_list, np.int32)
+        self.hq, self.hkv, self.d, self.layers, self.vocab = hq, hkv, d, layers, vocab
+        self.B = len(P_list)
+        self.cu = W.cu_from_q(self.Q)
+        self.total_q = int(self.cu[-1])
+        g = torch.Generator(device="cuda"); g.manual_seed(seed)
+        rng = np.random.default_rng(seed)
+        table, self.num_pages = W.build_page_table(rng, self.P.astype(np.int64) + self.Q, 0, spare_pages=7)
+        self.page_table = torch.from_numpy(table).cuda()
+        bf = torch.bfloat16
+        rn = lambda *s: torch.randn(*s, generator=g, device="cuda", dtype=torch.float32).to(bf)
+        self.k_pools = [rn(self.num_pages, hkv, 16, d) for _ in range(layers)]
+        self.v_pools = [rn(self.num_pages, hkv, 16, d) for _ in range(layers)]
+        self.q_block = [rn(self.total_q, hq, d) for _ in range(layers)]
+        self.k_new = [rn(self.total_q, hkv, d) for _ in range(layers)]
+        self.v_new = [rn(self.total_q, hkv, d) for _ in range(layers)]
+        self.out = [torch.empty(self.total_q, hq, d, device="cuda", dtype=bf) for _ in range(layers)]
+        self.prefix_dev = torch.from_numpy(self.P).cuda()
+        self.cu_dev = torch.from_numpy(self.cu).cuda()
+        self.h = agx.Handle(hq, hkv, d, "bf16")
+        n = self.h.attn_workspace_bytes(self.P, self.Q)
+        self.ws = torch.empty(max(n, 256), dtype=torch.uint8, device="cuda") if n else None
+        if vocab:
+            aw = W.make_planted_accept("bench_accept", seed, "bf16", vocab, self.Q, self.P)
+            self.aw = aw
+            self.logits = torch.from_numpy(aw.logits).cuda().view(bf)
+            self.drafts = torch.from_numpy(aw.drafts if aw.drafts.size else np.zeros(1, np.int32)).cuda()
+            self.acc = torch.zeros(self.B, dtype=torch.int32, device="cuda")
+            self.nxt = torch.zeros(self.B, dtype=torch.int32, device="cuda")
+            self.seq_lens = torch.from_numpy(self.P.copy()).cuda()
+            self.acc_ws = torch.empty(self.h.accept_workspace_bytes(self.total_q, vocab), dtype=torch.uint8, device="cuda")
+        self.launches_per_step = 0
+
+    def attn_layer(self, l):
+        self.h.attn_prefixed(self.q_block[l], self.k_pools[l], self.v_pools[l], self.page_table, self.P, self.Q,
+                             self.out[l], None, self.ws)
+        return self.h.last_launch_count()
+
+    def step(self, attn_only=False):
+        n = 0
+        for l in range(self.layers):
+            if not attn_only:
+                self.h.kv_append(self.k_pools[l], self.v_pools[l], self.k_new[l], self.v_new[l], self.page_table,
+                                 self.prefix_dev, self.cu_dev)
+                n += self.h.last_launch_count()
+            n += self.attn_layer(l)
+        if not attn_only and self.vocab:
+            self.seq_lens.copy_(self.prefix_dev)
+            self.h.accept_greedy(self.logits, "bf16", self.vocab, self.drafts, self.cu_dev, self.acc, self.nxt, None,
+                                 self.seq_lens, self.acc_ws)
+            n += self.h.last_launch_count() + 1  # + the device-to-device length reset (a torch copy kernel)
+        return n
+
+    def bytes_per_layer(self):
+        return sum(alg_bytes_attn(int(p), int(q), self.hq, self.hkv, self.d) for p, q in zip(self.P, self.Q))
+
+    def flops_per_layer(self):
+        return sum(alg_flops_attn(int(p), int(q), self.hq, self.d) for p, q in zip(self.P, self.Q))
+
+
+def capture(torch, fn):
+    """Warm up (first calls configure kernels), then capture fn into a CUDA graph."""
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        for _ in range(2):
+            fn()
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        fn()
+    return g
+
+
+def time_graph(torch, g, steps, warmup, barrier=None):
+    for _ in range(warmup):
+        g.replay()
+    if barrier:
+        barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    return e0.elapsed_time(e1) / steps  # ms per step
+
+
+# --------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample_c2(W, seconds_target=15.0):
+    """Time the oracle, as it stands, on whole layers of the decode-verification workload."""
+    import oracle
+    w = W.c2_decode_verify()
+    aw = W.make_planted_accept("bench_accept", 2, "bf16", C2["vocab"], w.q_len, w.prefix_len)
+    kp, vp = w.k_pool.copy(), w.v_pool.copy()
+
+    def one_layer():
+        oracle.kv_append(kp, vp, w.k_new, w.v_new, "bf16", w.page_table, w.prefix_len, w.cu_q)
+        oracle.attn_paged_batch(w.q_block, kp, vp, w.page_table, "bf16", w.prefix_len, w.q_len, w.cu_q)
+
+    one_layer()  # page in
+    t0 = time.perf_counter(); one_layer(); dt = time.perf_counter() - t0
+    n = int(max(1, seconds_target / max(dt, 1e-3)))
+    t0 = time.perf_counter()
+    for _ in range(n):
+        one_layer()
+    oracle.accept_greedy(aw.logits, "bf16", aw.vocab, aw.drafts, aw.cu_q, aw.prefix_len)
+    total = time.perf_counter() - t0
+    return dict(value=n * C2["q"] / total, unit=UNIT, cores=oracle.num_threads(), kind="oracle",
+                sample=f"{n} layer calls of the decode-verification step (append + attention, fp64; a step has "
+                       f"{C2['layers']}) plus one accept over [8, {C2['vocab']}] logits, {total:.1f} s"), total, n
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    from paper_2605_10380_b200 import workloads as W
+    import oracle
+    w = W.c2_decode_verify()
+    aw = W.make_planted_accept("bench_accept", 2, "bf16", C2["vocab"], w.q_len, w.prefix_len)
+    kp, vp = w.k_pool.copy(), w.v_pool.copy()
+
+    def step():  # bounded sample of one step: one of the 32 layers, plus the accept
+        oracle.kv_append(kp, vp, w.k_new, w.v_new, "bf16", w.page_table, w.prefix_len, w.cu_q)
+        oracle.attn_paged_batch(w.q_block, kp, vp, w.page_table, "bf16", w.prefix_len, w.q_len, w.cu_q)
+        oracle.accept_greedy(aw.logits, "bf16", aw.vocab, aw.drafts, aw.cu_q, aw.prefix_len)
+
+    for _ in range(max(1, args.warmup)):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = args.steps * C2["q"] / dt
+    sample = "each step = 1 of 32 layers (append + attention, fp64 oracle) + accept over [8, 128256] logits"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "decode verification (c2): P=4096 q=8 GQA 32/8 d=128 bf16 storage", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- extra workloads (N = 1)
+def extra_workloads(torch, agx, W, peaks, steps, warmup):
+    out = {}
+    # long-context verify: 4 x (P = 32768, q = 8); 537 MB of KV per layer call, HBM-bound
+    try:
+        lv = LayeredVerify(torch, agx, W, [32768] * 4, [8] * 4, 32, 8, 128, 1, 0, 5)
+        g = capture(torch, lambda: lv.step(attn_only=True))
+        ms = time_graph(torch, g, max(steps, 20), max(warmup, 3))
+        by = lv.bytes_per_layer()
+        out["c5_long_context_verify"] = {
+            "ms": ms, "query_tok_per_s": 32 / (ms * 1e-3),
+            "roofline": {"bound": "hbm", "achieved": by / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                         "frac_of_nominal_8000": by / (ms * 1e-3) / 1e9 / 8000.0}}
+        del lv, g
+        torch.cuda.empty_cache()
+    except Exception as e:  # keep the headline line alive
+        out["c5_long_context_verify"] = {"error": repr(e)}
+    # prefix-cached prefill: P = 3072, q = 512, 24/8; tensor-bound.  4 layer pools are rotated.
+    for name, P, q, hq in (("c3_prefix_prefill", 3072, 512, 24), ("c5_long_context_prefill", 30720, 2048, 32)):
+        try:
+            layers = 4 if q == 512 else 1
+            lv = LayeredVerify(torch, agx, W, [P], [q], hq, 8, 128, layers, 0, 3)
+            g = capture(torch, lambda: lv.step(attn_only=True))
+            ms = time_graph(torch, g, max(steps // 2, 10), max(warmup, 3)) / layers
+            fl = lv.flops_per_layer()
+            pk = peaks["bf16_tflops_sustained"]
+            out[name] = {"ms": ms, "query_tok_per_s": q / (ms * 1e-3),
+                         "roofline": {"bound": "tensor", "achieved": fl / (ms * 1e-3) / 1e12, "peak": pk,
+                                      "unit": "TFLOP/s", "frac": fl / (ms * 1e-3) / 1e12 / pk,
+                                      "peak_source": peaks["source"] + " (sustained bf16)",
+                                      "frac_of_nominal_2250": fl / (ms * 1e-3) / 1e12 / 2250.0}}
+            del lv, g
+            torch.cuda.empty_cache()
+        except Exception as e:
+            out[name] = {"error": repr(e)}
+    return out
+
+
+# --------------------------------------------------------------------------- main arm
+def run_agx(args):
+    import torch
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the agx path")
+    torch.cuda.set_device(local_rank)
+    barrier = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        barrier = lambda: dist.barrier()
+    from paper_2605_10380_b200 import build as _build
+    if rank == 0:
+        _build.build()
+    if barrier:
+        barrier()
+    from paper_2605_10380_b200 import agx
+    from paper_2605_10380_b200 import workloads as W
+    peaks = load_peaks()
+    c = C2
+    lv = LayeredVerify(torch, agx, W, [c["P"]], [c["q"]], c["hq"], c["hkv"], c["d"], c["layers"], c["vocab"], 2 + rank)
+    launches = lv.step()  # eager warm-up, also counts launches
+    torch.cuda.synchronize()
+    assert lv.h.get_status() == 0
+    g_full = capture(torch, lv.step)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        t_wait = time.time()
+        while not sampler.lines and time.time() - t_wait < 3.0:
+            time.sleep(0.05)
+        sampler.lines.clear()  # keep only samples taken while the GPU is busy
+    ms = time_graph(torch, g_full, args.steps, args.warmup, barrier)
+    units = float(c["layers"] * c["q"])
+    # attention-only graph: per-call duration of the dominant kernel (split-KV kernel + its combine)
+    g_attn = capture(torch, lambda: lv.step(attn_only=True))
+    ms_attn = time_graph(torch, g_attn, args.steps, max(args.warmup, 3)) / c["layers"]
+    clocks = sampler.stop() if sampler else None
+    ms_max, units_all = aggregate_over_ranks(ms, units, torch.device("cuda", local_rank))
+    value = units_all / (ms_max * 1e-3)
+
+    # end to end through the host-buffer entry point: per layer H2D(q, k_new, v_new) + D2H(out); the last
+    # layer's call also uploads logits and drafts and downloads the accept results
+    pin = lambda t: t.cpu().pin_memory()
+    hq_, hk_, hv_ = [pin(t) for t in lv.q_block], [pin(t) for t in lv.k_new], [pin(t) for t in lv.v_new]
+    h_out = torch.empty_like(hq_[0]).pin_memory()
+    h_logits, h_drafts = pin(lv.logits), pin(lv.drafts)
+    h_acc = torch.zeros(1, dtype=torch.int32).pin_memory(); h_nxt = torch.zeros(1, dtype=torch.int32).pin_memory()
+    h_sl = torch.zeros(1, dtype=torch.int32).pin_memory()
+    ws_n = lv.h.verify_step_host_workspace_bytes(lv.P, lv.Q, "bf16", c["vocab"], c["vocab"])
+    ws_host = torch.empty(ws_n, dtype=torch.uint8, device="cuda")
+
+    def e2e_step():
+        for l in range(c["layers"]):
+            last = l == c["layers"] - 1
+            lv.h.verify_step_host(lv.k_pools[l], lv.v_pools[l], lv.page_table, lv.P, lv.Q, hq_[l], hk_[l], hv_[l],
+                                  h_logits if last else None, "bf16", c["vocab"], c["vocab"] if last else 0,
+                                  h_drafts if last else None, h_out, h_acc, h_nxt, h_sl, ws_host)
+
+    for _ in range(max(3, args.warmup)):
+        e2e_step()
+    if barrier:
+        barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) / args.steps * 1e3
+    e2e_ms_max, _ = aggregate_over_ranks(e2e_ms, units, torch.device("cuda", local_rank))
+    esz = 2
+    h2d = c["layers"] * (c["q"] * (c["hq"] + 2 * c["hkv"]) * c["d"] * esz + 2 * 4 + 2 * 4) + c["q"] * c["vocab"] * esz + 7 * 4
+    d2h = c["layers"] * c["q"] * c["hq"] * c["d"] * esz + 3 * 4
+    if rank != 0:
+        return
+    by = lv.bytes_per_layer()
+    achieved = by / (ms_attn * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": "decode verification (c2): batch 1, cached context 4096, q=8, GQA 32/8, d=128, bf16, "
+                               "page 16 shuffled, 32 per-layer KV pools + accept on bf16 logits [8,128256]",
+                   "step": "32 x (agx_kv_append + agx_attn_prefixed) + 1 x agx_accept_greedy, one CUDA graph",
+                   "l2": "inputs larger than L2: 32 distinct layer pools = 553 MB, each read once per step",
+                   "parallelism": f"{world} independent replica(s), no collective"},
+        "gpu_launches": launches,
+        "e2e": {"value": units_all / (e2e_ms_max * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_max,
+                "path": "agx_verify_step_host per layer (pinned host q/k_new/v_new/logits in, out/accept results back)"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                     "frac_of_nominal_8000": achieved / 8000.0,
+                     "kernel": "attn_small_bf16_kernel<2,3> + attn_combine_kernel (one agx_attn_prefixed call)",
+                     "algorithmic_bytes_per_launch": by, "us_per_launch": ms_attn * 1e3},
+        "clocks": clocks,
+    }
+    if world == 1:
+        cb, _, _ = oracle_sample_c2(W)
+        line["cpu_baseline"] = cb
+        if not args.no_extra:
+            line["workloads"] = extra_workloads(torch, agx, W, peaks, args.steps, args.warmup)
+    print(json.dumps(line))
+
+
+ONLY = {  # name: (P list, q list, Hq, layers)
+    "c2": ([4096], [8], 32, 4),
+    "c3": ([3072], [512], 24, 1),
+    "c5v": ([32768] * 4, [8] * 4, 32, 1),
+    "c5p": ([30720], [2048], 32, 1),
+    "c5p_small": ([7680], [1024], 32, 1),
+}
+
+
+def run_only(args):
+    """Profiling aid: eager (no graph) attention calls of ONE workload, a few launches, one line out."""
+    import torch
+    torch.cuda.set_device(0)
+    from paper_2605_10380_b200 import agx
+    from paper_2605_10380_b200 import workloads as W
+    P, q, hq, layers = ONLY[args.only]
+    lv = LayeredVerify(torch, agx, W, P, q, hq, 8, 128, layers, 0, 7)
+    for _ in range(args.warmup):
+        for l in range(layers):
+            lv.attn_layer(l)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        for l in range(layers):
+            lv.attn_layer(l)
+    e1.record()
+    torch.cuda.synchronize()
+    assert lv.h.get_status() == 0
+    ms = e0.elapsed_time(e1) / (args.steps * layers)
+    print(json.dumps({"only": args.only, "ms_per_call_eager": ms, "bytes": lv.bytes_per_layer(),
+                      "flops": lv.flops_per_layer(), "GBps": lv.bytes_per_layer() / ms / 1e6,
+                      "TFLOPs": lv.flops_per_layer() / ms / 1e9}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="agx", choices=["agx", "reference"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the extra workloads (c3, c5)")
+    ap.add_argument("--only", choices=sorted(ONLY), help="profiling aid: eager attention calls of one workload")
+    args = ap.parse_args()
+    if args.only:
+        return run_only(args)
+    args.warmup = max(args.warmup, 3) if args.impl == "agx" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_agx(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -199,6 +199,8 @@ AGX_API agx_status agx_get_status(agx_handle* handle, void* stream, int32_t* dev
  *   h_out                      : host, [total_q][num_q_heads][head_dim]
  *   h_accept_len, h_next_token, h_seq_lens : host int32 [B]; h_seq_lens receives
  *                                prefix_len + accept_len + 1
+ *   vocab == 0                 : attention only (a middle layer of a model): the logits, drafts
+ *                                and accept outputs are ignored and may be NULL
  *   workspace                  : device, >= agx_verify_step_host_workspace_bytes(...) bytes,
  *                                256-byte aligned; holds the staged copies and both scratch areas
  * Errors: as the three calls; nothing is launched when a check fails.

@@ -109,14 +109,27 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
             work += items * (P[s] + Q[s]);
         }
         int C = std::max(min_split, round_up((work + target - 1) / target, unit));
-        for (;;) {
+        auto count_items = [&](int c_tokens) {
             long long items = 0;
             for (size_t n = 0; n < seqs.size(); ++n) {
                 const int L = P[seqs[n]] + Q[seqs[n]];
-                items += per_seq_items[n] * ((L + C - 1) / C);
+                items += per_seq_items[n] * ((L + c_tokens - 1) / c_tokens);
             }
-            if (items <= std::max<long long>(target, base_items)) break;
-            C += unit;
+            return items;
+        };
+        if (k == KIND_TILE) {
+            // several waves are fine here: pick the split length with the smallest estimated makespan,
+            // waves * (tiles per item + fixed per-CTA cost of ~3 tiles)
+            int max_len = 0;
+            for (int s : seqs) max_len = std::max(max_len, P[s] + Q[s]);
+            long long best_cost = -1;
+            for (int c_tokens = min_split; c_tokens < max_len + unit; c_tokens += unit) {
+                const long long waves = (count_items(c_tokens) + h->sm_count - 1) / h->sm_count;
+                const long long cost = waves * (std::min(c_tokens, round_up(max_len, unit)) / unit + 3);
+                if (best_cost < 0 || cost < best_cost) { best_cost = cost; C = c_tokens; }
+            }
+        } else {
+            while (count_items(C) > std::max<long long>(target, base_items)) C += unit;
         }
         // ---- emit launches of at most kMaxSeqs sequences
         for (size_t a = 0; a < seqs.size(); a += kMaxSeqs) {
@@ -294,7 +307,8 @@ agx_status agx_attn_prefixed(agx_handle* h, const void* q_block, const void* k_p
             case KIND_SMALL2: e = launch_attn_small_bf16(p, 2, stream); break;
             case KIND_SMALL4: e = launch_attn_small_bf16(p, 4, stream); break;
             case KIND_SIMT: e = launch_attn_simt_f32(p, stream); break;
-            default: return fail(h, AGX_E_UNSUPPORTED, "tile kernel not built");
+            case KIND_TILE: e = launch_attn_tile_bf16(p, stream); break;
+            default: return fail(h, AGX_E_UNSUPPORTED, "unknown kernel kind");
         }
         if (e != cudaSuccess) return cuda_fail(h, e, "attention launch");
         h->last_launches++;
@@ -381,8 +395,13 @@ struct HostStepLayout {
 agx_status host_step_layout(agx_handle* h, int B, const int32_t* P, const int32_t* Q, int logits_dtype,
                             int64_t row_stride, int vocab, HostStepLayout& L) {
     if (B < 1 || !P || !Q) return fail(h, AGX_E_INVAL, "B < 1 or null lengths");
-    if (logits_dtype != AGX_BF16 && logits_dtype != AGX_F32) return fail(h, AGX_E_UNSUPPORTED, "logits dtype");
-    if (vocab < 1 || row_stride < vocab) return fail(h, AGX_E_RANGE, "vocab < 1 or row_stride < vocab");
+    const bool with_accept = vocab > 0;  // vocab == 0: attention only
+    if (with_accept) {
+        if (logits_dtype != AGX_BF16 && logits_dtype != AGX_F32) return fail(h, AGX_E_UNSUPPORTED, "logits dtype");
+        if (row_stride < vocab) return fail(h, AGX_E_RANGE, "row_stride < vocab");
+    } else if (vocab < 0) {
+        return fail(h, AGX_E_RANGE, "vocab < 0");
+    }
     long long tq = 0;
     for (int s = 0; s < B; ++s) {
         if (Q[s] < 1) return fail(h, AGX_E_INVAL, "q_len[%d] = %d < 1", s, Q[s]);
@@ -391,13 +410,13 @@ agx_status host_step_layout(agx_handle* h, int B, const int32_t* P, const int32_
     if (tq > 65535) return fail(h, AGX_E_RANGE, "more than 65535 rows in one host step");
     const int64_t aws = agx_attn_workspace_bytes(h, B, P, Q);
     if (aws < 0) return (agx_status)aws;
-    const int64_t cws = agx_accept_workspace_bytes(h, (int)tq, vocab);
+    const int64_t cws = with_accept ? agx_accept_workspace_bytes(h, (int)tq, vocab) : 0;
     if (cws < 0) return (agx_status)cws;
     const size_t es = elem_size(h->cfg.dtype);
     L.total_q = (int)tq;
     L.q_bytes = (size_t)tq * h->cfg.num_q_heads * h->cfg.head_dim * es;
     L.kv_bytes = (size_t)tq * h->cfg.num_kv_heads * h->cfg.head_dim * es;
-    L.logits_bytes = (size_t)tq * row_stride * elem_size(logits_dtype);
+    L.logits_bytes = with_accept ? (size_t)tq * row_stride * elem_size(logits_dtype) : 0;
     L.attn_ws_bytes = (size_t)aws;
     L.accept_ws_bytes = (size_t)cws;
     size_t off = 0;
@@ -432,9 +451,10 @@ agx_status agx_verify_step_host(agx_handle* h, void* k_pool, void* v_pool, int64
     HostStepLayout L;
     agx_status st = host_step_layout(h, B, P, Q, logits_dtype, row_stride, vocab, L);
     if (st != AGX_OK) return st;
-    if (!k_pool || !v_pool || !page_table || !h_q || !h_k || !h_v || !h_logits || !h_out || !h_accept || !h_next ||
-        !h_seq_lens || (!h_drafts && L.total_q > B))
-        return fail(h, AGX_E_INVAL, "null pointer");
+    const bool with_accept = vocab > 0;
+    if (!k_pool || !v_pool || !page_table || !h_q || !h_k || !h_v || !h_out) return fail(h, AGX_E_INVAL, "null pointer");
+    if (with_accept && (!h_logits || !h_accept || !h_next || !h_seq_lens || (!h_drafts && L.total_q > B)))
+        return fail(h, AGX_E_INVAL, "null pointer (accept arguments)");
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < L.total)
         return fail(h, AGX_E_INVAL, "host-step workspace missing, misaligned or too small (%zu needed)", L.total);
     cudaStream_t stream = (cudaStream_t)stream_v;
@@ -447,8 +467,10 @@ agx_status agx_verify_step_host(agx_handle* h, void* k_pool, void* v_pool, int64
         if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(ws + off, src, bytes, cudaMemcpyHostToDevice, stream);
     };
     h2d(L.q, h_q, L.q_bytes); h2d(L.k, h_k, L.kv_bytes); h2d(L.v, h_v, L.kv_bytes);
-    h2d(L.logits, h_logits, L.logits_bytes);
-    h2d(L.drafts, h_drafts, (size_t)(L.total_q - B) * 4);
+    if (with_accept) {
+        h2d(L.logits, h_logits, L.logits_bytes);
+        h2d(L.drafts, h_drafts, (size_t)(L.total_q - B) * 4);
+    }
     h2d(L.prefix, P, (size_t)B * 4);
     h2d(L.seqlen, P, (size_t)B * 4);
     h2d(L.cu, cu.data(), (size_t)(B + 1) * 4);
@@ -462,16 +484,21 @@ agx_status agx_verify_step_host(agx_handle* h, void* k_pool, void* v_pool, int64
                            L.attn_ws_bytes ? ws + L.attn_ws : nullptr, L.attn_ws_bytes, stream);
     if (st != AGX_OK) return st;
     launches += h->last_launches;
-    st = agx_accept_greedy(h, ws + L.logits, logits_dtype, row_stride, vocab, (const int32_t*)(ws + L.drafts),
-                           (const int32_t*)(ws + L.cu), B, L.total_q, (int32_t*)(ws + L.acc), (int32_t*)(ws + L.next),
-                           nullptr, (int32_t*)(ws + L.seqlen), ws + L.accept_ws, L.accept_ws_bytes, stream);
-    if (st != AGX_OK) return st;
-    launches += h->last_launches;
+    if (with_accept) {
+        st = agx_accept_greedy(h, ws + L.logits, logits_dtype, row_stride, vocab, (const int32_t*)(ws + L.drafts),
+                               (const int32_t*)(ws + L.cu), B, L.total_q, (int32_t*)(ws + L.acc),
+                               (int32_t*)(ws + L.next), nullptr, (int32_t*)(ws + L.seqlen), ws + L.accept_ws,
+                               L.accept_ws_bytes, stream);
+        if (st != AGX_OK) return st;
+        launches += h->last_launches;
+    }
     auto d2h = [&](void* dst, size_t off, size_t bytes) {
         if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, ws + off, bytes, cudaMemcpyDeviceToHost, stream);
     };
     d2h(h_out, L.out, L.q_bytes);
-    d2h(h_accept, L.acc, (size_t)B * 4); d2h(h_next, L.next, (size_t)B * 4); d2h(h_seq_lens, L.seqlen, (size_t)B * 4);
+    if (with_accept) {
+        d2h(h_accept, L.acc, (size_t)B * 4); d2h(h_next, L.next, (size_t)B * 4); d2h(h_seq_lens, L.seqlen, (size_t)B * 4);
+    }
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return cuda_fail(h, e, "host step: download");
     h->last_launches = launches;

@@ -470,7 +470,6 @@ cudaError_t launch_small(const AttnParams& p, cudaStream_t stream) {
 }  // namespace
 
 int attn_small_bf16_kv_tile() { return kStageTokens; }
-bool attn_tile_available() { return false; }
 
 cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, cudaStream_t stream) {
     if (p.num_items == 0) return cudaSuccess;

@@ -1,0 +1,531 @@
+// Large-q attention over a paged KV cache: the uncached suffix of a prompt attending over its cached
+// prefix plus itself (Sec. 2.3, prefix caching; Sec. 4.2 makes the suffix a few hundred tokens over a
+// prefix of thousands).  Here Q K^T and P V are dense contractions, so they run on the 5th-generation
+// tensor cores: tcgen05.mma issued by one thread, operands staged in shared memory by TMA,
+// accumulators in tensor memory (TMEM).
+//
+// Work item = (sequence, KV head g, chunk of 256 query rows, KV split).  The q * G rows of one KV
+// head (row r = i * G + h % G) are cut into two 128-row tiles A and B that share every K/V tile.
+// CTA = 12 warps:
+//   warp 0      TMA producer: per 128-token tile, 8 pages x 2 boxes of [16 tokens][64 dims] for K and
+//               for V (SWIZZLE_128B), page ids read through the page table; 2-stage rings.
+//   warp 1      MMA issuer (one lane) and TMEM owner.  Order on the tensor pipe:
+//               S_A(0) S_B(0) | O_A+=P_A V(t)  S_A(t+1)  O_B+=P_B V(t)  S_B(t+1) | ...
+//               so the softmax of one tile overlaps the MMAs of the other.
+//   warps 4-7   softmax of tile A, warps 8-11 softmax of tile B: one thread per query row (TMEM lane),
+//               S read with tcgen05.ld, P written back over S as packed bf16 (A operand of the P V MMA
+//               comes from TMEM), O rescaled in TMEM only when the row maximum grew by more than 2^8.
+// TMEM columns: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512).
+// Every mbarrier wait is bounded: on time-out the CTA records AGX_DEV_WAIT_TIMEOUT and tears down.
+#include <cuda.h>
+#include <math.h>
+
+#include "agx_internal.cuh"
+
+namespace agx {
+
+namespace {
+
+constexpr int kD = 128;
+constexpr int kBN = 128;                    // KV tokens per tile
+constexpr int kRowsPerCta = 256;
+constexpr int kStages = 2;
+constexpr int kThreads = 384;
+constexpr uint32_t kTileBytes = 128 * 256;  // one operand tile: [2 halves of 64 dims][128 rows][128 B]
+constexpr uint32_t kHalfBytes = 128 * 128;
+constexpr uint32_t kOffQ = 0;
+constexpr uint32_t kOffK = 2 * kTileBytes;
+constexpr uint32_t kOffV = kOffK + kStages * kTileBytes;
+constexpr uint32_t kOffBar = kOffV + kStages * kTileBytes;
+constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // + barriers + alignment slack
+constexpr long long kWaitLimitCycles = 4000000000ll;   // ~2 s at 1.9 GHz
+constexpr float kRescaleThreshold = 8.0f;              // log2 units
+
+// barrier slots (8 bytes each)
+enum { BAR_K_FULL = 0, BAR_K_EMPTY = 2, BAR_V_FULL = 4, BAR_V_EMPTY = 6, BAR_S_FULL = 8, BAR_P_READY = 10,
+       BAR_O_FULL = 12, BAR_COUNT = 13 };
+
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 256;  // + 128 * tile
+
+// tcgen05 instruction descriptor, kind::f16: D = f32, A = B = bf16, M = 128, N = 128
+constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescQK = kIdescBase;              // A, B both K-major
+constexpr uint32_t kIdescPV = kIdescBase | (1u << 16); // B (= V) is MN-major
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// shared-memory matrix descriptor, SWIZZLE_128B, descriptor version 1
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the CTA's abort flag) when the limit is hit or another
+// role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    int spins = 0;
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitLimitCycles) {
+                *abort_flag = 1;
+                atomicOr(status, AGX_DEV_WAIT_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_x64(uint32_t taddr, uint32_t (&r)[64]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+                 : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st_x32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n"
+                 :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]));
+}
+
+
+__device__ __forceinline__ int find_seq(const AttnParams& p, int item) {
+    int s = 0;
+#pragma unroll 1
+    for (int i = 1; i < p.num_seqs; ++i)
+        if (p.seq[i].item0 <= item) s = i;
+    return s;
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtensorMap map_k,
+                      const __grid_constant__ CUtensorMap map_v) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+    volatile int* abort_flag = (volatile int*)(smem + kOffBar + BAR_COUNT * 8);
+    uint32_t* tmem_slot = (uint32_t*)(smem + kOffBar + BAR_COUNT * 8 + 8);
+    auto bar = [&](int i) { return smem_base + kOffBar + 8u * i; };
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // ---- work item
+    const int si = find_seq(p, blockIdx.x);
+    const SeqPlan sp = p.seq[si];
+    int local = blockIdx.x - sp.item0;  // ((g * row_chunks) + rc) * nsplit + split
+    const int split = local % sp.nsplit;
+    local /= sp.nsplit;
+    const int rc = local % sp.row_chunks;
+    const int g = local / sp.row_chunks;
+    const int G = p.hq / p.hkv;
+    const int P = sp.prefix_len, q = sp.q_len, L = P + q;
+    const int rows = q * G;
+    const int row0 = rc * kRowsPerCta;
+    const int vis_end = P + min(q - 1, (row0 + kRowsPerCta - 1) / G) + 1;  // tokens the chunk's last row sees
+    const int kv_begin = split * sp.split_tokens;
+    const int kv_end = min(vis_end, kv_begin + sp.split_tokens);
+    const int n_tiles = max(0, (kv_end - kv_begin + kBN - 1) / kBN);
+
+    if (n_tiles == 0) {  // nothing visible in this split: publish empty partials (nsplit > 1 by construction)
+        for (int idx = tid; idx < kRowsPerCta * (kD / 4); idx += kThreads) {
+            const int r = row0 + idx / (kD / 4), c4 = (idx % (kD / 4)) * 4;
+            if (r >= rows) continue;
+            const int i = r / G, h = g * G + (r - i * G);
+            const long long e = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit + split;
+            *(float4*)(p.part_o + e * kD + c4) = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c4 == 0) p.part_ml[e] = make_float2(-INFINITY, 0.f);
+        }
+        return;
+    }
+
+    // ---- setup: barriers, TMEM, Q tiles
+    if (tid == 0) {
+        for (int i = 0; i < BAR_COUNT; ++i) mbar_init(bar(i), (i == BAR_P_READY || i == BAR_P_READY + 1) ? 128u : 1u);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&map_k) : "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&map_v) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    // Q: 256 rows x 256 B, plain 16-byte loads, written in the 128-byte-swizzled K-major operand layout
+    for (int c = tid; c < kRowsPerCta * 16; c += kThreads) {
+        const int rl = c >> 4, ch = c & 15;     // row in chunk, 16-byte chunk of the 256-byte row
+        const int r = row0 + rl;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (r < rows) {
+            const int i = r / G, hg = r - i * G;
+            v = __ldg((const uint4*)((const unsigned char*)p.q + (((long long)(sp.q_row0 + i) * p.hq + g * G + hg) * 256 + ch * 16)));
+        }
+        const int tile = rl >> 7, rt = rl & 127, half = ch >> 3, u = ch & 7;
+        *(uint4*)(smem + kOffQ + tile * kTileBytes + half * kHalfBytes + rt * 128 + ((u ^ (rt & 7)) << 4)) = v;
+    }
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    auto pages_in_tile = [&](int t) { return min(8, (kv_end - (kv_begin + t * kBN) + kPage - 1) / kPage); };
+
+    if (warp == 0) {
+        // ================= TMA producer (whole warp stays converged; lane 0 issues) =================
+        const int* pt_row = p.page_table + (long long)sp.seq_index * p.pt_stride;
+        const int page0 = kv_begin / kPage;
+        const int n_pages_total = (kv_end - kv_begin + kPage - 1) / kPage;
+        int ids = 0;  // page ids of the current group of 4 tiles: lane l holds page (group * 32 + l)
+        bool ok = true;
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            if ((t & 3) == 0) {
+                const int pi = t * 8 + lane;
+                long long id = 0;
+                if (pi < n_pages_total) {
+                    id = __ldg(pt_row + page0 + pi);
+                    if (id < 0 || id >= p.num_pages) { id = 0; atomicOr(p.status, AGX_DEV_BAD_PAGE); }
+                }
+                ids = (int)id;
+            }
+            const int stage = t & 1, ph = (t >> 1) & 1;
+            const int npg = pages_in_tile(t);
+            const int tok0 = kv_begin + t * kBN;
+            // ---- K
+            ok = mbar_wait(bar(BAR_K_EMPTY + stage), ph ^ 1, abort_flag, p.status);
+            if (!ok) break;
+            if (lane == 0) mbar_arrive_expect_tx(bar(BAR_K_FULL + stage), npg * 4096u);
+            for (int pg = 0; pg < npg; ++pg) {
+                const int id = __shfl_sync(0xFFFFFFFFu, ids, (t & 3) * 8 + pg);
+                if (lane == 0) {
+                    const int y = (id * p.hkv + g) * kPage;
+                    const uint32_t dst = smem_base + kOffK + stage * kTileBytes + pg * 2048;
+                    tma_load_2d(dst, &map_k, 0, y, bar(BAR_K_FULL + stage));
+                    tma_load_2d(dst + kHalfBytes, &map_k, 64, y, bar(BAR_K_FULL + stage));
+                }
+            }
+            // ---- V (the page that holds token L, if L is not page-aligned, is copied by hand so that
+            //      slots past the end of the sequence are zeros whatever the pool holds there)
+            ok = mbar_wait(bar(BAR_V_EMPTY + stage), ph ^ 1, abort_flag, p.status);
+            if (!ok) break;
+            const int ragged_pg = ((L & 15) != 0 && (L >> 4) >= (tok0 >> 4) && (L >> 4) < (tok0 >> 4) + npg) ? (L >> 4) - (tok0 >> 4) : -1;
+            if (ragged_pg >= 0) {
+                const int id = __shfl_sync(0xFFFFFFFFu, ids, (t & 3) * 8 + ragged_pg);
+                const unsigned char* src = (const unsigned char*)p.v_pool + ((long long)id * p.hkv + g) * (kPage * 256);
+                const int valid_rows = L & 15;
+                for (int idx = lane; idx < 256; idx += 32) {
+                    const int r = idx >> 4, ch = idx & 15, half = ch >> 3, u = ch & 7;
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (r < valid_rows) v = __ldg((const uint4*)(src + r * 256 + ch * 16));
+                    *(uint4*)(smem + kOffV + stage * kTileBytes + half * kHalfBytes + ragged_pg * 2048 + r * 128 + ((u ^ (r & 7)) << 4)) = v;
+                }
+                asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+                __syncwarp();
+            }
+            if (lane == 0) mbar_arrive_expect_tx(bar(BAR_V_FULL + stage), (npg - (ragged_pg >= 0 ? 1 : 0)) * 4096u);
+            for (int pg = 0; pg < npg; ++pg) {
+                const int id = __shfl_sync(0xFFFFFFFFu, ids, (t & 3) * 8 + pg);
+                if (lane == 0 && pg != ragged_pg) {
+                    const int y = (id * p.hkv + g) * kPage;
+                    const uint32_t dst = smem_base + kOffV + stage * kTileBytes + pg * 2048;
+                    tma_load_2d(dst, &map_v, 0, y, bar(BAR_V_FULL + stage));
+                    tma_load_2d(dst + kHalfBytes, &map_v, 64, y, bar(BAR_V_FULL + stage));
+                }
+            }
+        }
+        // drain: the copies this warp started must land before the CTA's shared memory goes away
+        if (lane == 0) {
+            for (int t = max(0, n_tiles - kStages); t < n_tiles; ++t) {
+                mbar_wait(bar(BAR_K_FULL + (t & 1)), (t >> 1) & 1, abort_flag, p.status);
+                mbar_wait(bar(BAR_V_FULL + (t & 1)), (t >> 1) & 1, abort_flag, p.status);
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            const uint32_t q_addr[2] = {smem_base + kOffQ, smem_base + kOffQ + kTileBytes};
+            const uint32_t tS[2] = {tmem_base + kColS, tmem_base + kColS + 128};
+            const uint32_t tO[2] = {tmem_base + kColO, tmem_base + kColO + 128};
+            auto issue_qk = [&](int x, int stage) {   // S_x = Q_x K^T : 8 k-steps of 16 dims
+                const uint32_t k_addr = smem_base + kOffK + stage * kTileBytes;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                    umma_ss(tS[x], make_desc(q_addr[x] + off, 16, 1024), make_desc(k_addr + off, 16, 1024), kIdescQK, ks > 0);
+                }
+            };
+            auto issue_pv = [&](int x, int stage, int npg, bool first) {  // O_x += P_x V : one k-step per page
+                const uint32_t v_addr = smem_base + kOffV + stage * kTileBytes;
+                for (int ks = 0; ks < npg; ++ks)
+                    umma_ts(tO[x], tS[x] + ks * 8, make_desc(v_addr + ks * 2048, kHalfBytes, 1024), kIdescPV, !(first && ks == 0));
+            };
+            bool ok = mbar_wait(bar(BAR_K_FULL + 0), 0, abort_flag, p.status);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(0, 0); umma_commit(bar(BAR_S_FULL + 0));
+                issue_qk(1, 0); umma_commit(bar(BAR_S_FULL + 1));
+                umma_commit(bar(BAR_K_EMPTY + 0));
+            }
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                const int stage = t & 1, ph = (t >> 1) & 1, npg = pages_in_tile(t);
+                const bool more = t + 1 < n_tiles;
+                const int nstage = (t + 1) & 1, nph = ((t + 1) >> 1) & 1;
+                ok = mbar_wait(bar(BAR_V_FULL + stage), ph, abort_flag, p.status);
+                if (!ok) break;
+                ok = mbar_wait(bar(BAR_P_READY + 0), t & 1, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                issue_pv(0, stage, npg, t == 0);
+                if (more) {
+                    ok = mbar_wait(bar(BAR_K_FULL + nstage), nph, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(0, nstage); umma_commit(bar(BAR_S_FULL + 0));
+                }
+                ok = mbar_wait(bar(BAR_P_READY + 1), t & 1, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                issue_pv(1, stage, npg, t == 0);
+                umma_commit(bar(BAR_V_EMPTY + stage));
+                if (more) {
+                    issue_qk(1, nstage); umma_commit(bar(BAR_S_FULL + 1));
+                    umma_commit(bar(BAR_K_EMPTY + nstage));
+                }
+            }
+            umma_commit(bar(BAR_O_FULL));  // arrives when every MMA issued above has completed
+            mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
+        }
+        __syncwarp();
+    } else if (warp >= 4) {
+        // ================= softmax + epilogue: one thread per query row =================
+        const int x = (warp - 4) >> 2;                       // tile A / B
+        const int rt = ((warp & 3) << 5) + lane;             // row in tile == TMEM lane
+        const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
+        const uint32_t tS = tmem_base + lane_addr + kColS + x * 128;
+        const uint32_t tO = tmem_base + lane_addr + kColO + x * 128;
+        const int r = row0 + x * 128 + rt;
+        const int limit = P + min(r / G, q - 1);             // last token this row sees
+        const int tile_i_min = min((row0 + x * 128) / G, q - 1);
+        float m_ref = -INFINITY, l_sum = 0.f;
+        bool ok = true;
+        for (int t = 0; t < n_tiles; ++t) {
+            ok = mbar_wait(bar(BAR_S_FULL + x), t & 1, abort_flag, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            const int tok0 = kv_begin + t * kBN;
+            const bool masked = (tok0 + kBN - 1 > P + tile_i_min) || (tok0 + kBN > kv_end);  // uniform per tile
+            const int nvis = max(0, min(min(limit + 1, kv_end) - tok0, kBN));            // visible columns: [0, nvis)
+            uint32_t sreg[64];
+            // ---- pass 1: row maximum
+            float mx = -INFINITY;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                tmem_ld_x64(tS + hf * 64, sreg);
+                tmem_wait_ld();
+                if (masked) {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) mx = fmaxf(mx, (hf * 64 + c < nvis) ? __uint_as_float(sreg[c]) : -INFINITY);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sreg[c]));
+                }
+            }
+            const float m_tile = mx * p.scale_log2;
+            const bool need = m_tile > m_ref + kRescaleThreshold;
+            if (__any_sync(0xFFFFFFFFu, need)) {
+                const float m_new = need ? m_tile : m_ref;
+                const float factor = need ? ex2(m_ref - m_new) : 1.f;   // m_ref = -inf gives 0
+                if (t > 0) {
+                    uint32_t oreg[32];
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        tmem_ld_x32(tO + c4 * 32, oreg);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * factor);
+                        tmem_st_x32(tO + c4 * 32, oreg);
+                    }
+                    tmem_wait_st();
+                }
+                l_sum *= factor;
+                m_ref = m_new;
+            }
+            const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+            // ---- pass 2: P = 2^(S * scale - m), packed bf16 pairs written over S
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                tmem_ld_x64(tS + hf * 64, sreg);
+                tmem_wait_ld();
+                uint32_t preg[32];
+#pragma unroll
+                for (int c = 0; c < 64; c += 2) {
+                    float p0 = ex2(fmaf(__uint_as_float(sreg[c]), p.scale_log2, -m_use));
+                    float p1 = ex2(fmaf(__uint_as_float(sreg[c + 1]), p.scale_log2, -m_use));
+                    if (masked) {
+                        if (hf * 64 + c >= nvis) p0 = 0.f;
+                        if (hf * 64 + c + 1 >= nvis) p1 = 0.f;
+                    }
+                    l_sum += p0 + p1;
+                    preg[c >> 1] = pack_bf16(p0, p1);
+                }
+                tmem_st_x32(tS + hf * 32, preg);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar(BAR_P_READY + x));
+        }
+        // ---- epilogue
+        if (ok) ok = mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
+        if (ok) {
+            tc_fence_after();
+            const bool valid = r < rows;
+            const int i = r / G, h = g * G + (r - (r / G) * G);
+            const float inv = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
+            uint32_t oreg[32];
+            if (sp.nsplit == 1) {
+                __nv_bfloat16* dst = (__nv_bfloat16*)p.out + ((long long)(sp.q_row0 + i) * p.hq + h) * kD;
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    tmem_ld_x32(tO + c4 * 32, oreg);
+                    tmem_wait_ld();
+                    if (valid) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            uint4 pk;
+                            pk.x = pack_bf16(__uint_as_float(oreg[8 * v + 0]) * inv, __uint_as_float(oreg[8 * v + 1]) * inv);
+                            pk.y = pack_bf16(__uint_as_float(oreg[8 * v + 2]) * inv, __uint_as_float(oreg[8 * v + 3]) * inv);
+                            pk.z = pack_bf16(__uint_as_float(oreg[8 * v + 4]) * inv, __uint_as_float(oreg[8 * v + 5]) * inv);
+                            pk.w = pack_bf16(__uint_as_float(oreg[8 * v + 6]) * inv, __uint_as_float(oreg[8 * v + 7]) * inv);
+                            *(uint4*)(dst + c4 * 32 + v * 8) = pk;
+                        }
+                    }
+                }
+                if (valid && p.lse) p.lse[(long long)(sp.q_row0 + i) * p.hq + h] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+            } else {
+                const long long e = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit + split;
+                float* dst = p.part_o + e * kD;
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    tmem_ld_x32(tO + c4 * 32, oreg);
+                    tmem_wait_ld();
+                    if (valid) {
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            *(uint4*)(dst + c4 * 32 + v * 4) = make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
+                    }
+                }
+                if (valid) p.part_ml[e] = make_float2(m_ref, l_sum);
+            }
+        }
+    }
+    // ---- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// --------------------------------------------------------------------------------------------
+bool attn_tile_available() { return true; }
+
+namespace {
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+    }
+    return fn;
+}
+// 2-D view of a pool: [num_pages * Hkv * 16 rows][128 dims] bf16; box = 16 rows x 64 dims, 128-byte swizzle
+bool make_pool_map(CUtensorMap* map, const void* pool, long long num_pages, int hkv) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)num_pages * hkv * kPage};
+    const cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kPage};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(pool), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+}  // namespace
+
+cudaError_t launch_attn_tile_bf16(const AttnParams& p, cudaStream_t stream) {
+    if (p.num_items == 0) return cudaSuccess;
+    if ((long long)p.num_pages * p.hkv * kPage > 0x7FFFFFFFll) return cudaErrorInvalidValue;
+    alignas(64) CUtensorMap map_k, map_v;
+    if (!make_pool_map(&map_k, p.k_pool, p.num_pages, p.hkv) || !make_pool_map(&map_v, p.v_pool, p.num_pages, p.hkv))
+        return cudaErrorNotSupported;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(attn_tile_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    attn_tile_bf16_kernel<<<p.num_items, kThreads, kSmemBytes, stream>>>(p, map_k, map_v);
+    return cudaGetLastError();
+}
+
+}  // namespace agx

@@ -60,9 +60,7 @@ cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, 
 
 bool attn_tile_available();
 // Large-q tensor-core tile kernel (bf16, d = 128, tcgen05 + TMEM + TMA).
-struct TileLaunch;  // opaque to other translation units
-cudaError_t launch_attn_tile_bf16(const AttnParams& p, const void* tmap_k, const void* tmap_v, int sm_count,
-                                  cudaStream_t stream);
+cudaError_t launch_attn_tile_bf16(const AttnParams& p, cudaStream_t stream);
 
 cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_stride, int vocab, const int* drafts,
                           const int* cu_q, int B, int total_q, int* accept_len, int* next_token, int* argmax,

@@ -237,3 +237,50 @@ def test_argument_errors_are_reported_not_faulted():
     with pytest.raises(agx.AgxError) as e:  # split launch without workspace
         b2.h.attn_prefixed(b2.q_block, b2.k_pool, b2.v_pool, b2.page_table, w2.prefix_len, w2.q_len, b2.out)
     assert e.value.status == -1
+
+
+# ------------------------------------------------------------------ tensor-core tile kernel (large q)
+@pytest.mark.parametrize("P,q,hq,hkv", [
+    (0, 128, 8, 2),        # pure causal prefill, G = 4, one tile pair, exact multiples
+    (256, 64, 8, 2),       # 256 rows: exactly one CTA chunk
+    (100, 90, 6, 2),       # G = 3, ragged rows, P not page-aligned
+    (777, 130, 32, 8),     # L % 16 != 0 (ragged last page), several chunks
+    (3000, 40, 32, 8),     # 160 rows: tile B mostly padding
+    (1030, 300, 24, 8),    # G = 3, several KV splits
+    (5, 200, 4, 4),        # G = 1 (MHA)
+])
+def test_tile_kernel_shapes(P, q, hq, hkv):
+    w = W.make_attn_workload(f"tile_{P}_{q}", 2000 + P + q, "bf16", hq, hkv, 128, [P], [q], spare_pages=2)
+    run_and_check(w, sample=(11, 150), poison=True)
+
+
+def test_c3_prefix_cached_prefill_and_full_prefill_rows():
+    """Prefix-cached prefill (P = 3072, q = 512, 24/8 heads) against the oracle, and the oracle's own
+    check that these rows equal rows 3072.. of a full 3584-token uncached prefill."""
+    w = W.c3_prefix_prefill()
+    b, stats = run_and_check(w, sample=(5, 300), strict=True)
+    out = b.out.to(torch.float64).cpu().numpy()
+    kp, vp = oracle_pools_after_append(w)
+    P, q = 3072, 512
+    K = W.gather_contiguous(kp, w.page_table[0], P + q); V = W.gather_contiguous(vp, w.page_table[0], P + q)
+    rng = np.random.default_rng(1)
+    si = rng.integers(0, q, 40).astype(np.int32); sh = rng.integers(0, 24, 40).astype(np.int32)
+    Qfull = np.zeros((P + q, 24, 128), dtype=np.uint16); Qfull[P:] = w.q_block
+    full, _, _ = oracle.attn_contiguous(Qfull, K, V, "bf16", 0, select=(si + P, sh))
+    check_attention(out[si, sh], full, "c3 vs full prefill rows", strict=True)
+
+
+def test_tile_and_small_kernels_in_one_ragged_batch():
+    P = [2048, 2300, 2048 + 7, 4000, 2600, 3000]
+    q = [8, 200, 1, 130, 16, 513]
+    w = W.make_attn_workload("mixed", 91, "bf16", 32, 8, 128, P, q, shared_prefix_tokens=2048)
+    b, _ = run_and_check(w, sample=(2, 60))
+    assert b.launches >= 3
+
+
+def test_tile_kernel_matches_mma_sync_baseline(monkeypatch):
+    w = W.make_attn_workload("tile_vs_mma", 17, "bf16", 32, 8, 128, [900], [260])
+    b = DeviceBatch(w); b.append(); a, _ = b.attend()
+    monkeypatch.setenv("AGX_FORCE_MMA_SYNC", "1")
+    b2 = DeviceBatch(w); b2.append(); c, _ = b2.attend()
+    assert np.max(np.abs(a - c)) < 2e-2
