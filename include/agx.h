@@ -179,6 +179,38 @@ AGX_API agx_status agx_accept_greedy(agx_handle* handle, const void* logits, int
                              void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * agx_accept_greedy_static - agx_accept_greedy for callers that cannot allocate device memory.
+ * The paper has no counterpart: this is a packaging variant of the accept step above, with the
+ * same inputs, outputs and results.
+ *
+ * Who needs it: code that verifies drafts from inside a memory arena sized once at start-up (an
+ * embedded or serving runtime with a fixed device-memory budget), or next to an allocator it does
+ * not own, where a cudaMalloc may synchronise the whole device, fragment the pool or simply be
+ * forbidden.  This call takes no handle and no workspace and performs no allocation of any kind;
+ * it uses a fixed scratch array inside the library (about 73 KB of device memory on every GPU that
+ * loads the library, held until the process exits).
+ *
+ * Limits: total_q <= 2048 logits rows per call, and rows x vocabulary chunks <= 8192 (the call
+ * uses fewer, larger chunks to stay inside that); larger requests return AGX_E_RANGE and should
+ * use agx_accept_greedy with a workspace.
+ *
+ * The first call on each device looks up the device address of the scratch array (that device
+ * must be current); make that first call outside any stream capture.  Every call uses the same
+ * array: the call clears the part that has to start at zero, but two calls that overlap on the GPU
+ * (different streams, no ordering between them) race on it and give undefined results.  Calls on
+ * one stream, or ordered by events, are safe.
+ *
+ * Arguments and error codes are those of agx_accept_greedy; every pointer is a device pointer.
+ * There is no handle, so no error text is kept: the status code is all a failing call reports.
+ */
+AGX_API agx_status agx_accept_greedy_static(const void* logits, int32_t logits_dtype,
+                                            int64_t row_stride, int32_t vocab,
+                                            const int32_t* drafts, const int32_t* cu_q, int32_t B,
+                                            int32_t total_q, int32_t* accept_len,
+                                            int32_t* next_token, int32_t* argmax,
+                                            int32_t* seq_lens, void* stream);
+
+/*
  * agx_get_status - synchronise the stream, read and clear the device status word.
  * *device_status receives the AGX_DEV_* bits (0 = clean).  Returns AGX_E_DEVICE when non-zero.
  */

@@ -25,7 +25,7 @@ EXPORTS = (
     "agx_create", "agx_destroy", "agx_status_string", "agx_last_error", "agx_kv_append",
     "agx_attn_workspace_bytes", "agx_attn_prefixed", "agx_accept_workspace_bytes",
     "agx_accept_greedy", "agx_get_status", "agx_last_launch_count",
-    "agx_verify_step_host_workspace_bytes", "agx_verify_step_host",
+    "agx_verify_step_host_workspace_bytes", "agx_verify_step_host", "agx_accept_greedy_static",
 )
 
 
@@ -84,6 +84,8 @@ def load() -> ctypes.CDLL:
                                          vp, vp, vp, vp,                        # host outputs
                                          vp, ctypes.c_size_t, vp]
     lib.agx_verify_step_host.restype = i32
+    lib.agx_accept_greedy_static.argtypes = [vp, i32, i64, i32, vp, vp, i32, i32, vp, vp, vp, vp, vp]
+    lib.agx_accept_greedy_static.restype = i32
     _lib = lib
     return lib
 
@@ -112,6 +114,18 @@ def _stream_ptr(stream) -> Optional[int]:
 
 def _h_i32(a) -> np.ndarray:
     return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def accept_greedy_static(logits, logits_dtype: str, vocab: int, drafts, cu_q, accept_len, next_token, argmax=None,
+                         seq_lens=None, stream=None) -> None:
+    """agx_accept_greedy_static: the accept step without handle, workspace or any allocation (for
+    callers that may not allocate device memory).  Same tensors as ``Handle.accept_greedy``."""
+    B = int(cu_q.shape[0]) - 1
+    st = load().agx_accept_greedy_static(_ptr(logits), DTYPES[logits_dtype], int(logits.stride(0)), int(vocab),
+                                         _ptr(drafts), _ptr(cu_q), B, int(logits.shape[0]), _ptr(accept_len),
+                                         _ptr(next_token), _ptr(argmax), _ptr(seq_lens), _stream_ptr(stream))
+    if st != AGX_OK:
+        raise AgxError(st, "agx_accept_greedy_static")
 
 
 class Handle:

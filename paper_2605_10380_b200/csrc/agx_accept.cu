@@ -170,3 +170,80 @@ cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_st
 }
 
 }  // namespace agx
+
+// --------------------------------------------------------------------------------------------
+// Allocation-free variant of the accept step.
+//
+// Some callers cannot allocate device memory at the point where they verify drafts: code running
+// inside a pre-sized serving arena or an embedded runtime whose memory is fixed at start-up, and
+// code that must not disturb a caching allocator owned by someone else (a cudaMalloc there can
+// synchronise the device or fail outright).  agx_accept_greedy needs a caller-provided workspace
+// and a handle whose creation allocates; the entry point below needs neither.  Its scratch (the
+// per-chunk argmax keys, the per-row winners and the ticket counter) lives in a fixed array that
+// is part of the loaded module, so every GPU that loads the library carries these 73 KB until the
+// process exits.
+namespace agx {
+namespace {
+constexpr int kStaticMaxRows = 2048;    // logits rows per call
+constexpr int kStaticMaxSlots = 8192;   // rows * chunks partial keys per call
+constexpr int kStaticDevices = 64;
+// layout: [0, 256) ticket counter | partial keys (8 B each) | per-row winners (4 B each)
+constexpr size_t kStaticBytes = 256 + (size_t)kStaticMaxSlots * 8 + (size_t)kStaticMaxRows * 4;
+static __device__ __align__(256) unsigned char g_accept_scratch[kStaticBytes];
+
+struct StaticDeviceState {
+    void* scratch;  // device address of g_accept_scratch on that device (NULL until resolved)
+    int sm_count;
+};
+StaticDeviceState g_static_state[kStaticDevices];
+}  // namespace
+}  // namespace agx
+
+extern "C" AGX_API agx_status agx_accept_greedy_static(const void* logits, int32_t logits_dtype, int64_t row_stride,
+                                                       int32_t vocab, const int32_t* drafts, const int32_t* cu_q,
+                                                       int32_t B, int32_t total_q, int32_t* accept_len,
+                                                       int32_t* next_token, int32_t* argmax, int32_t* seq_lens,
+                                                       void* stream) {
+    using namespace agx;
+    if (B < 0 || total_q < 0) return AGX_E_INVAL;
+    if (B == 0) return AGX_OK;
+    if (total_q < B) return AGX_E_INVAL;
+    if (logits_dtype != AGX_BF16 && logits_dtype != AGX_F32) return AGX_E_UNSUPPORTED;
+    if (vocab < 1 || row_stride < vocab) return AGX_E_RANGE;
+    if (!logits || !cu_q || !accept_len || !next_token || (!drafts && total_q > B)) return AGX_E_INVAL;
+    if (total_q > kStaticMaxRows) return AGX_E_RANGE;  // beyond the fixed scratch: use agx_accept_greedy
+
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kStaticDevices) return AGX_E_CUDA;
+    StaticDeviceState& st = g_static_state[device];
+    if (!st.scratch) {
+        // One-time set-up for this device, with it current.  In host code the array's name is only a
+        // stand-in for the symbol; the address kernels can use has to be asked for.
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_accept_scratch) != cudaSuccess || !ptr) return AGX_E_CUDA;
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1) return AGX_E_CUDA;
+        st.sm_count = sms;
+        st.scratch = ptr;
+    }
+    // same chunking rule as the workspace variant, then shrunk to the fixed number of slots
+    const int vec = logits_dtype == AGX_BF16 ? 8 : 4;
+    int want = (2 * st.sm_count + total_q - 1) / total_q;
+    const int max_chunks = (vocab + 256 * vec * 2 - 1) / (256 * vec * 2);
+    if (want > max_chunks) want = max_chunks;
+    if (want > kStaticMaxSlots / total_q) want = kStaticMaxSlots / total_q;
+    if (want < 1) want = 1;
+    int chunk_elems = (vocab + want - 1) / want;
+    chunk_elems = (chunk_elems + vec - 1) / vec * vec;
+    const int chunks = (vocab + chunk_elems - 1) / chunk_elems;
+    if ((long long)chunks * total_q > kStaticMaxSlots) return AGX_E_RANGE;
+
+    unsigned char* base = (unsigned char*)st.scratch;
+    // the array keeps whatever the previous call left: the ticket counter must start at zero
+    if (cudaMemsetAsync(base, 0, 256, (cudaStream_t)stream) != cudaSuccess) return AGX_E_CUDA;
+    // launch_accept places the per-row winners right behind total_q * chunks keys
+    cudaError_t e = launch_accept(logits, logits_dtype, row_stride, vocab, drafts, cu_q, B, total_q, accept_len,
+                                  next_token, argmax, seq_lens, (unsigned long long*)(base + 256), chunks,
+                                  (unsigned int*)base, (cudaStream_t)stream);
+    return e == cudaSuccess ? AGX_OK : AGX_E_CUDA;
+}
