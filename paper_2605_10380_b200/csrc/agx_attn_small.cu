@@ -9,13 +9,16 @@
 //
 // Work item = (sequence, KV head, KV split).  A CTA of 4 * MT warps: warp (mt, kg) owns query rows
 // [16 mt, 16 mt + 16) and, in every 64-token stage, page kg.  K/V pages stream through a
-// multi-stage cp.async ring (16-byte chunks, XOR-swizzled rows so ldmatrix is conflict-free); the
-// four KV groups keep private online-softmax states that are merged through shared memory at the
-// end.  Splits write fp32 (m, l, O) partials; a combine kernel merges them in fixed order, so
+// multi-stage ring filled by TMA (per page two [16 tokens][64 dims] boxes for K and for V,
+// SWIZZLE_128B so ldmatrix is conflict-free; page ids come from the page table, prefetched 32 at a
+// time) and handed over with full/empty mbarriers, so no thread spends instructions on addresses and
+// warps never meet at a CTA-wide barrier inside the loop; the four KV groups keep private
+// online-softmax states that are merged through shared memory at the end.  Splits write fp32 (m, l, O) partials; a combine kernel merges them in fixed order, so
 // results are bit-reproducible run to run.
 #include <math.h>
 
 #include "agx_internal.cuh"
+#include "agx_sm100.cuh"
 
 namespace agx {
 
@@ -28,14 +31,7 @@ constexpr int kStageTokens = kKW * kPage;  // 64
 constexpr int kStageBytes = 2 * kStageTokens * kRowBytes;  // K + V = 32 KB
 constexpr int kMergeStride = 136;          // floats per merged row (conflict-free float2 stores)
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes));
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
@@ -50,10 +46,6 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
 }
 
 // byte offset of 16-byte chunk `ch` (0..15) of row `r` in a [rows][256 B] tile, XOR-swizzled
@@ -72,12 +64,21 @@ __device__ __forceinline__ int find_seq(const AttnParams& p, int item) {
 
 template <int MT, int NS>
 __global__ void __launch_bounds__(128 * MT, (MT <= 2) ? 2 : 1)
-attn_small_bf16_kernel(const __grid_constant__ AttnParams p) {
-    extern __shared__ __align__(1024) unsigned char smem[];
+attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtensorMap map_k,
+                       const __grid_constant__ CUtensorMap map_v) {
+    extern __shared__ unsigned char smem_raw[];
     constexpr int kThreads = 128 * MT;
-    constexpr int kQBytes = MT * 16 * kRowBytes;
-    unsigned char* q_smem = smem;
-    unsigned char* ring = smem + kQBytes;
+    constexpr int kWarps = 4 * MT;
+    constexpr int kRingBytes = NS * kStageBytes;
+    constexpr int kMergeBytes = MT * kKW * 16 * (kMergeStride * 4 + 8);
+    constexpr int kRegion = kRingBytes > kMergeBytes ? kRingBytes : kMergeBytes;
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* ring = smem_raw + (smem_base - smem_u32(smem_raw));   // 1024-aligned: TMA swizzle atoms
+    unsigned char* q_smem = ring + kRegion;
+    const uint32_t bar_base = smem_base + kRegion + MT * 16 * kRowBytes;  // full[NS], empty[NS]
+    volatile int* abort_flag = (volatile int*)(q_smem + MT * 16 * kRowBytes + 2 * NS * 8);
+    auto full_bar = [&](int i) { return bar_base + 8u * i; };
+    auto empty_bar = [&](int i) { return bar_base + 8u * (NS + i); };
 
     const int tid = threadIdx.x;
     const int lane = tid & 31;
@@ -95,6 +96,7 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p) {
     const int G = p.hq / p.hkv;
     const int P = sp.prefix_len;
     const int q = sp.q_len;
+    const int L = P + q;
     const int rows = q * G;          // query rows of this KV head, r = i * G + (h % G)
     const int row0 = rc * 16 * MT;   // first row of this CTA's chunk
     // the chunk's last row sees tokens 0 .. P + i_last
@@ -102,43 +104,15 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p) {
     const int tok_begin = split * sp.split_tokens;
     const int tok_end = min(vis_end, tok_begin + sp.split_tokens);
     const int n_stages = max(0, (tok_end - tok_begin + kStageTokens - 1) / kStageTokens);
-    const int* pt_row = p.page_table + (long long)sp.seq_index * p.pt_stride;
-    const unsigned char* k_pool = (const unsigned char*)p.k_pool;
-    const unsigned char* v_pool = (const unsigned char*)p.v_pool;
 
-    // ---- stage loader: 2048 16-byte chunks (K then V), each thread 2048 / kThreads of them
-    auto load_stage = [&](int stage) {
-        if (stage < n_stages) {
-            unsigned char* buf = ring + (stage % NS) * kStageBytes;
-            const int tok0 = tok_begin + stage * kStageTokens;
-#pragma unroll
-            for (int it = 0; it < 2048 / kThreads; ++it) {
-                const int c = it * kThreads + tid;
-                const int kv = c >> 10;
-                const int pg = (c >> 8) & 3;
-                const int r = (c >> 4) & 15;
-                const int ch = c & 15;
-                const int tok = tok0 + pg * kPage + r;
-                bool valid = tok < tok_end;
-                long long page = 0;
-                if (valid) {
-                    page = __ldg(pt_row + (tok >> 4));
-                    if (page < 0 || page >= p.num_pages) {
-                        valid = false;
-                        page = 0;
-                        atomicOr(p.status, AGX_DEV_BAD_PAGE);
-                    }
-                }
-                const unsigned char* src = (kv ? v_pool : k_pool) +
-                                           (((page * p.hkv + g) * kPage + r) * (long long)kRowBytes + ch * 16);
-                const uint32_t dst = smem_u32(buf + kv * (kStageTokens * kRowBytes) + pg * (kPage * kRowBytes)) + swz(r, ch);
-                cp_async16(dst, src, valid ? 16 : 0);
-            }
-        }
-        cp_async_commit();
-    };
-
-    // ---- Q tile -> shared (rows beyond q*G are zero), then A fragments in registers
+    if (tid == 0) {
+        for (int i = 0; i < NS; ++i) { mbar_init(full_bar(i), 1); mbar_init(empty_bar(i), kWarps); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&map_k) : "memory");
+        asm volatile("prefetch.tensormap [%0];\n" ::"l"(&map_v) : "memory");
+    }
+    // ---- Q tile -> shared (rows beyond q*G are zero)
     for (int c = tid; c < MT * 16 * 16; c += kThreads) {
         const int r = c >> 4, ch = c & 15;
         uint4 v = make_uint4(0, 0, 0, 0);
@@ -149,9 +123,57 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p) {
         }
         *(uint4*)(q_smem + swz(r, ch)) = v;
     }
+    __syncthreads();  // barriers initialised, Q tile visible
+
+    // ---- producer state (warp 0; lane 0 issues the TMA copies).  Page ids are fetched 32 at a time,
+    //      one group ahead, so the page-table latency never sits in front of a copy.
+    const int* pt_row = p.page_table + (long long)sp.seq_index * p.pt_stride;
+    const int page0 = tok_begin / kPage;
+    const int n_pages = (tok_end - tok_begin + kPage - 1) / kPage;
+    int ids_cur = 0, ids_next = 0, group_cur = 0;
+    auto fetch_ids = [&](int group) {
+        const int pi = group * 32 + lane;
+        long long id = 0;
+        if (pi < n_pages) {
+            id = __ldg(pt_row + page0 + pi);
+            if (id < 0 || id >= p.num_pages) { id = 0; atomicOr(p.status, AGX_DEV_BAD_PAGE); }
+        }
+        return (int)id;
+    };
+    bool alive = true;
+    auto produce = [&](int stage) {   // called by all lanes of warp 0
+        if (stage >= n_stages || !alive) return;
+        const int slot = stage % NS;
+        alive = mbar_wait(empty_bar(slot), ((stage / NS) & 1) ^ 1, abort_flag, p.status);
+        if (!alive) return;
+        const int pi0 = stage * kKW;
+        if ((pi0 >> 5) != group_cur) { ids_cur = ids_next; group_cur = pi0 >> 5; ids_next = fetch_ids(group_cur + 1); }
+        const int npg = min(kKW, n_pages - pi0);
+        int id[kKW];
 #pragma unroll
-    for (int s = 0; s < NS - 1; ++s) load_stage(s);
-    __syncthreads();  // Q tile visible
+        for (int pg = 0; pg < kKW; ++pg) id[pg] = __shfl_sync(0xFFFFFFFFu, ids_cur, (pi0 + pg) & 31);
+        if (lane == 0) {
+            mbar_arrive_expect_tx(full_bar(slot), npg * 8192u);
+            const uint32_t dst0 = smem_base + slot * kStageBytes;
+#pragma unroll
+            for (int pg = 0; pg < kKW; ++pg) {
+                if (pg < npg) {
+                    const int y = (id[pg] * p.hkv + g) * kPage;
+                    const uint32_t dk = dst0 + pg * 4096, dv = dk + kStageTokens * kRowBytes;
+                    tma_load_2d(dk, &map_k, 0, y, full_bar(slot));
+                    tma_load_2d(dk + 2048, &map_k, 64, y, full_bar(slot));
+                    tma_load_2d(dv, &map_v, 0, y, full_bar(slot));
+                    tma_load_2d(dv + 2048, &map_v, 64, y, full_bar(slot));
+                }
+            }
+        }
+    };
+    if (warp == 0) {
+        ids_cur = fetch_ids(0);
+        ids_next = fetch_ids(1);
+#pragma unroll
+        for (int s = 0; s < NS - 1; ++s) produce(s);
+    }
 
     uint32_t qa[8][4];
     {
@@ -176,17 +198,36 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p) {
         limit[0] = P + min(rA / G, q - 1);
         limit[1] = P + min((rA + 8) / G, q - 1);
     }
+    // Per-lane ldmatrix offsets inside one page of the TMA layout [half 2][16 rows][128 B], where the
+    // 16-byte unit u of row r sits at ((u ^ (r & 7)) << 4).  K (x4): row = nt*8 + lane%8, unit = (kp&1)*4 + lane/8.
+    // V (x4.trans): row = lane%8 + 8*((lane/8)&1), unit = (cp&3)*2 + lane/16.
+    const uint32_t k_x = ((lane >> 3) ^ (lane & 7));
+    const uint32_t k_off[2] = {(uint32_t)((lane & 7) * 128 + (k_x << 4)), (uint32_t)((lane & 7) * 128 + ((k_x ^ 4u) << 4))};
+    const uint32_t v_row = (lane & 7) + ((lane >> 3) & 1) * 8;
+    const uint32_t v_x = (lane >> 4) ^ (lane & 7);
+    uint32_t v_off[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v_off[j] = v_row * 128 + ((v_x ^ (uint32_t)(j << 1)) << 4);
 
     for (int stage = 0; stage < n_stages; ++stage) {
-        cp_async_wait<NS - 2>();
-        __syncthreads();             // stage data visible to all; ring slot (stage-1) % NS is free
-        load_stage(stage + NS - 1);  // refill it
+        const int slot = stage % NS;
+        if (warp == 0) produce(stage + NS - 1);
+        if (!mbar_wait(full_bar(slot), (stage / NS) & 1, abort_flag, p.status)) break;
 
         const int tok0 = tok_begin + stage * kStageTokens + kg * kPage;
         if (tok0 < tok_end) {
-            const unsigned char* buf = ring + (stage % NS) * kStageBytes;
-            const uint32_t k_base = smem_u32(buf + kg * (kPage * kRowBytes));
+            const uint32_t k_base = smem_base + slot * kStageBytes + kg * 4096;
             const uint32_t v_base = k_base + kStageTokens * kRowBytes;
+            // slots past the end of the sequence may hold anything: zero those V rows (P is 0 there,
+            // but 0 * NaN is not).  Every warp sharing the page writes the same zeros.
+            if (tok0 + kPage > L) {
+                const int valid_rows = L - tok0;
+                for (int idx = lane; idx < (kPage - valid_rows) * 16; idx += 32) {
+                    const int r = valid_rows + (idx >> 4), ch = idx & 15;
+                    *(uint4*)(ring + (v_base - smem_base) + (ch >> 3) * 2048 + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+                }
+                __syncwarp();
+            }
 
             // S = Q K^T for 16 tokens: two n-tiles of 8 tokens
             float s[2][4];
@@ -197,41 +238,38 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p) {
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt) {
                     uint32_t b0, b1, b2, b3;
-                    ldmatrix_x4(b0, b1, b2, b3, k_base + swz(nt * 8 + (lane & 7), kp * 4 + (lane >> 3)));
+                    ldmatrix_x4(b0, b1, b2, b3, k_base + (kp >> 1) * 2048 + nt * 1024 + k_off[kp & 1]);
                     mma_bf16(s[nt], qa[2 * kp], b0, b1);
                     mma_bf16(s[nt], qa[2 * kp + 1], b2, b3);
                 }
             }
-            // scale to log2 units, mask the causal edge / the end of the split
-            const bool need_mask = (tok0 + kPage - 1 > P) || (tok0 + kPage > tok_end);
+            // mask the causal edge / the end of the split (raw scores; the scale is folded into the exp)
+            if ((tok0 + kPage - 1 > P) || (tok0 + kPage > tok_end)) {
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt) {
+                for (int nt = 0; nt < 2; ++nt) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    float v = s[nt][e] * p.scale_log2;
-                    if (need_mask) {
+                    for (int e = 0; e < 4; ++e) {
                         const int tok = tok0 + nt * 8 + 2 * (lane & 3) + (e & 1);
-                        if (tok > limit[e >> 1] || tok >= tok_end) v = -INFINITY;
+                        if (tok > limit[e >> 1] || tok >= tok_end) s[nt][e] = -INFINITY;
                     }
-                    s[nt][e] = v;
                 }
             }
-            // online softmax for rows A (e = 0,1) and B (e = 2,3)
+            // online softmax for rows A (e = 0,1) and B (e = 2,3); running max kept in log2 units
             float corr[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 float mx = fmaxf(fmaxf(s[0][2 * h], s[0][2 * h + 1]), fmaxf(s[1][2 * h], s[1][2 * h + 1]));
                 mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
                 mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
-                const float m_new = fmaxf(m_run[h], mx);
+                const float m_new = fmaxf(m_run[h], mx * p.scale_log2);
                 const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
-                corr[h] = exp2f(m_run[h] - m_ref);
+                corr[h] = ex2(m_run[h] - m_ref);
                 m_run[h] = m_new;
                 float sum = 0.f;
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt) {
-                    s[nt][2 * h] = exp2f(s[nt][2 * h] - m_ref);
-                    s[nt][2 * h + 1] = exp2f(s[nt][2 * h + 1] - m_ref);
+                    s[nt][2 * h] = ex2(fmaf(s[nt][2 * h], p.scale_log2, -m_ref));
+                    s[nt][2 * h + 1] = ex2(fmaf(s[nt][2 * h + 1], p.scale_log2, -m_ref));
                     sum += s[nt][2 * h] + s[nt][2 * h + 1];
                 }
                 l_run[h] = l_run[h] * corr[h] + sum;
@@ -252,15 +290,15 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p) {
 #pragma unroll
             for (int cp = 0; cp < 8; ++cp) {
                 uint32_t b0, b1, b2, b3;
-                ldmatrix_x4_trans(b0, b1, b2, b3,
-                                  v_base + swz((lane & 7) + ((lane >> 3) & 1) * 8, cp * 2 + (lane >> 4)));
+                ldmatrix_x4_trans(b0, b1, b2, b3, v_base + (cp >> 2) * 2048 + v_off[cp & 3]);
                 mma_bf16(o[2 * cp], pa, b0, b1);
                 mma_bf16(o[2 * cp + 1], pa, b2, b3);
             }
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar(slot));
     }
-    cp_async_wait<0>();
-    __syncthreads();  // ring is dead: reuse it for the cross-group merge
+    __syncthreads();  // every armed stage has been consumed: the ring is dead, reuse it for the merge
 
     // ---- merge the 4 KV groups of each m-tile through shared memory
     float* merge_o = (float*)ring;                                    // [MT*4][16][kMergeStride]
@@ -420,17 +458,40 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
     if (sp.nsplit == 1) return;  // written directly by the attention kernel
     const int i = lrow - acc_rows;
     const long long e0 = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit;
+    const int ns = sp.nsplit;
+    // pass 1: lanes take splits side by side (independent loads), then warp reductions in fixed order
     float m_all = -INFINITY;
-    for (int k = 0; k < sp.nsplit; ++k) m_all = fmaxf(m_all, p.part_ml[e0 + k].x);
-    const int D = p.head_dim;
+    for (int k = lane; k < ns; k += 32) m_all = fmaxf(m_all, p.part_ml[e0 + k].x);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, off));
     float l_all = 0.f;
+    for (int k = lane; k < ns; k += 32) {
+        const float2 ml = p.part_ml[e0 + k];
+        l_all += (ml.x == -INFINITY) ? 0.f : ml.y * exp2f(ml.x - m_all);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xFFFFFFFFu, l_all, off);
+    // pass 2: each lane owns 4 output columns; 4 splits' loads are in flight together
+    const int D = p.head_dim;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     const int c4 = lane * 4;
-    for (int k = 0; k < sp.nsplit; ++k) {
-        const float2 ml = p.part_ml[e0 + k];
-        const float w = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m_all);
-        l_all += ml.y * w;
-        if (c4 < D) {
+    if (c4 < D) {
+        int k = 0;
+        for (; k + 4 <= ns; k += 4) {
+            float w[4];
+            float4 v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float mk = p.part_ml[e0 + k + j].x;
+                w[j] = (mk == -INFINITY) ? 0.f : exp2f(mk - m_all);
+                v[j] = *(const float4*)(p.part_o + (e0 + k + j) * D + c4);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { acc.x += v[j].x * w[j]; acc.y += v[j].y * w[j]; acc.z += v[j].z * w[j]; acc.w += v[j].w * w[j]; }
+        }
+        for (; k < ns; ++k) {
+            const float mk = p.part_ml[e0 + k].x;
+            const float w = (mk == -INFINITY) ? 0.f : exp2f(mk - m_all);
             const float4 v = *(const float4*)(p.part_o + (e0 + k) * D + c4);
             acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
         }
@@ -453,18 +514,18 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
 // --------------------------------------------------------------------------------------------
 namespace {
 template <int MT, int NS>
-cudaError_t launch_small(const AttnParams& p, cudaStream_t stream) {
-    constexpr int kQBytes = MT * 16 * kRowBytes;
+cudaError_t launch_small(const AttnParams& p, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
     constexpr int kMergeBytes = MT * kKW * 16 * (kMergeStride * 4 + 8);
     constexpr int kRing = NS * kStageBytes;
-    constexpr int kSmem = kQBytes + (kRing > kMergeBytes ? kRing : kMergeBytes);
+    // [ring | merge region][Q tile][2 * NS barriers + abort flag] + slack for the 1024-byte alignment
+    constexpr int kSmem = (kRing > kMergeBytes ? kRing : kMergeBytes) + MT * 16 * kRowBytes + 2 * NS * 8 + 16 + 1024;
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(attn_small_bf16_kernel<MT, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    attn_small_bf16_kernel<MT, NS><<<p.num_items, 128 * MT, kSmem, stream>>>(p);
+    attn_small_bf16_kernel<MT, NS><<<p.num_items, 128 * MT, kSmem, stream>>>(p, map_k, map_v);
     return cudaGetLastError();
 }
 }  // namespace
@@ -473,10 +534,14 @@ int attn_small_bf16_kv_tile() { return kStageTokens; }
 
 cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, cudaStream_t stream) {
     if (p.num_items == 0) return cudaSuccess;
+    if ((long long)p.num_pages * p.hkv * kPage > 0x7FFFFFFFll) return cudaErrorInvalidValue;
+    alignas(64) CUtensorMap map_k, map_v;
+    if (!make_pool_map(&map_k, p.k_pool, p.num_pages, p.hkv) || !make_pool_map(&map_v, p.v_pool, p.num_pages, p.hkv))
+        return cudaErrorNotSupported;
     switch (mt) {
-        case 1: return launch_small<1, 3>(p, stream);
-        case 2: return launch_small<2, 3>(p, stream);
-        case 4: return launch_small<4, 5>(p, stream);
+        case 1: return launch_small<1, 3>(p, map_k, map_v, stream);
+        case 2: return launch_small<2, 3>(p, map_k, map_v, stream);
+        case 4: return launch_small<4, 5>(p, map_k, map_v, stream);
         default: return cudaErrorInvalidValue;
     }
 }
