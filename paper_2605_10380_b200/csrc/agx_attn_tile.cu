@@ -12,9 +12,14 @@
 //   warp 1      MMA issuer (one lane) and TMEM owner.  Order on the tensor pipe:
 //               S_A(0) S_B(0) | O_A+=P_A V(t)  S_A(t+1)  O_B+=P_B V(t)  S_B(t+1) | ...
 //               so the softmax of one tile overlaps the MMAs of the other.
-//   warps 4-7   softmax of tile A, warps 8-11 softmax of tile B: one thread per query row (TMEM lane),
-//               S read with tcgen05.ld, P written back over S as packed bf16 (A operand of the P V MMA
-//               comes from TMEM), O rescaled in TMEM only when the row maximum grew by more than 2^8.
+//   warps 4-7   softmax of tile A, warps 8-11 softmax of tile B: one thread per query row (TMEM lane).
+//               The whole 128-column score row is held in registers (the two softmax warpgroups take
+//               registers from warps 0-3 with setmaxnreg), so S is read from TMEM once: row maximum,
+//               exponentials with packed f32x2 arithmetic, P written back over S as packed bf16 (the A
+//               operand of the P V MMA comes from TMEM), O rescaled in TMEM only when the row maximum
+//               grew by more than 2^8.
+// The Q tiles arrive by cp.async from warps 2-11 while warp 0 already streams K/V; results leave through
+// a per-warp shared-memory staging area so that global stores are whole rows.
 // TMEM columns: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512).
 // Every mbarrier wait is bounded: on time-out the CTA records AGX_DEV_WAIT_TIMEOUT and tears down.
 #include <cuda.h>
@@ -43,7 +48,9 @@ constexpr float kRescaleThreshold = 8.0f;              // log2 units
 
 // barrier slots (8 bytes each)
 enum { BAR_K_FULL = 0, BAR_K_EMPTY = 2, BAR_V_FULL = 4, BAR_V_EMPTY = 6, BAR_S_FULL = 8, BAR_P_READY = 10,
-       BAR_O_FULL = 12, BAR_COUNT = 13 };
+       BAR_O_FULL = 12, BAR_Q_FULL = 13, BAR_COUNT = 14 };
+constexpr int kQLoadThreads = kThreads - 64;  // warps 2..11 bring the Q tiles in
+constexpr int kRegsLow = 72, kRegsHigh = 208; // 128 * 72 + 256 * 208 <= 384 * 168
 
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;  // + 128 * tile
@@ -75,21 +82,42 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 
-__device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t* r) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr));
 }
-__device__ __forceinline__ void tmem_ld_x64(uint32_t taddr, uint32_t (&r)[64]) {
+__device__ __forceinline__ void tmem_ld_x64(uint32_t taddr, uint32_t* r) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];\n"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
                  : "r"(taddr));
 }
-__device__ __forceinline__ void tmem_st_x32(uint32_t taddr, const uint32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_st_x32(uint32_t taddr, const uint32_t* r) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n"
                  :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]));
 }
 
+
+// (d0, d1) = (a0, a1) * b + c, one packed instruction
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b, float c) {
+    asm("{\n.reg .b64 ra, rb, rc, rd;\nmov.b64 ra, {%2, %3};\nmov.b64 rb, {%4, %4};\nmov.b64 rc, {%5, %5};\n"
+        "fma.rn.f32x2 rd, ra, rb, rc;\nmov.b64 {%0, %1}, rd;\n}\n"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b), "f"(c));
+}
+// (d0, d1) += (a0, a1)
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
+    asm("{\n.reg .b64 ra, rd;\nmov.b64 ra, {%2, %3};\nmov.b64 rd, {%0, %1};\n"
+        "add.rn.f32x2 rd, rd, ra;\nmov.b64 {%0, %1}, rd;\n}\n"
+        : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
 
 __device__ __forceinline__ int find_seq(const AttnParams& p, int item) {
     int s = 0;
@@ -144,7 +172,8 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
 
     // ---- setup: barriers, TMEM, Q tiles
     if (tid == 0) {
-        for (int i = 0; i < BAR_COUNT; ++i) mbar_init(bar(i), (i == BAR_P_READY || i == BAR_P_READY + 1) ? 128u : 1u);
+        for (int i = 0; i < BAR_COUNT; ++i)
+            mbar_init(bar(i), (i == BAR_P_READY || i == BAR_P_READY + 1) ? 128u : (i == BAR_Q_FULL) ? (uint32_t)kQLoadThreads : 1u);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&map_k) : "memory");
@@ -154,26 +183,34 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
-    // Q: 256 rows x 256 B, plain 16-byte loads, written in the 128-byte-swizzled K-major operand layout
-    for (int c = tid; c < kRowsPerCta * 16; c += kThreads) {
-        const int rl = c >> 4, ch = c & 15;     // row in chunk, 16-byte chunk of the 256-byte row
-        const int r = row0 + rl;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (r < rows) {
-            const int i = r / G, hg = r - i * G;
-            v = __ldg((const uint4*)((const unsigned char*)p.q + (((long long)(sp.q_row0 + i) * p.hq + g * G + hg) * 256 + ch * 16)));
+    // Q: 256 rows x 256 B by 16-byte cp.async (all of a thread's copies in flight at once), written in
+    // the 128-byte-swizzled K-major operand layout; rows past q * G are zero-filled.
+    if (warp >= 2) {
+        for (int c = tid - 64; c < kRowsPerCta * 16; c += kQLoadThreads) {
+            const int rl = c >> 4, ch = c & 15;     // row in chunk, 16-byte chunk of the 256-byte row
+            const int r = row0 + rl;
+            const bool valid = r < rows;
+            const int rr = valid ? r : 0;
+            const int i = rr / G, hg = rr - i * G;
+            const unsigned char* src = (const unsigned char*)p.q + (((long long)(sp.q_row0 + i) * p.hq + g * G + hg) * 256 + ch * 16);
+            const int tile = rl >> 7, rt = rl & 127, half = ch >> 3, u = ch & 7;
+            cp_async_16(smem_base + kOffQ + tile * kTileBytes + half * kHalfBytes + rt * 128 + ((u ^ (rt & 7)) << 4), src, valid ? 16u : 0u);
         }
-        const int tile = rl >> 7, rt = rl & 127, half = ch >> 3, u = ch & 7;
-        *(uint4*)(smem + kOffQ + tile * kTileBytes + half * kHalfBytes + rt * 128 + ((u ^ (rt & 7)) << 4)) = v;
     }
-    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
     tc_fence_before();
-    __syncthreads();
+    __syncthreads();   // barriers initialised, TMEM address published
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-
+    if (warp >= 2) {
+        asm volatile("cp.async.wait_all;\n" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+        mbar_arrive(bar(BAR_Q_FULL));
+    }
     auto pages_in_tile = [&](int t) { return min(8, (kv_end - (kv_begin + t * kBN) + kPage - 1) / kPage); };
 
+    // the softmax warpgroups keep a whole score row in registers: warps 0-3 hand registers over to them
+    if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsLow));
     if (warp == 0) {
         // ================= TMA producer (whole warp stays converged; lane 0 issues) =================
         const int* pt_row = p.page_table + (long long)sp.seq_index * p.pt_stride;
@@ -262,7 +299,8 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                 for (int ks = 0; ks < npg; ++ks)
                     umma_ts(tO[x], tS[x] + ks * 8, make_desc(v_addr + ks * 2048, kHalfBytes, 1024), kIdescPV, !(first && ks == 0));
             };
-            bool ok = mbar_wait(bar(BAR_K_FULL + 0), 0, abort_flag, p.status);
+            bool ok = mbar_wait(bar(BAR_Q_FULL), 0, abort_flag, p.status);
+            if (ok) ok = mbar_wait(bar(BAR_K_FULL + 0), 0, abort_flag, p.status);
             if (ok) {
                 tc_fence_after();
                 issue_qk(0, 0); umma_commit(bar(BAR_S_FULL + 0));
@@ -299,7 +337,9 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
         }
         __syncwarp();
-    } else if (warp >= 4) {
+    }
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsHigh));
         // ================= softmax + epilogue: one thread per query row =================
         const int x = (warp - 4) >> 2;                       // tile A / B
         const int rt = ((warp & 3) << 5) + lane;             // row in tile == TMEM lane
@@ -309,31 +349,35 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         const int r = row0 + x * 128 + rt;
         const int limit = P + min(r / G, q - 1);             // last token this row sees
         const int tile_i_min = min((row0 + x * 128) / G, q - 1);
-        float m_ref = -INFINITY, l_sum = 0.f;
+        const float sc = p.scale_log2;
+        float m_ref = -INFINITY;
+        float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;        // four partial row sums (two packed pairs)
         bool ok = true;
         for (int t = 0; t < n_tiles; ++t) {
             ok = mbar_wait(bar(BAR_S_FULL + x), t & 1, abort_flag, p.status);
             if (!ok) break;
             tc_fence_after();
+            uint32_t sreg[128];
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) tmem_ld_x32(tS + c4 * 32, sreg + c4 * 32);
+            tmem_wait_ld();
             const int tok0 = kv_begin + t * kBN;
             const bool masked = (tok0 + kBN - 1 > P + tile_i_min) || (tok0 + kBN > kv_end);  // uniform per tile
-            const int nvis = max(0, min(min(limit + 1, kv_end) - tok0, kBN));            // visible columns: [0, nvis)
-            uint32_t sreg[64];
-            // ---- pass 1: row maximum
-            float mx = -INFINITY;
+            if (masked) {
+                const int nvis = max(0, min(min(limit + 1, kv_end) - tok0, kBN));            // visible columns: [0, nvis)
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                tmem_ld_x64(tS + hf * 64, sreg);
-                tmem_wait_ld();
-                if (masked) {
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) mx = fmaxf(mx, (hf * 64 + c < nvis) ? __uint_as_float(sreg[c]) : -INFINITY);
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sreg[c]));
-                }
+                for (int c = 0; c < 128; ++c)
+                    if (c >= nvis) sreg[c] = 0xFF800000u;  // -inf: its exponential is exactly 0
             }
-            const float m_tile = mx * p.scale_log2;
+            // ---- row maximum (four independent chains of 3-input max)
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int c = 0; c < 128; c += 8) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    mx[k] = max3(mx[k], __uint_as_float(sreg[c + 2 * k]), __uint_as_float(sreg[c + 2 * k + 1]));
+            }
+            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;
             const bool need = m_tile > m_ref + kRescaleThreshold;
             if (__any_sync(0xFFFFFFFFu, need)) {
                 const float m_new = need ? m_tile : m_ref;
@@ -350,74 +394,99 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                     }
                     tmem_wait_st();
                 }
-                l_sum *= factor;
+                l0 *= factor; l1 *= factor; l2 *= factor; l3 *= factor;
                 m_ref = m_new;
             }
-            const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-            // ---- pass 2: P = 2^(S * scale - m), packed bf16 pairs written over S
+            const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+            // ---- P = 2^(S * scale - m) as packed bf16 pairs, in place: sreg[c / 2] <- (p[c], p[c + 1])
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                tmem_ld_x64(tS + hf * 64, sreg);
-                tmem_wait_ld();
-                uint32_t preg[32];
-#pragma unroll
-                for (int c = 0; c < 64; c += 2) {
-                    float p0 = ex2(fmaf(__uint_as_float(sreg[c]), p.scale_log2, -m_use));
-                    float p1 = ex2(fmaf(__uint_as_float(sreg[c + 1]), p.scale_log2, -m_use));
-                    if (masked) {
-                        if (hf * 64 + c >= nvis) p0 = 0.f;
-                        if (hf * 64 + c + 1 >= nvis) p1 = 0.f;
-                    }
-                    l_sum += p0 + p1;
-                    preg[c >> 1] = pack_bf16(p0, p1);
-                }
-                tmem_st_x32(tS + hf * 32, preg);
+            for (int c = 0; c < 128; c += 4) {
+                float a0, a1, b0, b1;
+                fma2(a0, a1, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]), sc, neg_m);
+                fma2(b0, b1, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]), sc, neg_m);
+                a0 = ex2(a0); a1 = ex2(a1); b0 = ex2(b0); b1 = ex2(b1);
+                add2(l0, l1, a0, a1);
+                add2(l2, l3, b0, b1);
+                sreg[c >> 1] = pack_bf16(a0, a1);
+                sreg[(c >> 1) + 1] = pack_bf16(b0, b1);
             }
+            tmem_st_x32(tS, sreg);
+            tmem_st_x32(tS + 32, sreg + 32);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(BAR_P_READY + x));
         }
-        // ---- epilogue
+        // ---- epilogue: O rows go through this warp's 16 KB of the (now idle) K/V rings, so that the
+        //      global stores are whole rows
         if (ok) ok = mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
         if (ok) {
             tc_fence_after();
+            const float l_sum = (l0 + l1) + (l2 + l3);
             const bool valid = r < rows;
             const int i = r / G, h = g * G + (r - (r / G) * G);
-            const float inv = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
+            unsigned char* stage = smem + kOffK + (warp - 4) * 16384;
+            const int r_warp0 = row0 + x * 128 + ((warp & 3) << 5);   // first row of this warp
             uint32_t oreg[32];
             if (sp.nsplit == 1) {
-                __nv_bfloat16* dst = (__nv_bfloat16*)p.out + ((long long)(sp.q_row0 + i) * p.hq + h) * kD;
+                const float inv = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
 #pragma unroll
                 for (int c4 = 0; c4 < 4; ++c4) {
                     tmem_ld_x32(tO + c4 * 32, oreg);
                     tmem_wait_ld();
-                    if (valid) {
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) {
-                            uint4 pk;
-                            pk.x = pack_bf16(__uint_as_float(oreg[8 * v + 0]) * inv, __uint_as_float(oreg[8 * v + 1]) * inv);
-                            pk.y = pack_bf16(__uint_as_float(oreg[8 * v + 2]) * inv, __uint_as_float(oreg[8 * v + 3]) * inv);
-                            pk.z = pack_bf16(__uint_as_float(oreg[8 * v + 4]) * inv, __uint_as_float(oreg[8 * v + 5]) * inv);
-                            pk.w = pack_bf16(__uint_as_float(oreg[8 * v + 6]) * inv, __uint_as_float(oreg[8 * v + 7]) * inv);
-                            *(uint4*)(dst + c4 * 32 + v * 8) = pk;
-                        }
+                    for (int v = 0; v < 4; ++v) {
+                        uint4 pk;
+                        pk.x = pack_bf16(__uint_as_float(oreg[8 * v + 0]) * inv, __uint_as_float(oreg[8 * v + 1]) * inv);
+                        pk.y = pack_bf16(__uint_as_float(oreg[8 * v + 2]) * inv, __uint_as_float(oreg[8 * v + 3]) * inv);
+                        pk.z = pack_bf16(__uint_as_float(oreg[8 * v + 4]) * inv, __uint_as_float(oreg[8 * v + 5]) * inv);
+                        pk.w = pack_bf16(__uint_as_float(oreg[8 * v + 6]) * inv, __uint_as_float(oreg[8 * v + 7]) * inv);
+                        *(uint4*)(stage + lane * 256 + (((c4 * 4 + v) ^ (lane & 7)) << 4)) = pk;
                     }
                 }
                 if (valid && p.lse) p.lse[(long long)(sp.q_row0 + i) * p.hq + h] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
-            } else {
-                const long long e = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit + split;
-                float* dst = p.part_o + e * kD;
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    tmem_ld_x32(tO + c4 * 32, oreg);
-                    tmem_wait_ld();
-                    if (valid) {
-#pragma unroll
-                        for (int v = 0; v < 8; ++v)
-                            *(uint4*)(dst + c4 * 32 + v * 4) = make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
+                __syncwarp();
+                // two rows per trip: a half-warp writes one 256-byte row
+                const int sub = lane >> 4, ch = lane & 15;
+#pragma unroll 4
+                for (int rr = 0; rr < 32; rr += 2) {
+                    const int rl = rr + sub, ro = r_warp0 + rl;
+                    if (ro < rows) {
+                        const int io = ro / G, ho = g * G + (ro - io * G);
+                        const uint4 v = *(const uint4*)(stage + rl * 256 + ((ch ^ (rl & 7)) << 4));
+                        *(uint4*)((unsigned char*)p.out + (((long long)(sp.q_row0 + io) * p.hq + ho) * 256 + ch * 16)) = v;
                     }
                 }
-                if (valid) p.part_ml[e] = make_float2(m_ref, l_sum);
+            } else {
+                // fp32 partials: 512 bytes per row, staged in two passes of 64 columns (16 KB per warp)
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+                    for (int c4 = 0; c4 < 2; ++c4) {
+                        tmem_ld_x32(tO + hf * 64 + c4 * 32, oreg);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            *(uint4*)(stage + lane * 256 + (((c4 * 8 + v) ^ (lane & 7)) << 4)) =
+                                make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
+                    }
+                    __syncwarp();
+                    const int sub = lane >> 4, ch = lane & 15;
+#pragma unroll 4
+                    for (int rr = 0; rr < 32; rr += 2) {
+                        const int rl = rr + sub, ro = r_warp0 + rl;
+                        if (ro < rows) {
+                            const int io = ro / G, ho = g * G + (ro - io * G);
+                            const long long e = (long long)sp.part_base + ((long long)io * p.hq + ho) * sp.nsplit + split;
+                            const uint4 v = *(const uint4*)(stage + rl * 256 + ((ch ^ (rl & 7)) << 4));
+                            *(uint4*)((unsigned char*)(p.part_o + e * kD) + hf * 256 + ch * 16) = v;
+                        }
+                    }
+                    __syncwarp();
+                }
+                if (valid) {
+                    const long long e = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit + split;
+                    p.part_ml[e] = make_float2(m_ref, l_sum);
+                }
             }
         }
     }

@@ -97,6 +97,29 @@ def test_c1_accept_fp32_first_two_of_three_match():
     assert got[1][0] == 2 and got[2][0] == am[2] and got[3][0] == 259
 
 
+def test_c4_ragged_mixed_batch_shared_prefix():
+    """16 sequences, lognormal prefixes, verify blocks and suffix prefills in one call, first 2048
+    tokens' pages shared by all: every sequence's first and last block row plus seeded samples."""
+    w = W.c4_ragged_mixed()
+    assert np.all(w.page_table[:, :128] == w.page_table[0, :128])
+    b, _ = run_and_check(w, sample=(4, 24), strict=True)
+    assert b.launches >= 3  # split-KV kernel(s), tile kernel, combine
+
+
+def test_c5_long_context_verify_and_prefill():
+    """4 x (P = 32768, q = 8) plus 1 x (P = 30720, q = 2048) in one call, sampled rows against the
+    oracle; then the accept step on bf16 logits [4 x 8, 128256]."""
+    w = W.c5_long_context()
+    b, _ = run_and_check(w, sample=(6, 24), strict=True)
+    h = agx.Handle(32, 8, 128, "bf16")
+    aw = W.make_planted_accept("c5_accept", 55, "bf16", 128256, [8] * 4, [32768] * 4)
+    ref = oracle.accept_greedy(aw.logits, "bf16", aw.vocab, aw.drafts, aw.cu_q, aw.prefix_len)
+    got = run_accept(h, aw)
+    for g, r in zip(got, ref):
+        assert np.array_equal(g, r)
+    assert np.array_equal(got[1], aw.planned_accept)
+
+
 # ------------------------------------------------------------------ small-q kernel: shapes and edges
 @pytest.mark.parametrize("P,q,hq,hkv", [
     (0, 1, 32, 8), (1, 1, 32, 8), (15, 1, 8, 8), (16, 2, 32, 8), (17, 4, 32, 8), (63, 8, 32, 8), (64, 8, 32, 8),
