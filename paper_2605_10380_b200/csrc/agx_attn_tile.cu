@@ -35,22 +35,23 @@ namespace {
 constexpr int kD = 128;
 constexpr int kBN = 128;                    // KV tokens per tile
 constexpr int kRowsPerCta = 256;
-constexpr int kStages = 2;
+constexpr int kStagesK = 3;                 // K is wanted right after the previous tile's softmax: one more stage
+constexpr int kStagesV = 2;
 constexpr int kThreads = 384;
 constexpr uint32_t kTileBytes = 128 * 256;  // one operand tile: [2 halves of 64 dims][128 rows][128 B]
 constexpr uint32_t kHalfBytes = 128 * 128;
 constexpr uint32_t kOffQ = 0;
 constexpr uint32_t kOffK = 2 * kTileBytes;
-constexpr uint32_t kOffV = kOffK + kStages * kTileBytes;
-constexpr uint32_t kOffBar = kOffV + kStages * kTileBytes;
+constexpr uint32_t kOffV = kOffK + kStagesK * kTileBytes;
+constexpr uint32_t kOffBar = kOffV + kStagesV * kTileBytes;
 constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // + barriers + alignment slack
 constexpr float kRescaleThreshold = 8.0f;              // log2 units
 
 // barrier slots (8 bytes each)
-enum { BAR_K_FULL = 0, BAR_K_EMPTY = 2, BAR_V_FULL = 4, BAR_V_EMPTY = 6, BAR_S_FULL = 8, BAR_P_READY = 10,
-       BAR_O_FULL = 12, BAR_Q_FULL = 13, BAR_COUNT = 14 };
+enum { BAR_K_FULL = 0, BAR_K_EMPTY = 3, BAR_V_FULL = 6, BAR_V_EMPTY = 8, BAR_S_FULL = 10, BAR_P_READY = 12,
+       BAR_O_FULL = 14, BAR_Q_FULL = 15, BAR_COUNT = 16 };
 constexpr int kQLoadThreads = kThreads - 64;  // warps 2..11 bring the Q tiles in
-constexpr int kRegsLow = 72, kRegsHigh = 208; // 128 * 72 + 256 * 208 <= 384 * 168
+constexpr int kRegsLow = 96, kRegsHigh = 200; // 128 * 96 + 256 * 200 <= 384 * 168
 
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;  // + 128 * tile
@@ -212,7 +213,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
     if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsLow));
     if (warp == 0) {
-        // ================= TMA producer (whole warp stays converged; lane 0 issues) =================
+        // ================= TMA producer: lane l of the warp copies page l of the tile =================
         const int* pt_row = p.page_table + (long long)sp.seq_index * p.pt_stride;
         const int page0 = kv_begin / kPage;
         const int n_pages_total = (kv_end - kv_begin + kPage - 1) / kPage;
@@ -228,25 +229,26 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                 }
                 ids = (int)id;
             }
-            const int stage = t & 1, ph = (t >> 1) & 1;
+            const int ks = t % kStagesK, kph = (t / kStagesK) & 1;
+            const int vs = t % kStagesV, vph = (t / kStagesV) & 1;
             const int npg = pages_in_tile(t);
             const int tok0 = kv_begin + t * kBN;
+            const int pg = lane - (t & 3) * 8;              // this lane's page of the tile
+            const bool mine = pg >= 0 && pg < npg;
+            const int y = (ids * p.hkv + g) * kPage;
             // ---- K
-            ok = mbar_wait(bar(BAR_K_EMPTY + stage), ph ^ 1, abort_flag, p.status);
+            ok = mbar_wait(bar(BAR_K_EMPTY + ks), kph ^ 1, abort_flag, p.status);
             if (!ok) break;
-            if (lane == 0) mbar_arrive_expect_tx(bar(BAR_K_FULL + stage), npg * 4096u);
-            for (int pg = 0; pg < npg; ++pg) {
-                const int id = __shfl_sync(0xFFFFFFFFu, ids, (t & 3) * 8 + pg);
-                if (lane == 0) {
-                    const int y = (id * p.hkv + g) * kPage;
-                    const uint32_t dst = smem_base + kOffK + stage * kTileBytes + pg * 2048;
-                    tma_load_2d(dst, &map_k, 0, y, bar(BAR_K_FULL + stage));
-                    tma_load_2d(dst + kHalfBytes, &map_k, 64, y, bar(BAR_K_FULL + stage));
-                }
+            if (lane == 0) mbar_arrive_expect_tx(bar(BAR_K_FULL + ks), npg * 4096u);
+            __syncwarp();
+            if (mine) {
+                const uint32_t dst = smem_base + kOffK + ks * kTileBytes + pg * 2048;
+                tma_load_2d(dst, &map_k, 0, y, bar(BAR_K_FULL + ks));
+                tma_load_2d(dst + kHalfBytes, &map_k, 64, y, bar(BAR_K_FULL + ks));
             }
             // ---- V (the page that holds token L, if L is not page-aligned, is copied by hand so that
             //      slots past the end of the sequence are zeros whatever the pool holds there)
-            ok = mbar_wait(bar(BAR_V_EMPTY + stage), ph ^ 1, abort_flag, p.status);
+            ok = mbar_wait(bar(BAR_V_EMPTY + vs), vph ^ 1, abort_flag, p.status);
             if (!ok) break;
             const int ragged_pg = ((L & 15) != 0 && (L >> 4) >= (tok0 >> 4) && (L >> 4) < (tok0 >> 4) + npg) ? (L >> 4) - (tok0 >> 4) : -1;
             if (ragged_pg >= 0) {
@@ -257,47 +259,53 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                     const int r = idx >> 4, ch = idx & 15, half = ch >> 3, u = ch & 7;
                     uint4 v = make_uint4(0, 0, 0, 0);
                     if (r < valid_rows) v = __ldg((const uint4*)(src + r * 256 + ch * 16));
-                    *(uint4*)(smem + kOffV + stage * kTileBytes + half * kHalfBytes + ragged_pg * 2048 + r * 128 + ((u ^ (r & 7)) << 4)) = v;
+                    *(uint4*)(smem + kOffV + vs * kTileBytes + half * kHalfBytes + ragged_pg * 2048 + r * 128 + ((u ^ (r & 7)) << 4)) = v;
                 }
                 asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                 __syncwarp();
             }
-            if (lane == 0) mbar_arrive_expect_tx(bar(BAR_V_FULL + stage), (npg - (ragged_pg >= 0 ? 1 : 0)) * 4096u);
-            for (int pg = 0; pg < npg; ++pg) {
-                const int id = __shfl_sync(0xFFFFFFFFu, ids, (t & 3) * 8 + pg);
-                if (lane == 0 && pg != ragged_pg) {
-                    const int y = (id * p.hkv + g) * kPage;
-                    const uint32_t dst = smem_base + kOffV + stage * kTileBytes + pg * 2048;
-                    tma_load_2d(dst, &map_v, 0, y, bar(BAR_V_FULL + stage));
-                    tma_load_2d(dst + kHalfBytes, &map_v, 64, y, bar(BAR_V_FULL + stage));
-                }
+            if (lane == 0) mbar_arrive_expect_tx(bar(BAR_V_FULL + vs), (npg - (ragged_pg >= 0 ? 1 : 0)) * 4096u);
+            __syncwarp();
+            if (mine && pg != ragged_pg) {
+                const uint32_t dst = smem_base + kOffV + vs * kTileBytes + pg * 2048;
+                tma_load_2d(dst, &map_v, 0, y, bar(BAR_V_FULL + vs));
+                tma_load_2d(dst + kHalfBytes, &map_v, 64, y, bar(BAR_V_FULL + vs));
             }
         }
         // drain: the copies this warp started must land before the CTA's shared memory goes away
         if (lane == 0) {
-            for (int t = max(0, n_tiles - kStages); t < n_tiles; ++t) {
-                mbar_wait(bar(BAR_K_FULL + (t & 1)), (t >> 1) & 1, abort_flag, p.status);
-                mbar_wait(bar(BAR_V_FULL + (t & 1)), (t >> 1) & 1, abort_flag, p.status);
-            }
+            for (int t = max(0, n_tiles - kStagesK); t < n_tiles; ++t)
+                mbar_wait(bar(BAR_K_FULL + t % kStagesK), (t / kStagesK) & 1, abort_flag, p.status);
+            for (int t = max(0, n_tiles - kStagesV); t < n_tiles; ++t)
+                mbar_wait(bar(BAR_V_FULL + t % kStagesV), (t / kStagesV) & 1, abort_flag, p.status);
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            const uint32_t q_addr[2] = {smem_base + kOffQ, smem_base + kOffQ + kTileBytes};
             const uint32_t tS[2] = {tmem_base + kColS, tmem_base + kColS + 128};
             const uint32_t tO[2] = {tmem_base + kColO, tmem_base + kColO + 128};
+            // descriptors differ only in the start address: add (byte offset >> 4) to a base descriptor
+            const uint64_t q_desc[2] = {make_desc(smem_base + kOffQ, 16, 1024), make_desc(smem_base + kOffQ + kTileBytes, 16, 1024)};
+            const uint64_t k_desc0 = make_desc(smem_base + kOffK, 16, 1024);
+            const uint64_t v_desc0 = make_desc(smem_base + kOffV, kHalfBytes, 1024);
             auto issue_qk = [&](int x, int stage) {   // S_x = Q_x K^T : 8 k-steps of 16 dims
-                const uint32_t k_addr = smem_base + kOffK + stage * kTileBytes;
+                const uint64_t kd = k_desc0 + (uint64_t)((stage * kTileBytes) >> 4);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                    umma_ss(tS[x], make_desc(q_addr[x] + off, 16, 1024), make_desc(k_addr + off, 16, 1024), kIdescQK, ks > 0);
+                    const uint64_t off = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+                    umma_ss(tS[x], q_desc[x] + off, kd + off, kIdescQK, ks > 0);
                 }
             };
             auto issue_pv = [&](int x, int stage, int npg, bool first) {  // O_x += P_x V : one k-step per page
-                const uint32_t v_addr = smem_base + kOffV + stage * kTileBytes;
-                for (int ks = 0; ks < npg; ++ks)
-                    umma_ts(tO[x], tS[x] + ks * 8, make_desc(v_addr + ks * 2048, kHalfBytes, 1024), kIdescPV, !(first && ks == 0));
+                const uint64_t vd = v_desc0 + (uint64_t)((stage * kTileBytes) >> 4);
+                if (npg == 8) {
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        umma_ts(tO[x], tS[x] + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescPV, !(first && ks == 0));
+                } else {
+                    for (int ks = 0; ks < npg; ++ks)
+                        umma_ts(tO[x], tS[x] + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescPV, !(first && ks == 0));
+                }
             };
             bool ok = mbar_wait(bar(BAR_Q_FULL), 0, abort_flag, p.status);
             if (ok) ok = mbar_wait(bar(BAR_K_FULL + 0), 0, abort_flag, p.status);
@@ -308,29 +316,29 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                 umma_commit(bar(BAR_K_EMPTY + 0));
             }
             for (int t = 0; t < n_tiles && ok; ++t) {
-                const int stage = t & 1, ph = (t >> 1) & 1, npg = pages_in_tile(t);
+                const int vs = t % kStagesV, vph = (t / kStagesV) & 1, npg = pages_in_tile(t);
                 const bool more = t + 1 < n_tiles;
-                const int nstage = (t + 1) & 1, nph = ((t + 1) >> 1) & 1;
-                ok = mbar_wait(bar(BAR_V_FULL + stage), ph, abort_flag, p.status);
+                const int nks = (t + 1) % kStagesK, nkph = ((t + 1) / kStagesK) & 1;
+                ok = mbar_wait(bar(BAR_V_FULL + vs), vph, abort_flag, p.status);
                 if (!ok) break;
                 ok = mbar_wait(bar(BAR_P_READY + 0), t & 1, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
-                issue_pv(0, stage, npg, t == 0);
+                issue_pv(0, vs, npg, t == 0);
                 if (more) {
-                    ok = mbar_wait(bar(BAR_K_FULL + nstage), nph, abort_flag, p.status);
+                    ok = mbar_wait(bar(BAR_K_FULL + nks), nkph, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_qk(0, nstage); umma_commit(bar(BAR_S_FULL + 0));
+                    issue_qk(0, nks); umma_commit(bar(BAR_S_FULL + 0));
                 }
                 ok = mbar_wait(bar(BAR_P_READY + 1), t & 1, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
-                issue_pv(1, stage, npg, t == 0);
-                umma_commit(bar(BAR_V_EMPTY + stage));
+                issue_pv(1, vs, npg, t == 0);
+                umma_commit(bar(BAR_V_EMPTY + vs));
                 if (more) {
-                    issue_qk(1, nstage); umma_commit(bar(BAR_S_FULL + 1));
-                    umma_commit(bar(BAR_K_EMPTY + nstage));
+                    issue_qk(1, nks); umma_commit(bar(BAR_S_FULL + 1));
+                    umma_commit(bar(BAR_K_EMPTY + nks));
                 }
             }
             umma_commit(bar(BAR_O_FULL));  // arrives when every MMA issued above has completed
