@@ -29,7 +29,6 @@
 #include "agx_sm100.cuh"
 
 namespace agx {
-
 namespace {
 
 constexpr int kD = 128;
@@ -46,6 +45,10 @@ constexpr uint32_t kOffV = kOffK + kStagesK * kTileBytes;
 constexpr uint32_t kOffBar = kOffV + kStagesV * kTileBytes;
 constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // + barriers + alignment slack
 constexpr float kRescaleThreshold = 8.0f;              // log2 units
+#ifndef AGX_POLY_PAIRS
+#define AGX_POLY_PAIRS 3
+#endif
+constexpr int kPolyPairsOf8 = AGX_POLY_PAIRS;          // of every 8 column pairs, this many take the polynomial 2^x
 
 // barrier slots (8 bytes each)
 enum { BAR_K_FULL = 0, BAR_K_EMPTY = 3, BAR_V_FULL = 6, BAR_V_EMPTY = 8, BAR_S_FULL = 10, BAR_P_READY = 12,
@@ -99,22 +102,70 @@ __device__ __forceinline__ void tmem_st_x32(uint32_t taddr, const uint32_t* r) {
 }
 
 
-// (d0, d1) = (a0, a1) * b + c, one packed instruction
-__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b, float c) {
-    asm("{\n.reg .b64 ra, rb, rc, rd;\nmov.b64 ra, {%2, %3};\nmov.b64 rb, {%4, %4};\nmov.b64 rc, {%5, %5};\n"
-        "fma.rn.f32x2 rd, ra, rb, rc;\nmov.b64 {%0, %1}, rd;\n}\n"
-        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b), "f"(c));
+// Packed pairs of floats in one 64-bit register, for the f32x2 arithmetic instructions.
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};\n" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
 }
-// (d0, d1) += (a0, a1)
+__device__ __forceinline__ void upk2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;\n" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2p(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2p(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;\n" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// 2^x for a packed pair on the FMA pipes instead of the special-function unit: n = round(x) by the
+// 1.5 * 2^23 trick, f = x - n in [-0.5, 0.5], 2^f by a cubic fitted to minimise the maximum relative
+// error on that interval (7.5e-5, far below the 2^-9 rounding of P to bfloat16), then n is added
+// into the exponent field.  x is clamped at -126 so the exponent cannot wrap.
+__device__ __forceinline__ void ex2_poly2(uint64_t x, float& p0, float& p1) {
+    float x0, x1;
+    upk2(x, x0, x1);
+    x = pk2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+    const uint64_t magic = pk2(12582912.f, 12582912.f), neg_magic = pk2(-12582912.f, -12582912.f);
+    const uint64_t t = add2p(x, magic);
+    const uint64_t n = add2p(t, neg_magic);
+    const uint64_t f = fma2p(n, pk2(-1.f, -1.f), x);
+    uint64_t q = fma2p(f, pk2(0.0551716648042202f, 0.0551716648042202f), pk2(0.2426111251115799f, 0.2426111251115799f));
+    q = fma2p(q, f, pk2(0.6932609677314758f, 0.6932609677314758f));
+    q = fma2p(q, f, pk2(0.9999280571937561f, 0.9999280571937561f));
+    float q0, q1, t0, t1;
+    upk2(q, q0, q1);
+    upk2(t, t0, t1);
+    p0 = __int_as_float(__float_as_int(t0) * 8388608 + __float_as_int(q0));
+    p1 = __int_as_float(__float_as_int(t1) * 8388608 + __float_as_int(q1));
+}
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b, float c) {
+    upk2(fma2p(pk2(a0, a1), pk2(b, b), pk2(c, c)), d0, d1);
+}
 __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
-    asm("{\n.reg .b64 ra, rd;\nmov.b64 ra, {%2, %3};\nmov.b64 rd, {%0, %1};\n"
-        "add.rn.f32x2 rd, rd, ra;\nmov.b64 {%0, %1}, rd;\n}\n"
-        : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
+    upk2(add2p(pk2(d0, d1), pk2(a0, a1)), d0, d1);
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;\n" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;\n" ::: "memory"); }
+// address of the same shared-memory location in the CTA of rank `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_u4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void st_cluster_f2(uint32_t addr, float a, float b) {
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};\n" ::"r"(addr), "f"(a), "f"(b) : "memory");
 }
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
@@ -159,17 +210,13 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
     const int kv_end = min(vis_end, kv_begin + sp.split_tokens);
     const int n_tiles = max(0, (kv_end - kv_begin + kBN - 1) / kBN);
 
-    if (n_tiles == 0) {  // nothing visible in this split: publish empty partials (nsplit > 1 by construction)
-        for (int idx = tid; idx < kRowsPerCta * (kD / 4); idx += kThreads) {
-            const int r = row0 + idx / (kD / 4), c4 = (idx % (kD / 4)) * 4;
-            if (r >= rows) continue;
-            const int i = r / G, h = g * G + (r - i * G);
-            const long long e = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit + split;
-            *(float4*)(p.part_o + e * kD + c4) = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (c4 == 0) p.part_ml[e] = make_float2(-INFINITY, 0.f);
-        }
+    if (n_tiles == 0) {  // nothing visible in this split: only keep the cluster's two barriers company
+        cluster_arrive(); cluster_wait();
+        cluster_arrive(); cluster_wait();
         return;
     }
+    // splits are in token order, so the active ones are ranks 0 .. n_active - 1
+    const int n_active = min(sp.nsplit, (vis_end + sp.split_tokens - 1) / sp.split_tokens);
 
     // ---- setup: barriers, TMEM, Q tiles
     if (tid == 0) {
@@ -346,6 +393,13 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         }
         __syncwarp();
     }
+    tc_fence_before();
+    cluster_arrive(); cluster_wait();       // every CTA of the cluster has left its main loop
+    cluster_arrive(); cluster_wait();       // every CTA has delivered its O rows: the softmax warps are done with TMEM
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsHigh));
         // ================= softmax + epilogue: one thread per query row =================
@@ -359,7 +413,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         const int tile_i_min = min((row0 + x * 128) / G, q - 1);
         const float sc = p.scale_log2;
         float m_ref = -INFINITY;
-        float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;        // four partial row sums (two packed pairs)
+        float l_run = 0.f;                                   // running row sum, relative to m_ref
         bool ok = true;
         for (int t = 0; t < n_tiles; ++t) {
             ok = mbar_wait(bar(BAR_S_FULL + x), t & 1, abort_flag, p.status);
@@ -371,139 +425,163 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             tmem_wait_ld();
             const int tok0 = kv_begin + t * kBN;
             const bool masked = (tok0 + kBN - 1 > P + tile_i_min) || (tok0 + kBN > kv_end);  // uniform per tile
-            if (masked) {
-                const int nvis = max(0, min(min(limit + 1, kv_end) - tok0, kBN));            // visible columns: [0, nvis)
+            const uint64_t sc2 = pk2(sc, sc);
+            float lt0 = 0.f, lt1 = 0.f, lt2 = 0.f, lt3 = 0.f;   // this tile's row sum, four partial sums
+            bool done = false;
+            if (t > 0 && !masked) {
+                // ---- common case, one sweep: exponentials against the running reference m_ref (the
+                //      maximum of earlier tiles, so P may exceed 1) while the tile's own maximum is
+                //      collected on the side; only if that maximum tops m_ref by more than 2^8 is the
+                //      tile redone below with a new reference.
+                const uint64_t nm2 = pk2(-m_ref, -m_ref);
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int c = 0; c < 128; ++c)
-                    if (c >= nvis) sreg[c] = 0xFF800000u;  // -inf: its exponential is exactly 0
-            }
-            // ---- row maximum (four independent chains of 3-input max)
-            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-            for (int c = 0; c < 128; c += 8) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    mx[k] = max3(mx[k], __uint_as_float(sreg[c + 2 * k]), __uint_as_float(sreg[c + 2 * k + 1]));
-            }
-            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;
-            const bool need = m_tile > m_ref + kRescaleThreshold;
-            if (__any_sync(0xFFFFFFFFu, need)) {
-                const float m_new = need ? m_tile : m_ref;
-                const float factor = need ? ex2(m_ref - m_new) : 1.f;   // m_ref = -inf gives 0
-                if (t > 0) {
-                    uint32_t oreg[32];
-#pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        tmem_ld_x32(tO + c4 * 32, oreg);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * factor);
-                        tmem_st_x32(tO + c4 * 32, oreg);
-                    }
-                    tmem_wait_st();
+                for (int c = 0; c < 128; c += 4) {   // in place: sreg[c / 2] <- (p[c], p[c + 1])
+                    const float s0 = __uint_as_float(sreg[c]), s1 = __uint_as_float(sreg[c + 1]);
+                    const float s2 = __uint_as_float(sreg[c + 2]), s3 = __uint_as_float(sreg[c + 3]);
+                    mx[(c >> 2) & 3] = max3(mx[(c >> 2) & 3], s0, s1);
+                    mx[((c >> 2) + 2) & 3] = max3(mx[((c >> 2) + 2) & 3], s2, s3);
+                    const uint64_t xa = fma2p(pk2(s0, s1), sc2, nm2), xb = fma2p(pk2(s2, s3), sc2, nm2);
+                    float a0, a1, b0, b1;
+                    if (((c >> 1) & 7) < kPolyPairsOf8) ex2_poly2(xa, a0, a1);
+                    else { upk2(xa, a0, a1); a0 = ex2(a0); a1 = ex2(a1); }
+                    if ((((c >> 1) + 1) & 7) < kPolyPairsOf8) ex2_poly2(xb, b0, b1);
+                    else { upk2(xb, b0, b1); b0 = ex2(b0); b1 = ex2(b1); }
+                    add2(lt0, lt1, a0, a1);
+                    add2(lt2, lt3, b0, b1);
+                    sreg[c >> 1] = pack_bf16(a0, a1);
+                    sreg[(c >> 1) + 1] = pack_bf16(b0, b1);
                 }
-                l0 *= factor; l1 *= factor; l2 *= factor; l3 *= factor;
-                m_ref = m_new;
-            }
-            const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-            // ---- P = 2^(S * scale - m) as packed bf16 pairs, in place: sreg[c / 2] <- (p[c], p[c + 1])
+                const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;
+                if (!__any_sync(0xFFFFFFFFu, m_tile > m_ref + kRescaleThreshold)) {
+                    done = true;
+                } else {   // rare: fetch the scores again (P has not been stored over them yet)
+                    lt0 = lt1 = lt2 = lt3 = 0.f;
 #pragma unroll
-            for (int c = 0; c < 128; c += 4) {
-                float a0, a1, b0, b1;
-                fma2(a0, a1, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]), sc, neg_m);
-                fma2(b0, b1, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]), sc, neg_m);
-                a0 = ex2(a0); a1 = ex2(a1); b0 = ex2(b0); b1 = ex2(b1);
-                add2(l0, l1, a0, a1);
-                add2(l2, l3, b0, b1);
-                sreg[c >> 1] = pack_bf16(a0, a1);
-                sreg[(c >> 1) + 1] = pack_bf16(b0, b1);
+                    for (int c4 = 0; c4 < 4; ++c4) tmem_ld_x32(tS + c4 * 32, sreg + c4 * 32);
+                    tmem_wait_ld();
+                }
             }
+            if (!done) {
+                if (masked) {
+                    const int nvis = max(0, min(min(limit + 1, kv_end) - tok0, kBN));        // visible columns: [0, nvis)
+#pragma unroll
+                    for (int c = 0; c < 128; ++c)
+                        if (c >= nvis) sreg[c] = 0xFF800000u;  // -inf: its exponential is exactly 0
+                }
+                // ---- row maximum (four independent chains of 3-input max)
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                for (int c = 0; c < 128; c += 8) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        mx[k] = max3(mx[k], __uint_as_float(sreg[c + 2 * k]), __uint_as_float(sreg[c + 2 * k + 1]));
+                }
+                const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;
+                const bool need = m_tile > m_ref + kRescaleThreshold;
+                if (__any_sync(0xFFFFFFFFu, need)) {
+                    const float m_new = need ? m_tile : m_ref;
+                    const float factor = need ? ex2(m_ref - m_new) : 1.f;   // m_ref = -inf gives 0
+                    if (t > 0) {
+                        uint32_t oreg[32];
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4) {
+                            tmem_ld_x32(tO + c4 * 32, oreg);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * factor);
+                            tmem_st_x32(tO + c4 * 32, oreg);
+                        }
+                        tmem_wait_st();
+                    }
+                    l_run *= factor;
+                    m_ref = m_new;
+                }
+                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+                // ---- P = 2^(S * scale - m) as packed bf16 pairs, in place: sreg[c / 2] <- (p[c], p[c + 1])
+#pragma unroll
+                for (int c = 0; c < 128; c += 4) {
+                    float a0, a1, b0, b1;
+                    fma2(a0, a1, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]), sc, neg_m);
+                    fma2(b0, b1, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]), sc, neg_m);
+                    a0 = ex2(a0); a1 = ex2(a1); b0 = ex2(b0); b1 = ex2(b1);
+                    add2(lt0, lt1, a0, a1);
+                    add2(lt2, lt3, b0, b1);
+                    sreg[c >> 1] = pack_bf16(a0, a1);
+                    sreg[(c >> 1) + 1] = pack_bf16(b0, b1);
+                }
+            }
+            l_run += (lt0 + lt1) + (lt2 + lt3);
             tmem_st_x32(tS, sreg);
             tmem_st_x32(tS + 32, sreg + 32);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(BAR_P_READY + x));
         }
-        // ---- epilogue: O rows go through this warp's 16 KB of the (now idle) K/V rings, so that the
-        //      global stores are whole rows
+        // ---- epilogue.  Every KV split of this (sequence, KV head, row chunk) is one CTA of the
+        //      cluster.  Row rl of the chunk is owned by the active CTA of rank rl % n_active.  Once
+        //      every CTA of the cluster has left its main loop (first cluster barrier: the K/V rings are
+        //      idle everywhere), each CTA sends its un-normalised fp32 O rows and (m, l) into the owners'
+        //      shared memory with remote stores; after the second barrier an owner merges the splits of
+        //      its rows in rank order from its own shared memory and writes whole bf16 rows.  No
+        //      partials in global memory, no second kernel, fixed order: bit-reproducible.
         if (ok) ok = mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
-        if (ok) {
-            tc_fence_after();
-            const float l_sum = (l0 + l1) + (l2 + l3);
-            const bool valid = r < rows;
-            const int i = r / G, h = g * G + (r - (r / G) * G);
-            unsigned char* stage = smem + kOffK + (warp - 4) * 16384;
-            const int r_warp0 = row0 + x * 128 + ((warp & 3) << 5);   // first row of this warp
-            uint32_t oreg[32];
-            if (sp.nsplit == 1) {
-                const float inv = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
+        tc_fence_before();
+        cluster_arrive(); cluster_wait();
+        {
+            const int rl_own = x * 128 + rt;
+            const int owner = rl_own % n_active;
+            const int slot = (rl_own / n_active) * n_active + split;   // slots of one row are adjacent, in rank order
+            const uint32_t ml_dst = map_to_rank(smem_base + kOffQ + slot * 8, owner);
+            const uint32_t o_dst = map_to_rank(smem_base + kOffK + slot * 512, owner);
+            if (ok) {
+                tc_fence_after();
+                uint32_t oreg[32];
 #pragma unroll
                 for (int c4 = 0; c4 < 4; ++c4) {
                     tmem_ld_x32(tO + c4 * 32, oreg);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint4 pk;
-                        pk.x = pack_bf16(__uint_as_float(oreg[8 * v + 0]) * inv, __uint_as_float(oreg[8 * v + 1]) * inv);
-                        pk.y = pack_bf16(__uint_as_float(oreg[8 * v + 2]) * inv, __uint_as_float(oreg[8 * v + 3]) * inv);
-                        pk.z = pack_bf16(__uint_as_float(oreg[8 * v + 4]) * inv, __uint_as_float(oreg[8 * v + 5]) * inv);
-                        pk.w = pack_bf16(__uint_as_float(oreg[8 * v + 6]) * inv, __uint_as_float(oreg[8 * v + 7]) * inv);
-                        *(uint4*)(stage + lane * 256 + (((c4 * 4 + v) ^ (lane & 7)) << 4)) = pk;
-                    }
+                    for (int v = 0; v < 8; ++v)
+                        st_cluster_u4(o_dst + (((c4 * 8 + v) ^ (slot & 31)) << 4), oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
                 }
-                if (valid && p.lse) p.lse[(long long)(sp.q_row0 + i) * p.hq + h] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
-                __syncwarp();
-                // two rows per trip: a half-warp writes one 256-byte row
-                const int sub = lane >> 4, ch = lane & 15;
-#pragma unroll 4
-                for (int rr = 0; rr < 32; rr += 2) {
-                    const int rl = rr + sub, ro = r_warp0 + rl;
-                    if (ro < rows) {
-                        const int io = ro / G, ho = g * G + (ro - io * G);
-                        const uint4 v = *(const uint4*)(stage + rl * 256 + ((ch ^ (rl & 7)) << 4));
-                        *(uint4*)((unsigned char*)p.out + (((long long)(sp.q_row0 + io) * p.hq + ho) * 256 + ch * 16)) = v;
-                    }
-                }
+                st_cluster_f2(ml_dst, m_ref, l_run);
             } else {
-                // fp32 partials: 512 bytes per row, staged in two passes of 64 columns (16 KB per warp)
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-#pragma unroll
-                    for (int c4 = 0; c4 < 2; ++c4) {
-                        tmem_ld_x32(tO + hf * 64 + c4 * 32, oreg);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int v = 0; v < 8; ++v)
-                            *(uint4*)(stage + lane * 256 + (((c4 * 8 + v) ^ (lane & 7)) << 4)) =
-                                make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
-                    }
-                    __syncwarp();
-                    const int sub = lane >> 4, ch = lane & 15;
-#pragma unroll 4
-                    for (int rr = 0; rr < 32; rr += 2) {
-                        const int rl = rr + sub, ro = r_warp0 + rl;
-                        if (ro < rows) {
-                            const int io = ro / G, ho = g * G + (ro - io * G);
-                            const long long e = (long long)sp.part_base + ((long long)io * p.hq + ho) * sp.nsplit + split;
-                            const uint4 v = *(const uint4*)(stage + rl * 256 + ((ch ^ (rl & 7)) << 4));
-                            *(uint4*)((unsigned char*)(p.part_o + e * kD) + hf * 256 + ch * 16) = v;
-                        }
-                    }
-                    __syncwarp();
-                }
-                if (valid) {
-                    const long long e = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit + split;
-                    p.part_ml[e] = make_float2(m_ref, l_sum);
-                }
+                st_cluster_f2(ml_dst, -INFINITY, 0.f);   // this CTA gave up: contribute nothing
             }
         }
-    }
-    // ---- teardown
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        tc_fence_before();
+        cluster_arrive(); cluster_wait();
+        {
+            const float2* ml_stage = (const float2*)(smem + kOffQ);
+            const unsigned char* o_stage = smem + kOffK;
+            for (int j = warp - 4; split + n_active * j < kRowsPerCta; j += 8) {
+                const int rl = split + n_active * j;
+                const int ro = row0 + rl;
+                if (ro >= rows) break;
+                const int slot0 = j * n_active;
+                float m_all = -INFINITY;
+                for (int k = 0; k < n_active; ++k) m_all = fmaxf(m_all, ml_stage[slot0 + k].x);
+                float l_all = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int k = 0; k < n_active; ++k) {
+                    const float2 ml = ml_stage[slot0 + k];
+                    if (ml.x != -INFINITY) {
+                        const float w = ex2(ml.x - m_all);
+                        l_all += ml.y * w;
+                        const float4 v = *(const float4*)(o_stage + (slot0 + k) * 512 + ((lane ^ ((slot0 + k) & 31)) << 4));
+                        acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+                    }
+                }
+                const float inv = (l_all > 0.f) ? 1.f / l_all : 0.f;
+                const int io = ro / G, ho = g * G + (ro - io * G);
+                uint2 pk;
+                pk.x = pack_bf16(acc.x * inv, acc.y * inv);
+                pk.y = pack_bf16(acc.z * inv, acc.w * inv);
+                *(uint2*)((unsigned char*)p.out + (((long long)(sp.q_row0 + io) * p.hq + ho) * 256 + lane * 8)) = pk;
+                if (p.lse && lane == 0) p.lse[(long long)(sp.q_row0 + io) * p.hq + ho] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+            }
+        }
     }
 }
 
@@ -543,20 +621,65 @@ bool make_pool_map(CUtensorMap* map, const void* pool, long long num_pages, int 
     return make_pool_map_impl(map, pool, num_pages, hkv);
 }
 
-cudaError_t launch_attn_tile_bf16(const AttnParams& p, cudaStream_t stream) {
-    if (p.num_items == 0) return cudaSuccess;
-    if ((long long)p.num_pages * p.hkv * kPage > 0x7FFFFFFFll) return cudaErrorInvalidValue;
-    alignas(64) CUtensorMap map_k, map_v;
-    if (!make_pool_map(&map_k, p.k_pool, p.num_pages, p.hkv) || !make_pool_map(&map_v, p.v_pool, p.num_pages, p.hkv))
-        return cudaErrorNotSupported;
+namespace {
+cudaError_t configure_tile_kernel() {
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(attn_tile_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    attn_tile_bf16_kernel<<<p.num_items, kThreads, kSmemBytes, stream>>>(p, map_k, map_v);
-    return cudaGetLastError();
+    return cudaSuccess;
+}
+void fill_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int grid, int cluster, cudaStream_t stream) {
+    cfg = cudaLaunchConfig_t{};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+}
+}  // namespace
+
+// CTAs of the tile kernel that can be resident at once when launched in clusters of `cluster` (1..8);
+// 0 when such clusters cannot be placed.  Cached per cluster size (one device per process is assumed).
+int attn_tile_resident_ctas(int cluster) {
+    static int cache[kMaxTileCluster + 1] = {0};
+    static bool known[kMaxTileCluster + 1] = {false};
+    if (cluster < 1 || cluster > kMaxTileCluster) return 0;
+    if (!known[cluster]) {
+        int n = 0;
+        if (configure_tile_kernel() == cudaSuccess) {
+            cudaLaunchConfig_t cfg;
+            cudaLaunchAttribute attr[1];
+            fill_launch_config(cfg, attr, cluster, cluster, nullptr);
+            if (cudaOccupancyMaxActiveClusters(&n, attn_tile_bf16_kernel, &cfg) != cudaSuccess) { n = 0; (void)cudaGetLastError(); }
+        }
+        cache[cluster] = n * cluster;
+        known[cluster] = true;
+    }
+    return cache[cluster];
+}
+
+cudaError_t launch_attn_tile_bf16(const AttnParams& p, int cluster, cudaStream_t stream) {
+    if (p.num_items == 0) return cudaSuccess;
+    if (cluster < 1 || cluster > kMaxTileCluster || p.num_items % cluster != 0) return cudaErrorInvalidValue;
+    if ((long long)p.num_pages * p.hkv * kPage > 0x7FFFFFFFll) return cudaErrorInvalidValue;
+    alignas(64) CUtensorMap map_k, map_v;
+    if (!make_pool_map(&map_k, p.k_pool, p.num_pages, p.hkv) || !make_pool_map(&map_v, p.v_pool, p.num_pages, p.hkv))
+        return cudaErrorNotSupported;
+    cudaError_t e = configure_tile_kernel();
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    fill_launch_config(cfg, attr, p.num_items, cluster, stream);
+    return cudaLaunchKernelEx(&cfg, attn_tile_bf16_kernel, p, map_k, map_v);
 }
 
 }  // namespace agx
+
