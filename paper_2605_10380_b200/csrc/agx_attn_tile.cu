@@ -29,6 +29,7 @@
 #include "agx_sm100.cuh"
 
 namespace agx {
+
 namespace {
 
 constexpr int kD = 128;
@@ -43,6 +44,7 @@ constexpr uint32_t kOffQ = 0;
 constexpr uint32_t kOffK = 2 * kTileBytes;
 constexpr uint32_t kOffV = kOffK + kStagesK * kTileBytes;
 constexpr uint32_t kOffBar = kOffV + kStagesV * kTileBytes;
+constexpr uint32_t kOffML = kOffK + kRowsPerCta * 512;   // epilogue: (m, l) per row, behind the parked O rows
 constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // + barriers + alignment slack
 constexpr float kRescaleThreshold = 8.0f;              // log2 units
 #ifndef AGX_POLY_PAIRS
@@ -161,11 +163,15 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(saddr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_cluster_u4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};\n" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
 }
-__device__ __forceinline__ void st_cluster_f2(uint32_t addr, float a, float b) {
-    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};\n" ::"r"(addr), "f"(a), "f"(b) : "memory");
+__device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];\n" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+    return v;
 }
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
@@ -177,6 +183,128 @@ __device__ __forceinline__ int find_seq(const AttnParams& p, int item) {
     for (int i = 1; i < p.num_seqs; ++i)
         if (p.seq[i].item0 <= item) s = i;
     return s;
+}
+
+// What one CTA works on, derived from its block index alone.
+struct TileItem {
+    int g, G, P, q, rows, row0, split, nsplit, n_tiles, n_active, kv_begin, kv_end, vis_end, q_row0, seq_index;
+};
+__device__ __forceinline__ TileItem locate_item(const AttnParams& p, int block) {
+    const int si = find_seq(p, block);
+    const SeqPlan& sp = p.seq[si];
+    TileItem it;
+    int local = block - sp.item0;  // ((g * row_chunks) + rc) * nsplit + split
+    it.nsplit = sp.nsplit;
+    it.split = local % sp.nsplit;
+    local /= sp.nsplit;
+    const int rc = local % sp.row_chunks;
+    it.g = local / sp.row_chunks;
+    it.G = p.hq / p.hkv;
+    it.P = sp.prefix_len; it.q = sp.q_len;
+    it.rows = it.q * it.G;
+    it.row0 = rc * kRowsPerCta;
+    it.vis_end = it.P + min(it.q - 1, (it.row0 + kRowsPerCta - 1) / it.G) + 1;  // tokens the chunk's last row sees
+    it.kv_begin = it.split * sp.split_tokens;
+    it.kv_end = min(it.vis_end, it.kv_begin + sp.split_tokens);
+    it.n_tiles = max(0, (it.kv_end - it.kv_begin + kBN - 1) / kBN);
+    // splits are in token order, so the active ones are ranks 0 .. n_active - 1
+    it.n_active = min(sp.nsplit, (it.vis_end + sp.split_tokens - 1) / sp.split_tokens);
+    it.q_row0 = sp.q_row0; it.seq_index = sp.seq_index;
+    return it;
+}
+
+// Epilogue of a softmax thread.  Every KV split of one (sequence, KV head, row chunk) is one CTA of the
+// cluster.  Each CTA parks its un-normalised fp32 O rows and their (m, l) in its own shared memory (the
+// K/V rings are idle once its last MMA has completed).  After a cluster barrier, row rl of the chunk
+// belongs to the active CTA of rank rl % n_active: its softmax warps fetch the row's n_active partials
+// and (m, l) pairs from the peers' shared memory (whole 512-byte rows, eight rows in flight per warp),
+// merge them in rank order with the usual running-maximum update and write whole bf16 rows.  No partials in global memory, no second kernel, fixed order:
+// bit-reproducible.  A last barrier keeps every CTA's shared memory alive until its peers have read it.
+// Kept out of line, and re-deriving its indices from the block index, so that nothing but its few
+// arguments has to stay alive across the register-hungry main loop.
+__device__ __noinline__ void tile_epilogue(const AttnParams& p, unsigned char* smem, uint32_t tO, float m_ref, float l_run, bool ok) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const TileItem it = locate_item(p, blockIdx.x);
+    const uint32_t smem_base = smem_u32(smem);
+    const int n = it.n_active;
+    {
+        const int rl_own = tid - 128;                                   // row of the chunk this thread holds
+        if (ok) {
+            tc_fence_after();
+            uint32_t oreg[32];
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+                tmem_ld_x32(tO + c4 * 32, oreg);
+                tmem_wait_ld();
+#pragma unroll
+                for (int v = 0; v < 8; ++v)
+                    *(uint4*)(smem + kOffK + rl_own * 512 + (((c4 * 8 + v) ^ (rl_own & 31)) << 4)) =
+                        make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
+            }
+        }
+        // a CTA that gave up contributes nothing
+        *(float2*)(smem + kOffML + rl_own * 8) = ok ? make_float2(m_ref, l_run) : make_float2(-INFINITY, 0.f);
+    }
+    tc_fence_before();
+    cluster_arrive(); cluster_wait();
+    const uint64_t magic = (0x100000000ull + it.G - 1) / it.G;  // (row * magic) >> 32 == row / G exactly for rows < 2^22
+    constexpr int kBatch = 8;
+    for (int j0 = warp - 4; it.split + n * j0 < kRowsPerCta; j0 += 8 * kBatch) {
+        int rl[kBatch];
+        bool valid[kBatch];
+        float m_all[kBatch], l_all[kBatch];
+        float4 acc[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            rl[u] = it.split + n * (j0 + 8 * u);
+            valid[u] = rl[u] < kRowsPerCta && it.row0 + rl[u] < it.rows;
+            if (!valid[u]) rl[u] = it.split;       // harmless duplicate
+            m_all[u] = -INFINITY; l_all[u] = 0.f;
+            acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (int k = 0; k < n; ++k) {
+            float4 v[kBatch];
+            float2 ml[kBatch];
+            if (k == it.split) {   // this CTA's own partial: plain shared-memory loads
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    ml[u] = *(const float2*)(smem + kOffML + rl[u] * 8);
+                    v[u] = *(const float4*)(smem + kOffK + rl[u] * 512 + ((lane ^ (rl[u] & 31)) << 4));
+                }
+            } else {
+                const uint32_t peer_o = map_to_rank(smem_base + kOffK, k), peer_ml = map_to_rank(smem_base + kOffML, k);
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    ml[u] = ld_cluster_f2(peer_ml + rl[u] * 8);
+                    v[u] = ld_cluster_f4(peer_o + rl[u] * 512 + ((lane ^ (rl[u] & 31)) << 4));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                if (ml[u].x != -INFINITY) {
+                    const float m_new = fmaxf(m_all[u], ml[u].x);
+                    const float c = ex2(m_all[u] - m_new), w = ex2(ml[u].x - m_new);   // c = 0 on the first contribution
+                    m_all[u] = m_new;
+                    l_all[u] = l_all[u] * c + ml[u].y * w;
+                    acc[u].x = acc[u].x * c + v[u].x * w; acc[u].y = acc[u].y * c + v[u].y * w;
+                    acc[u].z = acc[u].z * c + v[u].z * w; acc[u].w = acc[u].w * c + v[u].w * w;
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            if (!valid[u]) continue;
+            const int ro = it.row0 + rl[u];
+            const float inv = (l_all[u] > 0.f) ? 1.f / l_all[u] : 0.f;
+            const int io = (int)(((uint64_t)(uint32_t)ro * magic) >> 32), ho = it.g * it.G + (ro - io * it.G);
+            uint2 pk;
+            pk.x = pack_bf16(acc[u].x * inv, acc[u].y * inv);
+            pk.y = pack_bf16(acc[u].z * inv, acc[u].w * inv);
+            *(uint2*)((unsigned char*)p.out + (((long long)(it.q_row0 + io) * p.hq + ho) * 256 + lane * 8)) = pk;
+            if (p.lse && lane == 0) p.lse[(long long)(it.q_row0 + io) * p.hq + ho] = (m_all[u] + log2f(l_all[u])) * 0.6931471805599453f;
+        }
+    }
+    cluster_arrive(); cluster_wait();   // peers may be reading this CTA's shared memory until here
 }
 
 }  // namespace
@@ -194,30 +322,16 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     // ---- work item
-    const int si = find_seq(p, blockIdx.x);
-    const SeqPlan sp = p.seq[si];
-    int local = blockIdx.x - sp.item0;  // ((g * row_chunks) + rc) * nsplit + split
-    const int split = local % sp.nsplit;
-    local /= sp.nsplit;
-    const int rc = local % sp.row_chunks;
-    const int g = local / sp.row_chunks;
-    const int G = p.hq / p.hkv;
-    const int P = sp.prefix_len, q = sp.q_len, L = P + q;
-    const int rows = q * G;
-    const int row0 = rc * kRowsPerCta;
-    const int vis_end = P + min(q - 1, (row0 + kRowsPerCta - 1) / G) + 1;  // tokens the chunk's last row sees
-    const int kv_begin = split * sp.split_tokens;
-    const int kv_end = min(vis_end, kv_begin + sp.split_tokens);
-    const int n_tiles = max(0, (kv_end - kv_begin + kBN - 1) / kBN);
+    const TileItem it = locate_item(p, blockIdx.x);
+    const SeqPlan& sp = p.seq[find_seq(p, blockIdx.x)];
+    const int split = it.split, g = it.g, G = it.G, P = it.P, q = it.q, L = P + q, rows = it.rows, row0 = it.row0;
+    const int kv_begin = it.kv_begin, kv_end = it.kv_end, n_tiles = it.n_tiles;
 
     if (n_tiles == 0) {  // nothing visible in this split: only keep the cluster's two barriers company
         cluster_arrive(); cluster_wait();
         cluster_arrive(); cluster_wait();
         return;
     }
-    // splits are in token order, so the active ones are ranks 0 .. n_active - 1
-    const int n_active = min(sp.nsplit, (vis_end + sp.split_tokens - 1) / sp.split_tokens);
-
     // ---- setup: barriers, TMEM, Q tiles
     if (tid == 0) {
         for (int i = 0; i < BAR_COUNT; ++i)
@@ -394,12 +508,12 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         __syncwarp();
     }
     tc_fence_before();
-    cluster_arrive(); cluster_wait();       // every CTA of the cluster has left its main loop
-    cluster_arrive(); cluster_wait();       // every CTA has delivered its O rows: the softmax warps are done with TMEM
+    cluster_arrive(); cluster_wait();       // every CTA of the cluster has parked its O rows: TMEM is no longer read
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
+    cluster_arrive(); cluster_wait();       // ... and merged its rows out of its peers' shared memory
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsHigh));
         // ================= softmax + epilogue: one thread per query row =================
@@ -518,70 +632,8 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             tc_fence_before();
             mbar_arrive(bar(BAR_P_READY + x));
         }
-        // ---- epilogue.  Every KV split of this (sequence, KV head, row chunk) is one CTA of the
-        //      cluster.  Row rl of the chunk is owned by the active CTA of rank rl % n_active.  Once
-        //      every CTA of the cluster has left its main loop (first cluster barrier: the K/V rings are
-        //      idle everywhere), each CTA sends its un-normalised fp32 O rows and (m, l) into the owners'
-        //      shared memory with remote stores; after the second barrier an owner merges the splits of
-        //      its rows in rank order from its own shared memory and writes whole bf16 rows.  No
-        //      partials in global memory, no second kernel, fixed order: bit-reproducible.
         if (ok) ok = mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
-        tc_fence_before();
-        cluster_arrive(); cluster_wait();
-        {
-            const int rl_own = x * 128 + rt;
-            const int owner = rl_own % n_active;
-            const int slot = (rl_own / n_active) * n_active + split;   // slots of one row are adjacent, in rank order
-            const uint32_t ml_dst = map_to_rank(smem_base + kOffQ + slot * 8, owner);
-            const uint32_t o_dst = map_to_rank(smem_base + kOffK + slot * 512, owner);
-            if (ok) {
-                tc_fence_after();
-                uint32_t oreg[32];
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    tmem_ld_x32(tO + c4 * 32, oreg);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int v = 0; v < 8; ++v)
-                        st_cluster_u4(o_dst + (((c4 * 8 + v) ^ (slot & 31)) << 4), oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
-                }
-                st_cluster_f2(ml_dst, m_ref, l_run);
-            } else {
-                st_cluster_f2(ml_dst, -INFINITY, 0.f);   // this CTA gave up: contribute nothing
-            }
-        }
-        tc_fence_before();
-        cluster_arrive(); cluster_wait();
-        {
-            const float2* ml_stage = (const float2*)(smem + kOffQ);
-            const unsigned char* o_stage = smem + kOffK;
-            for (int j = warp - 4; split + n_active * j < kRowsPerCta; j += 8) {
-                const int rl = split + n_active * j;
-                const int ro = row0 + rl;
-                if (ro >= rows) break;
-                const int slot0 = j * n_active;
-                float m_all = -INFINITY;
-                for (int k = 0; k < n_active; ++k) m_all = fmaxf(m_all, ml_stage[slot0 + k].x);
-                float l_all = 0.f;
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int k = 0; k < n_active; ++k) {
-                    const float2 ml = ml_stage[slot0 + k];
-                    if (ml.x != -INFINITY) {
-                        const float w = ex2(ml.x - m_all);
-                        l_all += ml.y * w;
-                        const float4 v = *(const float4*)(o_stage + (slot0 + k) * 512 + ((lane ^ ((slot0 + k) & 31)) << 4));
-                        acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
-                    }
-                }
-                const float inv = (l_all > 0.f) ? 1.f / l_all : 0.f;
-                const int io = ro / G, ho = g * G + (ro - io * G);
-                uint2 pk;
-                pk.x = pack_bf16(acc.x * inv, acc.y * inv);
-                pk.y = pack_bf16(acc.z * inv, acc.w * inv);
-                *(uint2*)((unsigned char*)p.out + (((long long)(sp.q_row0 + io) * p.hq + ho) * 256 + lane * 8)) = pk;
-                if (p.lse && lane == 0) p.lse[(long long)(sp.q_row0 + io) * p.hq + ho] = (m_all + log2f(l_all)) * 0.6931471805599453f;
-            }
-        }
+        tile_epilogue(p, smem, tO, m_ref, l_run, ok);
     }
 }
 
