@@ -51,7 +51,6 @@ enum Kind { KIND_SMALL1 = 0, KIND_SMALL2, KIND_SMALL4, KIND_TILE, KIND_SIMT, KIN
 
 struct Launch {
     Kind kind;
-    int cluster;     // KIND_TILE: CTAs per cluster (= KV splits of every sequence)
     int total_rows;  // sum of q_len over the launch's sequences
     int num_items;
     std::vector<SeqPlan> seqs;
@@ -119,26 +118,20 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
             }
             return items;
         };
-        int tile_cluster = 1;
         if (k == KIND_TILE) {
-            // Every sequence is cut into the same number n of KV splits (one thread-block cluster of n
-            // CTAs per row chunk).  Pick n by the estimated makespan: waves of resident CTAs times
-            // (KV tiles of the longest split + ~3 tiles of fixed per-CTA cost).
+            // several waves are fine here: pick the split length with the smallest estimated makespan,
+            // waves * (tiles per item + fixed per-CTA cost of ~3 tiles)
             int max_len = 0;
             for (int s : seqs) max_len = std::max(max_len, P[s] + Q[s]);
             long long best_cost = -1;
-            for (int n = 1; n <= kMaxTileCluster; ++n) {
-                const int resident = attn_tile_resident_ctas(n);
-                if (resident <= 0) continue;
-                const long long waves = (base_items * n + resident - 1) / resident;
-                const int tiles = (round_up((max_len + n - 1) / n, unit)) / unit;
-                const long long cost = waves * (tiles + 3);
-                if (best_cost < 0 || cost < best_cost) { best_cost = cost; tile_cluster = n; }
+            for (int c_tokens = min_split; c_tokens < max_len + unit; c_tokens += unit) {
+                const long long waves = (count_items(c_tokens) + h->sm_count - 1) / h->sm_count;
+                const long long cost = waves * (std::min(c_tokens, round_up(max_len, unit)) / unit + 3);
+                if (best_cost < 0 || cost < best_cost) { best_cost = cost; C = c_tokens; }
             }
-            if (best_cost < 0) return fail(h, AGX_E_CUDA, "the tile kernel cannot be placed on this device");
             if (h->debug_plan)
-                fprintf(stderr, "agx plan: tile kernel, %lld row chunks, longest sequence %d tokens -> clusters of %d (resident CTAs %d)\n",
-                        base_items, max_len, tile_cluster, attn_tile_resident_ctas(tile_cluster));
+                fprintf(stderr, "agx plan: tile kernel, %lld row chunks, longest sequence %d tokens -> KV splits of %d tokens, %lld CTAs\n",
+                        base_items, max_len, C, count_items(C));
         } else {
             while (count_items(C) > std::max<long long>(target, base_items)) C += unit;
         }
@@ -146,7 +139,6 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
         for (size_t a = 0; a < seqs.size(); a += kMaxSeqs) {
             Launch ln;
             ln.kind = (Kind)k;
-            ln.cluster = tile_cluster;
             ln.total_rows = 0;
             ln.num_items = 0;
             for (size_t n = a; n < std::min(seqs.size(), a + kMaxSeqs); ++n) {
@@ -157,18 +149,13 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
                 sp.q_len = Q[s];
                 sp.q_row0 = row0[s];
                 sp.seq_index = s;
-                if (k == KIND_TILE) {
-                    sp.nsplit = tile_cluster;   // splits past the end of a short sequence stay empty
-                    sp.split_tokens = round_up((L + sp.nsplit - 1) / sp.nsplit, unit);
-                } else {
-                    sp.nsplit = (L + C - 1) / C;
-                    sp.split_tokens = round_up((L + sp.nsplit - 1) / sp.nsplit, unit);
-                    sp.nsplit = (L + sp.split_tokens - 1) / sp.split_tokens;
-                }
+                sp.nsplit = (L + C - 1) / C;
+                sp.split_tokens = round_up((L + sp.nsplit - 1) / sp.nsplit, unit);
+                sp.nsplit = (L + sp.split_tokens - 1) / sp.split_tokens;
                 sp.row_chunks = (k == KIND_SIMT) ? 1 : (Q[s] * G + rows_per_chunk - 1) / rows_per_chunk;
                 sp.item0 = ln.num_items;
                 sp.part_base = 0;
-                if (sp.nsplit > 1 && k != KIND_TILE) {   // the tile kernel merges its splits on chip
+                if (sp.nsplit > 1) {
                     if (plan.part_entries + (long long)Q[s] * c.num_q_heads * sp.nsplit > 0x7FFFFFFFll)
                         return fail(h, AGX_E_RANGE, "split partials exceed 2^31 entries");
                     sp.part_base = (int)plan.part_entries;
@@ -319,14 +306,14 @@ agx_status agx_attn_prefixed(agx_handle* h, const void* q_block, const void* k_p
         p.num_seqs = (int)ln.seqs.size();
         p.num_items = ln.num_items;
         bool split = false;
-        for (int i = 0; i < p.num_seqs; ++i) { p.seq[i] = ln.seqs[i]; split |= ln.seqs[i].nsplit > 1 && ln.kind != KIND_TILE; }
+        for (int i = 0; i < p.num_seqs; ++i) { p.seq[i] = ln.seqs[i]; split |= ln.seqs[i].nsplit > 1; }
         cudaError_t e;
         switch (ln.kind) {
             case KIND_SMALL1: e = launch_attn_small_bf16(p, 1, stream); break;
             case KIND_SMALL2: e = launch_attn_small_bf16(p, 2, stream); break;
             case KIND_SMALL4: e = launch_attn_small_bf16(p, 4, stream); break;
             case KIND_SIMT: e = launch_attn_simt_f32(p, stream); break;
-            case KIND_TILE: e = launch_attn_tile_bf16(p, ln.cluster, stream); break;
+            case KIND_TILE: e = launch_attn_tile_bf16(p, stream); break;
             default: return fail(h, AGX_E_UNSUPPORTED, "unknown kernel kind");
         }
         if (e != cudaSuccess) return cuda_fail(h, e, "attention launch");

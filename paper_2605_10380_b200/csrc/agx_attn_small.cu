@@ -487,13 +487,17 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
                 v[j] = *(const float4*)(p.part_o + (e0 + k + j) * D + c4);
             }
 #pragma unroll
-            for (int j = 0; j < 4; ++j) { acc.x += v[j].x * w[j]; acc.y += v[j].y * w[j]; acc.z += v[j].z * w[j]; acc.w += v[j].w * w[j]; }
+            for (int j = 0; j < 4; ++j) {
+                if (w[j] != 0.f) {   // a split that saw no token for this row publishes only (m, l) = (-inf, 0)
+                    acc.x += v[j].x * w[j]; acc.y += v[j].y * w[j]; acc.z += v[j].z * w[j]; acc.w += v[j].w * w[j];
+                }
+            }
         }
         for (; k < ns; ++k) {
             const float mk = p.part_ml[e0 + k].x;
             const float w = (mk == -INFINITY) ? 0.f : exp2f(mk - m_all);
             const float4 v = *(const float4*)(p.part_o + (e0 + k) * D + c4);
-            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+            if (w != 0.f) { acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w; }
         }
     }
     const float inv = 1.f / l_all;

@@ -44,13 +44,16 @@ constexpr uint32_t kOffQ = 0;
 constexpr uint32_t kOffK = 2 * kTileBytes;
 constexpr uint32_t kOffV = kOffK + kStagesK * kTileBytes;
 constexpr uint32_t kOffBar = kOffV + kStagesV * kTileBytes;
-constexpr uint32_t kOffML = kOffK + kRowsPerCta * 512;   // epilogue: (m, l) per row, behind the parked O rows
 constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // + barriers + alignment slack
 constexpr float kRescaleThreshold = 8.0f;              // log2 units
+// Of every 8 column pairs, this many take the polynomial 2^x instead of the special-function unit.
+// Measured on B200 (P = 30720, q = 2048): 0 -> 950 us, 1 -> 957, 2 -> 964, 4 -> 982: the extra FMA-pipe
+// instructions cost more issue slots (shared with the MMA-issuing warp) than the special-function unit
+// gives back, so the default is 0 and the option only remains for experiments.
 #ifndef AGX_POLY_PAIRS
-#define AGX_POLY_PAIRS 3
+#define AGX_POLY_PAIRS 0
 #endif
-constexpr int kPolyPairsOf8 = AGX_POLY_PAIRS;          // of every 8 column pairs, this many take the polynomial 2^x
+constexpr int kPolyPairsOf8 = AGX_POLY_PAIRS;
 
 // barrier slots (8 bytes each)
 enum { BAR_K_FULL = 0, BAR_K_EMPTY = 3, BAR_V_FULL = 6, BAR_V_EMPTY = 8, BAR_S_FULL = 10, BAR_P_READY = 12,
@@ -155,24 +158,6 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;\n" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;\n" ::: "memory"); }
-// address of the same shared-memory location in the CTA of rank `rank` of this cluster
-__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(saddr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
-    float4 v;
-    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
-    float2 v;
-    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];\n" : "=f"(v.x), "=f"(v.y) : "r"(addr));
-    return v;
-}
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
@@ -187,7 +172,7 @@ __device__ __forceinline__ int find_seq(const AttnParams& p, int item) {
 
 // What one CTA works on, derived from its block index alone.
 struct TileItem {
-    int g, G, P, q, rows, row0, split, nsplit, n_tiles, n_active, kv_begin, kv_end, vis_end, q_row0, seq_index;
+    int g, G, P, q, rows, row0, split, nsplit, n_tiles, kv_begin, kv_end, vis_end, q_row0, seq_index;
 };
 __device__ __forceinline__ TileItem locate_item(const AttnParams& p, int block) {
     const int si = find_seq(p, block);
@@ -207,104 +192,69 @@ __device__ __forceinline__ TileItem locate_item(const AttnParams& p, int block) 
     it.kv_begin = it.split * sp.split_tokens;
     it.kv_end = min(it.vis_end, it.kv_begin + sp.split_tokens);
     it.n_tiles = max(0, (it.kv_end - it.kv_begin + kBN - 1) / kBN);
-    // splits are in token order, so the active ones are ranks 0 .. n_active - 1
-    it.n_active = min(sp.nsplit, (it.vis_end + sp.split_tokens - 1) / sp.split_tokens);
     it.q_row0 = sp.q_row0; it.seq_index = sp.seq_index;
     return it;
 }
 
-// Epilogue of a softmax thread.  Every KV split of one (sequence, KV head, row chunk) is one CTA of the
-// cluster.  Each CTA parks its un-normalised fp32 O rows and their (m, l) in its own shared memory (the
-// K/V rings are idle once its last MMA has completed).  After a cluster barrier, row rl of the chunk
-// belongs to the active CTA of rank rl % n_active: its softmax warps fetch the row's n_active partials
-// and (m, l) pairs from the peers' shared memory (whole 512-byte rows, eight rows in flight per warp),
-// merge them in rank order with the usual running-maximum update and write whole bf16 rows.  No partials in global memory, no second kernel, fixed order:
-// bit-reproducible.  A last barrier keeps every CTA's shared memory alive until its peers have read it.
-// Kept out of line, and re-deriving its indices from the block index, so that nothing but its few
-// arguments has to stay alive across the register-hungry main loop.
-__device__ __noinline__ void tile_epilogue(const AttnParams& p, unsigned char* smem, uint32_t tO, float m_ref, float l_run, bool ok) {
+// Epilogue of a softmax thread: the un-normalised fp32 O row leaves TMEM through this warp's 16 KB of
+// the (now idle) K/V rings, so that global stores are whole rows written by whole warps.  With a single
+// KV split the rows are normalised and written as bf16; otherwise fp32 partials and (m, l) go to the
+// workspace for the combine kernel.  Kept out of line, and re-deriving its indices from the block index,
+// so that nothing but its few arguments has to stay alive across the register-hungry main loop.
+__device__ __noinline__ void tile_epilogue(const AttnParams& p, unsigned char* smem, uint32_t tO, float m_ref, float l_run) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const TileItem it = locate_item(p, blockIdx.x);
-    const uint32_t smem_base = smem_u32(smem);
-    const int n = it.n_active;
+    const SeqPlan& sp = p.seq[find_seq(p, blockIdx.x)];
+    unsigned char* stage = smem + kOffK + (warp - 4) * 16384;    // [32 rows][512 B], 16-byte units XOR-swizzled by row
+    const int r_warp0 = it.row0 + (warp - 4) * 32;               // first row of this warp
+    const uint64_t magic = (0x100000000ull + it.G - 1) / it.G;   // (row * magic) >> 32 == row / G exactly for rows < 2^22
+    const bool single = it.nsplit == 1;
+    const float inv = (l_run > 0.f) ? 1.f / l_run : 0.f;
+    tc_fence_after();
     {
-        const int rl_own = tid - 128;                                   // row of the chunk this thread holds
-        if (ok) {
-            tc_fence_after();
-            uint32_t oreg[32];
+        uint32_t oreg[32];
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                tmem_ld_x32(tO + c4 * 32, oreg);
-                tmem_wait_ld();
+        for (int c4 = 0; c4 < 4; ++c4) {
+            tmem_ld_x32(tO + c4 * 32, oreg);
+            tmem_wait_ld();
+            if (single) {
 #pragma unroll
-                for (int v = 0; v < 8; ++v)
-                    *(uint4*)(smem + kOffK + rl_own * 512 + (((c4 * 8 + v) ^ (rl_own & 31)) << 4)) =
-                        make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
+                for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * inv);
             }
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+                *(uint4*)(stage + lane * 512 + (((c4 * 8 + v) ^ lane) << 4)) = make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
         }
-        // a CTA that gave up contributes nothing
-        *(float2*)(smem + kOffML + rl_own * 8) = ok ? make_float2(m_ref, l_run) : make_float2(-INFINITY, 0.f);
     }
-    tc_fence_before();
-    cluster_arrive(); cluster_wait();
-    const uint64_t magic = (0x100000000ull + it.G - 1) / it.G;  // (row * magic) >> 32 == row / G exactly for rows < 2^22
-    constexpr int kBatch = 8;
-    for (int j0 = warp - 4; it.split + n * j0 < kRowsPerCta; j0 += 8 * kBatch) {
-        int rl[kBatch];
-        bool valid[kBatch];
-        float m_all[kBatch], l_all[kBatch];
-        float4 acc[kBatch];
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            rl[u] = it.split + n * (j0 + 8 * u);
-            valid[u] = rl[u] < kRowsPerCta && it.row0 + rl[u] < it.rows;
-            if (!valid[u]) rl[u] = it.split;       // harmless duplicate
-            m_all[u] = -INFINITY; l_all[u] = 0.f;
-            acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        for (int k = 0; k < n; ++k) {
-            float4 v[kBatch];
-            float2 ml[kBatch];
-            if (k == it.split) {   // this CTA's own partial: plain shared-memory loads
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    ml[u] = *(const float2*)(smem + kOffML + rl[u] * 8);
-                    v[u] = *(const float4*)(smem + kOffK + rl[u] * 512 + ((lane ^ (rl[u] & 31)) << 4));
-                }
+    {   // per-row scalars
+        const int r = r_warp0 + lane;
+        if (r < it.rows) {
+            const int i = (int)(((uint64_t)(uint32_t)r * magic) >> 32), h = it.g * it.G + (r - i * it.G);
+            if (single) {
+                if (p.lse) p.lse[(long long)(it.q_row0 + i) * p.hq + h] = (m_ref + log2f(l_run)) * 0.6931471805599453f;
             } else {
-                const uint32_t peer_o = map_to_rank(smem_base + kOffK, k), peer_ml = map_to_rank(smem_base + kOffML, k);
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    ml[u] = ld_cluster_f2(peer_ml + rl[u] * 8);
-                    v[u] = ld_cluster_f4(peer_o + rl[u] * 512 + ((lane ^ (rl[u] & 31)) << 4));
-                }
+                p.part_ml[(long long)sp.part_base + ((long long)i * p.hq + h) * it.nsplit + it.split] = make_float2(m_ref, l_run);
             }
-#pragma unroll
-            for (int u = 0; u < kBatch; ++u) {
-                if (ml[u].x != -INFINITY) {
-                    const float m_new = fmaxf(m_all[u], ml[u].x);
-                    const float c = ex2(m_all[u] - m_new), w = ex2(ml[u].x - m_new);   // c = 0 on the first contribution
-                    m_all[u] = m_new;
-                    l_all[u] = l_all[u] * c + ml[u].y * w;
-                    acc[u].x = acc[u].x * c + v[u].x * w; acc[u].y = acc[u].y * c + v[u].y * w;
-                    acc[u].z = acc[u].z * c + v[u].z * w; acc[u].w = acc[u].w * c + v[u].w * w;
-                }
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            if (!valid[u]) continue;
-            const int ro = it.row0 + rl[u];
-            const float inv = (l_all[u] > 0.f) ? 1.f / l_all[u] : 0.f;
-            const int io = (int)(((uint64_t)(uint32_t)ro * magic) >> 32), ho = it.g * it.G + (ro - io * it.G);
-            uint2 pk;
-            pk.x = pack_bf16(acc[u].x * inv, acc[u].y * inv);
-            pk.y = pack_bf16(acc[u].z * inv, acc[u].w * inv);
-            *(uint2*)((unsigned char*)p.out + (((long long)(it.q_row0 + io) * p.hq + ho) * 256 + lane * 8)) = pk;
-            if (p.lse && lane == 0) p.lse[(long long)(it.q_row0 + io) * p.hq + ho] = (m_all[u] + log2f(l_all[u])) * 0.6931471805599453f;
         }
     }
-    cluster_arrive(); cluster_wait();   // peers may be reading this CTA's shared memory until here
+    __syncwarp();
+    // a warp writes one row per instruction: lane j moves 16-byte unit j (fp32) or converts it to 8 bytes of bf16
+#pragma unroll 8
+    for (int rl = 0; rl < 32; ++rl) {
+        const int ro = r_warp0 + rl;
+        if (ro >= it.rows) break;
+        const int io = (int)(((uint64_t)(uint32_t)ro * magic) >> 32), ho = it.g * it.G + (ro - io * it.G);
+        const uint4 v = *(const uint4*)(stage + rl * 512 + ((lane ^ rl) << 4));
+        if (single) {
+            uint2 pk;
+            pk.x = pack_bf16(__uint_as_float(v.x), __uint_as_float(v.y));
+            pk.y = pack_bf16(__uint_as_float(v.z), __uint_as_float(v.w));
+            *(uint2*)((unsigned char*)p.out + (((long long)(it.q_row0 + io) * p.hq + ho) * 256 + lane * 8)) = pk;
+        } else {
+            const long long e = (long long)sp.part_base + ((long long)io * p.hq + ho) * it.nsplit + it.split;
+            *(uint4*)((unsigned char*)(p.part_o + e * kD) + lane * 16) = v;
+        }
+    }
 }
 
 }  // namespace
@@ -327,11 +277,17 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
     const int split = it.split, g = it.g, G = it.G, P = it.P, q = it.q, L = P + q, rows = it.rows, row0 = it.row0;
     const int kv_begin = it.kv_begin, kv_end = it.kv_end, n_tiles = it.n_tiles;
 
-    if (n_tiles == 0) {  // nothing visible in this split: only keep the cluster's two barriers company
-        cluster_arrive(); cluster_wait();
-        cluster_arrive(); cluster_wait();
+    if (n_tiles == 0) {  // nothing visible in this split (nsplit > 1 by construction): publish (m, l) = (-inf, 0);
+                         // the combine kernel does not read the O rows of such entries
+        for (int rl = tid; rl < kRowsPerCta; rl += kThreads) {
+            const int r = row0 + rl;
+            if (r >= rows) break;
+            const int i = r / G, h = g * G + (r - i * G);
+            p.part_ml[(long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit + split] = make_float2(-INFINITY, 0.f);
+        }
         return;
     }
+
     // ---- setup: barriers, TMEM, Q tiles
     if (tid == 0) {
         for (int i = 0; i < BAR_COUNT; ++i)
@@ -507,13 +463,6 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         }
         __syncwarp();
     }
-    tc_fence_before();
-    cluster_arrive(); cluster_wait();       // every CTA of the cluster has parked its O rows: TMEM is no longer read
-    if (warp == 1) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
-    }
-    cluster_arrive(); cluster_wait();       // ... and merged its rows out of its peers' shared memory
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsHigh));
         // ================= softmax + epilogue: one thread per query row =================
@@ -633,7 +582,14 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             mbar_arrive(bar(BAR_P_READY + x));
         }
         if (ok) ok = mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
-        tile_epilogue(p, smem, tO, m_ref, l_run, ok);
+        if (ok) tile_epilogue(p, smem, tO, m_ref, l_run);
+    }
+    // ---- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -673,64 +629,20 @@ bool make_pool_map(CUtensorMap* map, const void* pool, long long num_pages, int 
     return make_pool_map_impl(map, pool, num_pages, hkv);
 }
 
-namespace {
-cudaError_t configure_tile_kernel() {
+cudaError_t launch_attn_tile_bf16(const AttnParams& p, cudaStream_t stream) {
+    if (p.num_items == 0) return cudaSuccess;
+    if ((long long)p.num_pages * p.hkv * kPage > 0x7FFFFFFFll) return cudaErrorInvalidValue;
+    alignas(64) CUtensorMap map_k, map_v;
+    if (!make_pool_map(&map_k, p.k_pool, p.num_pages, p.hkv) || !make_pool_map(&map_v, p.v_pool, p.num_pages, p.hkv))
+        return cudaErrorNotSupported;
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(attn_tile_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    return cudaSuccess;
-}
-void fill_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int grid, int cluster, cudaStream_t stream) {
-    cfg = cudaLaunchConfig_t{};
-    cfg.gridDim = dim3((unsigned)grid, 1, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = kSmemBytes;
-    cfg.stream = stream;
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)cluster;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-}
-}  // namespace
-
-// CTAs of the tile kernel that can be resident at once when launched in clusters of `cluster` (1..8);
-// 0 when such clusters cannot be placed.  Cached per cluster size (one device per process is assumed).
-int attn_tile_resident_ctas(int cluster) {
-    static int cache[kMaxTileCluster + 1] = {0};
-    static bool known[kMaxTileCluster + 1] = {false};
-    if (cluster < 1 || cluster > kMaxTileCluster) return 0;
-    if (!known[cluster]) {
-        int n = 0;
-        if (configure_tile_kernel() == cudaSuccess) {
-            cudaLaunchConfig_t cfg;
-            cudaLaunchAttribute attr[1];
-            fill_launch_config(cfg, attr, cluster, cluster, nullptr);
-            if (cudaOccupancyMaxActiveClusters(&n, attn_tile_bf16_kernel, &cfg) != cudaSuccess) { n = 0; (void)cudaGetLastError(); }
-        }
-        cache[cluster] = n * cluster;
-        known[cluster] = true;
-    }
-    return cache[cluster];
-}
-
-cudaError_t launch_attn_tile_bf16(const AttnParams& p, int cluster, cudaStream_t stream) {
-    if (p.num_items == 0) return cudaSuccess;
-    if (cluster < 1 || cluster > kMaxTileCluster || p.num_items % cluster != 0) return cudaErrorInvalidValue;
-    if ((long long)p.num_pages * p.hkv * kPage > 0x7FFFFFFFll) return cudaErrorInvalidValue;
-    alignas(64) CUtensorMap map_k, map_v;
-    if (!make_pool_map(&map_k, p.k_pool, p.num_pages, p.hkv) || !make_pool_map(&map_v, p.v_pool, p.num_pages, p.hkv))
-        return cudaErrorNotSupported;
-    cudaError_t e = configure_tile_kernel();
-    if (e != cudaSuccess) return e;
-    cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
-    fill_launch_config(cfg, attr, p.num_items, cluster, stream);
-    return cudaLaunchKernelEx(&cfg, attn_tile_bf16_kernel, p, map_k, map_v);
+    attn_tile_bf16_kernel<<<p.num_items, kThreads, kSmemBytes, stream>>>(p, map_k, map_v);
+    return cudaGetLastError();
 }
 
 }  // namespace agx

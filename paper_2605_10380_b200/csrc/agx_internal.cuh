@@ -59,12 +59,8 @@ cudaError_t launch_attn_simt_f32(const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, cudaStream_t stream);
 
 bool attn_tile_available();
-// Large-q tensor-core tile kernel (bf16, d = 128, tcgen05 + TMEM + TMA).  The KV splits of one
-// (sequence, KV head, row chunk) form a thread-block cluster of `cluster` CTAs that merges its partial
-// results through distributed shared memory: every sequence of the launch has nsplit == cluster.
-constexpr int kMaxTileCluster = 8;
-cudaError_t launch_attn_tile_bf16(const AttnParams& p, int cluster, cudaStream_t stream);
-int attn_tile_resident_ctas(int cluster);
+// Large-q tensor-core tile kernel (bf16, d = 128, tcgen05 + TMEM + TMA).
+cudaError_t launch_attn_tile_bf16(const AttnParams& p, cudaStream_t stream);
 
 cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_stride, int vocab, const int* drafts,
                           const int* cu_q, int B, int total_q, int* accept_len, int* next_token, int* argmax,
