@@ -21,6 +21,7 @@ struct agx_handle {
     int small_min_split;    // tokens; tuning knob (env AGX_SMALL_MIN_SPLIT)
     int force_mma_sync;     // route large q through the mma.sync kernel (env AGX_FORCE_MMA_SYNC)
     int debug_plan;         // print launch plans to stderr (env AGX_DEBUG_PLAN)
+    int stream_min_tokens;  // context length from which blocks of <= 64 rows take the tensor-core stream schedule (env AGX_STREAM_MIN_TOKENS)
     std::vector<int32_t> cu_host;  // staging for agx_verify_step_host (lives until its final sync)
     char err[512];
 };
@@ -47,7 +48,7 @@ inline bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 inline int round_up(long long v, int m) { return (int)((v + m - 1) / m * m); }
 inline int elem_size(int dtype) { return dtype == AGX_BF16 ? 2 : 4; }
 
-enum Kind { KIND_SMALL1 = 0, KIND_SMALL2, KIND_SMALL4, KIND_TILE, KIND_SIMT, KIND_COUNT };
+enum Kind { KIND_SMALL1 = 0, KIND_SMALL2, KIND_SMALL4, KIND_STREAM, KIND_TILE, KIND_SIMT, KIND_COUNT };
 
 struct Launch {
     Kind kind;
@@ -81,7 +82,11 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
         if (c.dtype == AGX_F32) k = KIND_SIMT;
         else {
             const int rows = Q[s] * G;
-            if (rows <= 16) k = KIND_SMALL1;
+            const bool tile_ok = !h->force_mma_sync && attn_tile_available();
+            // up to 128 rows over a long context: one Q tile per CTA, KV tiles alternating between two softmax
+            // warpgroups (HBM-bound streaming on the tcgen05 pipe); short contexts stay with the warp-MMA kernel
+            if (tile_ok && rows <= 128 && (rows > kSmallRowsMax || P[s] + Q[s] >= h->stream_min_tokens)) k = KIND_STREAM;
+            else if (rows <= 16) k = KIND_SMALL1;
             else if (rows <= 32) k = KIND_SMALL2;
             else if (rows <= kSmallRowsMax || h->force_mma_sync || !attn_tile_available()) k = KIND_SMALL4;
             else k = KIND_TILE;
@@ -96,9 +101,9 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
         long long base_items = 0;  // items per split, summed over sequences
         std::vector<long long> per_seq_items(seqs.size());
         if (k == KIND_SIMT) { unit = 64; min_split = 256; target = h->sm_count * 16; }
-        else if (k == KIND_TILE) { unit = 128; min_split = 512; target = h->sm_count; }
+        else if (k == KIND_TILE || k == KIND_STREAM) { unit = 128; min_split = k == KIND_TILE ? 512 : 256; target = h->sm_count; }
         else { unit = 64; min_split = h->small_min_split; target = h->sm_count * (k == KIND_SMALL4 ? 1 : 2); }
-        const int rows_per_chunk = (k == KIND_SMALL1) ? 16 : (k == KIND_SMALL2) ? 32 : (k == KIND_SMALL4) ? 64 : 256;
+        const int rows_per_chunk = (k == KIND_SMALL1) ? 16 : (k == KIND_SMALL2) ? 32 : (k == KIND_SMALL4) ? 64 : (k == KIND_STREAM) ? 128 : 256;
         long long work = 0;
         for (size_t n = 0; n < seqs.size(); ++n) {
             const int s = seqs[n];
@@ -118,7 +123,7 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
             }
             return items;
         };
-        if (k == KIND_TILE) {
+        if (k == KIND_TILE || k == KIND_STREAM) {
             // several waves are fine here: pick the split length with the smallest estimated makespan,
             // waves * (tiles per item + fixed per-CTA cost of ~3 tiles)
             int max_len = 0;
@@ -214,6 +219,8 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     h->small_min_split = env ? std::max(64, atoi(env) / 64 * 64) : 256;
     env = getenv("AGX_FORCE_MMA_SYNC");
     h->force_mma_sync = env ? atoi(env) : 0;
+    env = getenv("AGX_STREAM_MIN_TOKENS");
+    h->stream_min_tokens = env ? atoi(env) : 8192;
     env = getenv("AGX_DEBUG_PLAN");
     h->debug_plan = env ? atoi(env) : 0;
     cudaError_t e = cudaGetDevice(&h->device);
@@ -313,7 +320,8 @@ agx_status agx_attn_prefixed(agx_handle* h, const void* q_block, const void* k_p
             case KIND_SMALL2: e = launch_attn_small_bf16(p, 2, stream); break;
             case KIND_SMALL4: e = launch_attn_small_bf16(p, 4, stream); break;
             case KIND_SIMT: e = launch_attn_simt_f32(p, stream); break;
-            case KIND_TILE: e = launch_attn_tile_bf16(p, stream); break;
+            case KIND_TILE: e = launch_attn_tile_bf16(p, false, stream); break;
+            case KIND_STREAM: e = launch_attn_tile_bf16(p, true, stream); break;
             default: return fail(h, AGX_E_UNSUPPORTED, "unknown kernel kind");
         }
         if (e != cudaSuccess) return cuda_fail(h, e, "attention launch");

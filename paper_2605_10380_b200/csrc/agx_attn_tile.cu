@@ -34,16 +34,28 @@ namespace {
 
 constexpr int kD = 128;
 constexpr int kBN = 128;                    // KV tokens per tile
-constexpr int kRowsPerCta = 256;
 constexpr int kStagesK = 3;                 // K is wanted right after the previous tile's softmax: one more stage
-constexpr int kStagesV = 2;
+// Two schedules share the kernel (template parameter kStreams):
+//   false  two 128-row Q tiles A and B per CTA (256 rows), both meet every KV tile;
+//   true   ONE 128-row Q tile per CTA (verify blocks and short suffixes: q * G <= 128 rows, most of them
+//          padding); the two softmax warpgroups take the even and the odd KV tiles of the same rows, each with
+//          its own S and O accumulators in TMEM, and are merged inside the CTA at the end.  The step is
+//          HBM-bound, so the padded MMA rows cost nothing that matters, while every K/V byte is read once
+//          and the softmax of one tile hides behind the MMAs and copies of the next.
+template <bool kStreams> struct Sched {
+    static constexpr int kRows = kStreams ? 128 : 256;     // query rows per CTA
+    static constexpr int kStagesV = kStreams ? 3 : 2;      // the second Q tile's shared memory becomes a V stage
+};
 constexpr int kThreads = 384;
 constexpr uint32_t kTileBytes = 128 * 256;  // one operand tile: [2 halves of 64 dims][128 rows][128 B]
 constexpr uint32_t kHalfBytes = 128 * 128;
 constexpr uint32_t kOffQ = 0;
 constexpr uint32_t kOffK = 2 * kTileBytes;
 constexpr uint32_t kOffV = kOffK + kStagesK * kTileBytes;
-constexpr uint32_t kOffBar = kOffV + kStagesV * kTileBytes;
+constexpr uint32_t kOffBar = kOffV + 2 * kTileBytes;
+// V stage s: the first two behind the K ring, the third (kStreams only) in the unused second Q tile
+__host__ __device__ constexpr uint32_t v_stage_off(int s) { return s < 2 ? kOffV + s * kTileBytes : kOffQ + kTileBytes; }
+constexpr uint32_t kOffPark = kOffK + 2 * kTileBytes;   // kStreams epilogue: stream 1's O rows (64 KB), then its (m, l)
 constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // + barriers + alignment slack
 constexpr float kRescaleThreshold = 8.0f;              // log2 units
 // Of every 8 column pairs, this many take the polynomial 2^x instead of the special-function unit.
@@ -56,8 +68,8 @@ constexpr float kRescaleThreshold = 8.0f;              // log2 units
 constexpr int kPolyPairsOf8 = AGX_POLY_PAIRS;
 
 // barrier slots (8 bytes each)
-enum { BAR_K_FULL = 0, BAR_K_EMPTY = 3, BAR_V_FULL = 6, BAR_V_EMPTY = 8, BAR_S_FULL = 10, BAR_P_READY = 12,
-       BAR_O_FULL = 14, BAR_Q_FULL = 15, BAR_COUNT = 16 };
+enum { BAR_K_FULL = 0, BAR_K_EMPTY = 3, BAR_V_FULL = 6, BAR_V_EMPTY = 9, BAR_S_FULL = 12, BAR_P_READY = 14,
+       BAR_O_FULL = 16, BAR_Q_FULL = 17, BAR_COUNT = 18 };
 constexpr int kQLoadThreads = kThreads - 64;  // warps 2..11 bring the Q tiles in
 constexpr int kRegsLow = 96, kRegsHigh = 200; // 128 * 96 + 256 * 200 <= 384 * 168
 
@@ -174,7 +186,9 @@ __device__ __forceinline__ int find_seq(const AttnParams& p, int item) {
 struct TileItem {
     int g, G, P, q, rows, row0, split, nsplit, n_tiles, kv_begin, kv_end, vis_end, q_row0, seq_index;
 };
+template <bool kStreams>
 __device__ __forceinline__ TileItem locate_item(const AttnParams& p, int block) {
+    constexpr int kRowsPerCta = Sched<kStreams>::kRows;
     const int si = find_seq(p, block);
     const SeqPlan& sp = p.seq[si];
     TileItem it;
@@ -201,9 +215,39 @@ __device__ __forceinline__ TileItem locate_item(const AttnParams& p, int block) 
 // KV split the rows are normalised and written as bf16; otherwise fp32 partials and (m, l) go to the
 // workspace for the combine kernel.  Kept out of line, and re-deriving its indices from the block index,
 // so that nothing but its few arguments has to stay alive across the register-hungry main loop.
-__device__ __noinline__ void tile_epilogue(const AttnParams& p, unsigned char* smem, uint32_t tO, float m_ref, float l_run) {
+template <bool kStreams>
+__device__ __noinline__ void tile_epilogue(const AttnParams& p, unsigned char* smem, uint32_t tO, float m_ref, float l_run, bool ok) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const TileItem it = locate_item(p, blockIdx.x);
+    const TileItem it = locate_item<kStreams>(p, blockIdx.x);
+    float w_own = 1.f, w_other = 0.f;   // kStreams: weights of the two streams' accumulators
+    if (kStreams) {
+        // Stream 1 (warps 8-11) parks its rows in shared memory; stream 0 (warps 4-7) adds them to its own.
+        const int rt = ((warp & 3) << 5) + lane;
+        unsigned char* park = smem + kOffPark + rt * 512;
+        float2* park_ml = (float2*)(smem + kOffPark + 128 * 512);
+        if (warp >= 8 && ok) {
+            tc_fence_after();
+            uint32_t oreg[32];
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+                tmem_ld_x32(tO + c4 * 32, oreg);
+                tmem_wait_ld();
+#pragma unroll
+                for (int v = 0; v < 8; ++v)
+                    *(uint4*)(park + (((c4 * 8 + v) ^ lane) << 4)) = make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
+            }
+            park_ml[rt] = make_float2(m_ref, l_run);
+        }
+        // every softmax thread reaches this barrier, also after a bounded wait gave up somewhere in the CTA
+        asm volatile("bar.sync 1, 256;\n" ::: "memory");
+        if (warp >= 8 || !ok || *(volatile int*)(smem + kOffBar + BAR_COUNT * 8)) return;
+        const float2 other = park_ml[rt];
+        const float m_new = fmaxf(m_ref, other.x);
+        w_own = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_new);
+        w_other = (other.x == -INFINITY) ? 0.f : ex2(other.x - m_new);
+        l_run = l_run * w_own + other.y * w_other;
+        m_ref = m_new;
+    }
     const SeqPlan& sp = p.seq[find_seq(p, blockIdx.x)];
     unsigned char* stage = smem + kOffK + (warp - 4) * 16384;    // [32 rows][512 B], 16-byte units XOR-swizzled by row
     const int r_warp0 = it.row0 + (warp - 4) * 32;               // first row of this warp
@@ -217,6 +261,17 @@ __device__ __noinline__ void tile_epilogue(const AttnParams& p, unsigned char* s
         for (int c4 = 0; c4 < 4; ++c4) {
             tmem_ld_x32(tO + c4 * 32, oreg);
             tmem_wait_ld();
+            if (kStreams) {
+                const unsigned char* park = smem + kOffPark + ((((warp & 3) << 5) + lane) * 512);
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                    const float4 o1 = *(const float4*)(park + (((c4 * 8 + v) ^ lane) << 4));
+                    oreg[4 * v + 0] = __float_as_uint(__uint_as_float(oreg[4 * v + 0]) * w_own + (w_other != 0.f ? o1.x * w_other : 0.f));
+                    oreg[4 * v + 1] = __float_as_uint(__uint_as_float(oreg[4 * v + 1]) * w_own + (w_other != 0.f ? o1.y * w_other : 0.f));
+                    oreg[4 * v + 2] = __float_as_uint(__uint_as_float(oreg[4 * v + 2]) * w_own + (w_other != 0.f ? o1.z * w_other : 0.f));
+                    oreg[4 * v + 3] = __float_as_uint(__uint_as_float(oreg[4 * v + 3]) * w_own + (w_other != 0.f ? o1.w * w_other : 0.f));
+                }
+            }
             if (single) {
 #pragma unroll
                 for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * inv);
@@ -259,6 +314,7 @@ __device__ __noinline__ void tile_epilogue(const AttnParams& p, unsigned char* s
 
 }  // namespace
 
+template <bool kStreams>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtensorMap map_k,
                       const __grid_constant__ CUtensorMap map_v) {
@@ -271,8 +327,10 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+    constexpr int kRowsPerCta = Sched<kStreams>::kRows;
+    constexpr int kStagesV = Sched<kStreams>::kStagesV;
     // ---- work item
-    const TileItem it = locate_item(p, blockIdx.x);
+    const TileItem it = locate_item<kStreams>(p, blockIdx.x);
     const SeqPlan& sp = p.seq[find_seq(p, blockIdx.x)];
     const int split = it.split, g = it.g, G = it.G, P = it.P, q = it.q, L = P + q, rows = it.rows, row0 = it.row0;
     const int kv_begin = it.kv_begin, kv_end = it.kv_end, n_tiles = it.n_tiles;
@@ -304,7 +362,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
     // Q: 256 rows x 256 B by 16-byte cp.async (all of a thread's copies in flight at once), written in
     // the 128-byte-swizzled K-major operand layout; rows past q * G are zero-filled.
     if (warp >= 2) {
-        for (int c = tid - 64; c < kRowsPerCta * 16; c += kQLoadThreads) {
+        for (int c = tid - 64; c < kRowsPerCta * 16; c += kQLoadThreads) {   // kStreams: one tile
             const int rl = c >> 4, ch = c & 15;     // row in chunk, 16-byte chunk of the 256-byte row
             const int r = row0 + rl;
             const bool valid = r < rows;
@@ -376,7 +434,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                     const int r = idx >> 4, ch = idx & 15, half = ch >> 3, u = ch & 7;
                     uint4 v = make_uint4(0, 0, 0, 0);
                     if (r < valid_rows) v = __ldg((const uint4*)(src + r * 256 + ch * 16));
-                    *(uint4*)(smem + kOffV + vs * kTileBytes + half * kHalfBytes + ragged_pg * 2048 + r * 128 + ((u ^ (r & 7)) << 4)) = v;
+                    *(uint4*)(smem + v_stage_off(vs) + half * kHalfBytes + ragged_pg * 2048 + r * 128 + ((u ^ (r & 7)) << 4)) = v;
                 }
                 asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
                 __syncwarp();
@@ -384,7 +442,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             if (lane == 0) mbar_arrive_expect_tx(bar(BAR_V_FULL + vs), (npg - (ragged_pg >= 0 ? 1 : 0)) * 4096u);
             __syncwarp();
             if (mine && pg != ragged_pg) {
-                const uint32_t dst = smem_base + kOffV + vs * kTileBytes + pg * 2048;
+                const uint32_t dst = smem_base + v_stage_off(vs) + pg * 2048;
                 tma_load_2d(dst, &map_v, 0, y, bar(BAR_V_FULL + vs));
                 tma_load_2d(dst + kHalfBytes, &map_v, 64, y, bar(BAR_V_FULL + vs));
             }
@@ -404,17 +462,16 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             // descriptors differ only in the start address: add (byte offset >> 4) to a base descriptor
             const uint64_t q_desc[2] = {make_desc(smem_base + kOffQ, 16, 1024), make_desc(smem_base + kOffQ + kTileBytes, 16, 1024)};
             const uint64_t k_desc0 = make_desc(smem_base + kOffK, 16, 1024);
-            const uint64_t v_desc0 = make_desc(smem_base + kOffV, kHalfBytes, 1024);
-            auto issue_qk = [&](int x, int stage) {   // S_x = Q_x K^T : 8 k-steps of 16 dims
+            auto issue_qk = [&](int qt, int stage, int x) {   // S_x = Q_qt K^T : 8 k-steps of 16 dims
                 const uint64_t kd = k_desc0 + (uint64_t)((stage * kTileBytes) >> 4);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint64_t off = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
-                    umma_ss(tS[x], q_desc[x] + off, kd + off, kIdescQK, ks > 0);
+                    umma_ss(tS[x], q_desc[qt] + off, kd + off, kIdescQK, ks > 0);
                 }
             };
             auto issue_pv = [&](int x, int stage, int npg, bool first) {  // O_x += P_x V : one k-step per page
-                const uint64_t vd = v_desc0 + (uint64_t)((stage * kTileBytes) >> 4);
+                const uint64_t vd = make_desc(smem_base + v_stage_off(stage), kHalfBytes, 1024);
                 if (npg == 8) {
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
@@ -425,11 +482,39 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                 }
             };
             bool ok = mbar_wait(bar(BAR_Q_FULL), 0, abort_flag, p.status);
+            if (kStreams) {
+                // stream x = t & 1 owns KV tile t:  S_0(0) S_1(1) | O_x += P_x V(t), S_x(t + 2) | ...
+                for (int t = 0; t < 2 && t < n_tiles && ok; ++t) {
+                    ok = mbar_wait(bar(BAR_K_FULL + t), 0, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(0, t, t); umma_commit(bar(BAR_S_FULL + t));
+                    umma_commit(bar(BAR_K_EMPTY + t));
+                }
+                for (int t = 0; t < n_tiles && ok; ++t) {
+                    const int x = t & 1, vs = t % kStagesV, vph = (t / kStagesV) & 1, npg = pages_in_tile(t);
+                    ok = mbar_wait(bar(BAR_V_FULL + vs), vph, abort_flag, p.status);
+                    if (!ok) break;
+                    ok = mbar_wait(bar(BAR_P_READY + x), (t >> 1) & 1, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(x, vs, npg, t < 2);
+                    umma_commit(bar(BAR_V_EMPTY + vs));
+                    if (t + 2 < n_tiles) {
+                        const int nks = (t + 2) % kStagesK, nkph = ((t + 2) / kStagesK) & 1;
+                        ok = mbar_wait(bar(BAR_K_FULL + nks), nkph, abort_flag, p.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_qk(0, nks, x); umma_commit(bar(BAR_S_FULL + x));
+                        umma_commit(bar(BAR_K_EMPTY + nks));
+                    }
+                }
+            } else {
             if (ok) ok = mbar_wait(bar(BAR_K_FULL + 0), 0, abort_flag, p.status);
             if (ok) {
                 tc_fence_after();
-                issue_qk(0, 0); umma_commit(bar(BAR_S_FULL + 0));
-                issue_qk(1, 0); umma_commit(bar(BAR_S_FULL + 1));
+                issue_qk(0, 0, 0); umma_commit(bar(BAR_S_FULL + 0));
+                issue_qk(1, 0, 1); umma_commit(bar(BAR_S_FULL + 1));
                 umma_commit(bar(BAR_K_EMPTY + 0));
             }
             for (int t = 0; t < n_tiles && ok; ++t) {
@@ -446,7 +531,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                     ok = mbar_wait(bar(BAR_K_FULL + nks), nkph, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_qk(0, nks); umma_commit(bar(BAR_S_FULL + 0));
+                    issue_qk(0, nks, 0); umma_commit(bar(BAR_S_FULL + 0));
                 }
                 ok = mbar_wait(bar(BAR_P_READY + 1), t & 1, abort_flag, p.status);
                 if (!ok) break;
@@ -454,9 +539,10 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                 issue_pv(1, vs, npg, t == 0);
                 umma_commit(bar(BAR_V_EMPTY + vs));
                 if (more) {
-                    issue_qk(1, nks); umma_commit(bar(BAR_S_FULL + 1));
+                    issue_qk(1, nks, 1); umma_commit(bar(BAR_S_FULL + 1));
                     umma_commit(bar(BAR_K_EMPTY + nks));
                 }
+            }
             }
             umma_commit(bar(BAR_O_FULL));  // arrives when every MMA issued above has completed
             mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
@@ -471,16 +557,21 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
         const uint32_t tS = tmem_base + lane_addr + kColS + x * 128;
         const uint32_t tO = tmem_base + lane_addr + kColO + x * 128;
-        const int r = row0 + x * 128 + rt;
+        const int q_tile_row0 = row0 + (kStreams ? 0 : x * 128);   // kStreams: both warpgroups hold the same rows
+        const int r = q_tile_row0 + rt;
         const int limit = P + min(r / G, q - 1);             // last token this row sees
-        const int tile_i_min = min((row0 + x * 128) / G, q - 1);
+        const int tile_i_min = min(q_tile_row0 / G, q - 1);
+        // a warp whose 32 rows are all padding only keeps the barriers in step
+        const bool warp_has_rows = q_tile_row0 + ((warp & 3) << 5) < rows;
         const float sc = p.scale_log2;
         float m_ref = -INFINITY;
         float l_run = 0.f;                                   // running row sum, relative to m_ref
         bool ok = true;
-        for (int t = 0; t < n_tiles; ++t) {
-            ok = mbar_wait(bar(BAR_S_FULL + x), t & 1, abort_flag, p.status);
+        for (int t = kStreams ? x : 0; t < n_tiles; t += kStreams ? 2 : 1) {
+            const int j = kStreams ? (t >> 1) : t;           // this warpgroup's j-th tile
+            ok = mbar_wait(bar(BAR_S_FULL + x), j & 1, abort_flag, p.status);
             if (!ok) break;
+            if (!warp_has_rows) { mbar_arrive(bar(BAR_P_READY + x)); continue; }
             tc_fence_after();
             uint32_t sreg[128];
 #pragma unroll
@@ -491,7 +582,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             const uint64_t sc2 = pk2(sc, sc);
             float lt0 = 0.f, lt1 = 0.f, lt2 = 0.f, lt3 = 0.f;   // this tile's row sum, four partial sums
             bool done = false;
-            if (t > 0 && !masked) {
+            if (j > 0 && !masked) {
                 // ---- common case, one sweep: exponentials against the running reference m_ref (the
                 //      maximum of earlier tiles, so P may exceed 1) while the tile's own maximum is
                 //      collected on the side; only if that maximum tops m_ref by more than 2^8 is the
@@ -545,7 +636,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                 if (__any_sync(0xFFFFFFFFu, need)) {
                     const float m_new = need ? m_tile : m_ref;
                     const float factor = need ? ex2(m_ref - m_new) : 1.f;   // m_ref = -inf gives 0
-                    if (t > 0) {
+                    if (j > 0) {
                         uint32_t oreg[32];
 #pragma unroll
                         for (int c4 = 0; c4 < 4; ++c4) {
@@ -582,7 +673,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             mbar_arrive(bar(BAR_P_READY + x));
         }
         if (ok) ok = mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
-        if (ok) tile_epilogue(p, smem, tO, m_ref, l_run);
+        if (ok || kStreams) tile_epilogue<kStreams>(p, smem, tO, m_ref, l_run, ok);
     }
     // ---- teardown
     tc_fence_before();
@@ -629,20 +720,27 @@ bool make_pool_map(CUtensorMap* map, const void* pool, long long num_pages, int 
     return make_pool_map_impl(map, pool, num_pages, hkv);
 }
 
-cudaError_t launch_attn_tile_bf16(const AttnParams& p, cudaStream_t stream) {
+namespace {
+template <bool kStreams>
+cudaError_t launch_tile(const AttnParams& p, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(attn_tile_bf16_kernel<kStreams>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    attn_tile_bf16_kernel<kStreams><<<p.num_items, kThreads, kSmemBytes, stream>>>(p, map_k, map_v);
+    return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t launch_attn_tile_bf16(const AttnParams& p, bool streams, cudaStream_t stream) {
     if (p.num_items == 0) return cudaSuccess;
     if ((long long)p.num_pages * p.hkv * kPage > 0x7FFFFFFFll) return cudaErrorInvalidValue;
     alignas(64) CUtensorMap map_k, map_v;
     if (!make_pool_map(&map_k, p.k_pool, p.num_pages, p.hkv) || !make_pool_map(&map_v, p.v_pool, p.num_pages, p.hkv))
         return cudaErrorNotSupported;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tile_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
-    attn_tile_bf16_kernel<<<p.num_items, kThreads, kSmemBytes, stream>>>(p, map_k, map_v);
-    return cudaGetLastError();
+    return streams ? launch_tile<true>(p, map_k, map_v, stream) : launch_tile<false>(p, map_k, map_v, stream);
 }
 
 }  // namespace agx

@@ -59,8 +59,10 @@ cudaError_t launch_attn_simt_f32(const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, cudaStream_t stream);
 
 bool attn_tile_available();
-// Large-q tensor-core tile kernel (bf16, d = 128, tcgen05 + TMEM + TMA).
-cudaError_t launch_attn_tile_bf16(const AttnParams& p, cudaStream_t stream);
+// Tensor-core tile kernel (bf16, d = 128, tcgen05 + TMEM + TMA).  streams = false: 256 query rows per CTA
+// (two Q tiles); streams = true: 128 rows per CTA whose KV tiles alternate between two softmax warpgroups
+// (verify blocks and short suffixes over long contexts).
+cudaError_t launch_attn_tile_bf16(const AttnParams& p, bool streams, cudaStream_t stream);
 
 cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_stride, int vocab, const int* drafts,
                           const int* cu_q, int B, int total_q, int* accept_len, int* next_token, int* argmax,

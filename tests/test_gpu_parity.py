@@ -262,6 +262,33 @@ def test_argument_errors_are_reported_not_faulted():
     assert e.value.status == -1
 
 
+# ------------------------------------------------------------------ tensor-core stream schedule (few rows, long context)
+@pytest.mark.parametrize("P,q,hq,hkv", [
+    (0, 1, 32, 8), (1, 1, 32, 8), (15, 1, 8, 8), (17, 4, 32, 8), (127, 8, 32, 8), (128, 8, 32, 8), (129, 16, 32, 8),
+    (255, 2, 32, 8), (1000, 3, 24, 8), (2049, 5, 32, 8), (5000, 8, 32, 8), (777, 32, 32, 8), (300, 7, 4, 1),
+    (130, 100, 4, 4), (4095, 2, 16, 2), (20000, 8, 32, 8), (9000, 25, 32, 8),
+])
+def test_stream_schedule_shapes(P, q, hq, hkv, monkeypatch):
+    """Blocks of at most 128 query rows per KV head on the tcgen05 kernel whose two softmax warpgroups
+    alternate KV tiles; forced here for every context length."""
+    monkeypatch.setenv("AGX_STREAM_MIN_TOKENS", "0")
+    w = W.make_attn_workload(f"stream_{P}_{q}", 3000 + P + q, "bf16", hq, hkv, 128, [P], [q], spare_pages=3)
+    run_and_check(w, sample=(13, 64) if P > 6000 else None, poison=True)
+
+
+def test_stream_schedule_ragged_batch_matches_warp_mma_kernel(monkeypatch):
+    P = [2048, 2100, 4000, 2048 + 15, 9000, 2500, 3001, 2048]
+    q = [1, 2, 4, 8, 16, 3, 5, 30]
+    w = W.make_attn_workload("ragged_stream", 43, "bf16", 32, 8, 128, P, q, shared_prefix_tokens=2048)
+    monkeypatch.setenv("AGX_STREAM_MIN_TOKENS", "0")
+    b = DeviceBatch(w); b.append(); a, _ = b.attend()
+    monkeypatch.setenv("AGX_STREAM_MIN_TOKENS", "100000000")
+    b2 = DeviceBatch(w); b2.append(); c, _ = b2.attend()
+    assert b.status() == 0 and b2.status() == 0
+    assert np.max(np.abs(a - c)) < 2e-2
+    run_and_check(w, sample=(7, 12))
+
+
 # ------------------------------------------------------------------ tensor-core tile kernel (large q)
 @pytest.mark.parametrize("P,q,hq,hkv", [
     (0, 128, 8, 2),        # pure causal prefill, G = 4, one tile pair, exact multiples
