@@ -230,9 +230,14 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
             }
 
             // S = Q K^T for 16 tokens: two n-tiles of 8 tokens
-            float s[2][4];
+            // four accumulation chains of four MMAs each (even and odd k-steps of both n-tiles) instead of two
+            // of eight: a dependent mma.sync is slow to issue, and this chain sits on every page's critical path
+            float s[2][4], s_odd[2][4];
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt) { s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f; }
+            for (int nt = 0; nt < 2; ++nt) {
+                s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+                s_odd[nt][0] = s_odd[nt][1] = s_odd[nt][2] = s_odd[nt][3] = 0.f;
+            }
 #pragma unroll
             for (int kp = 0; kp < 4; ++kp) {
 #pragma unroll
@@ -240,8 +245,13 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
                     uint32_t b0, b1, b2, b3;
                     ldmatrix_x4(b0, b1, b2, b3, k_base + (kp >> 1) * 2048 + nt * 1024 + k_off[kp & 1]);
                     mma_bf16(s[nt], qa[2 * kp], b0, b1);
-                    mma_bf16(s[nt], qa[2 * kp + 1], b2, b3);
+                    mma_bf16(s_odd[nt], qa[2 * kp + 1], b2, b3);
                 }
+            }
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) s[nt][e] += s_odd[nt][e];
             }
             // mask the causal edge / the end of the split (raw scores; the scale is folded into the exp)
             if ((tok0 + kPage - 1 > P) || (tok0 + kPage > tok_end)) {
@@ -459,45 +469,79 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
     const int i = lrow - acc_rows;
     const long long e0 = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit;
     const int ns = sp.nsplit;
-    // pass 1: lanes take splits side by side (independent loads), then warp reductions in fixed order
-    float m_all = -INFINITY;
-    for (int k = lane; k < ns; k += 32) m_all = fmaxf(m_all, p.part_ml[e0 + k].x);
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, off));
-    float l_all = 0.f;
-    for (int k = lane; k < ns; k += 32) {
-        const float2 ml = p.part_ml[e0 + k];
-        l_all += (ml.x == -INFINITY) ? 0.f : ml.y * exp2f(ml.x - m_all);
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xFFFFFFFFu, l_all, off);
-    // pass 2: each lane owns 4 output columns; 4 splits' loads are in flight together
     const int D = p.head_dim;
+    const int c4 = lane * 4;               // each lane owns 4 output columns
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    const int c4 = lane * 4;
-    if (c4 < D) {
-        int k = 0;
-        for (; k + 4 <= ns; k += 4) {
-            float w[4];
-            float4 v[4];
+    float m_all, l_all;
+    if (ns <= 32) {
+        // One round trip to memory: lane k fetches (m, l) of split k while every lane already fetches its
+        // columns of up to 16 splits' O rows; the weights then travel by shuffle, splits in index order.
+        const float2 ml = (lane < ns) ? p.part_ml[e0 + lane] : make_float2(-INFINITY, 0.f);
+        float4 v[16];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float mk = p.part_ml[e0 + k + j].x;
-                w[j] = (mk == -INFINITY) ? 0.f : exp2f(mk - m_all);
-                v[j] = *(const float4*)(p.part_o + (e0 + k + j) * D + c4);
+        for (int j = 0; j < 16; ++j)
+            if (j < ns && c4 < D) v[j] = *(const float4*)(p.part_o + (e0 + j) * D + c4);
+        m_all = ml.x;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, off));
+        const float w_mine = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m_all);
+        l_all = ml.y * w_mine;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xFFFFFFFFu, l_all, off);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const float w = __shfl_sync(0xFFFFFFFFu, w_mine, j);
+            if (j < ns && w != 0.f && c4 < D) {   // a split that saw no token for this row publishes only (m, l) = (-inf, 0)
+                acc.x += v[j].x * w; acc.y += v[j].y * w; acc.z += v[j].z * w; acc.w += v[j].w * w;
             }
+        }
+        if (ns > 16) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (w[j] != 0.f) {   // a split that saw no token for this row publishes only (m, l) = (-inf, 0)
-                    acc.x += v[j].x * w[j]; acc.y += v[j].y * w[j]; acc.z += v[j].z * w[j]; acc.w += v[j].w * w[j];
+            for (int j = 0; j < 16; ++j)
+                if (16 + j < ns && c4 < D) v[j] = *(const float4*)(p.part_o + (e0 + 16 + j) * D + c4);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const float w = __shfl_sync(0xFFFFFFFFu, w_mine, 16 + j);
+                if (16 + j < ns && w != 0.f && c4 < D) {
+                    acc.x += v[j].x * w; acc.y += v[j].y * w; acc.z += v[j].z * w; acc.w += v[j].w * w;
                 }
             }
         }
-        for (; k < ns; ++k) {
-            const float mk = p.part_ml[e0 + k].x;
-            const float w = (mk == -INFINITY) ? 0.f : exp2f(mk - m_all);
-            const float4 v = *(const float4*)(p.part_o + (e0 + k) * D + c4);
-            if (w != 0.f) { acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w; }
+    } else {
+        // many splits: lanes take splits side by side for (m, l), then 4 O rows in flight at a time
+        m_all = -INFINITY;
+        for (int k = lane; k < ns; k += 32) m_all = fmaxf(m_all, p.part_ml[e0 + k].x);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, off));
+        l_all = 0.f;
+        for (int k = lane; k < ns; k += 32) {
+            const float2 ml = p.part_ml[e0 + k];
+            l_all += (ml.x == -INFINITY) ? 0.f : ml.y * exp2f(ml.x - m_all);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xFFFFFFFFu, l_all, off);
+        if (c4 < D) {
+            int k = 0;
+            for (; k + 4 <= ns; k += 4) {
+                float w[4];
+                float4 v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float mk = p.part_ml[e0 + k + j].x;
+                    w[j] = (mk == -INFINITY) ? 0.f : exp2f(mk - m_all);
+                    v[j] = *(const float4*)(p.part_o + (e0 + k + j) * D + c4);
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (w[j] != 0.f) { acc.x += v[j].x * w[j]; acc.y += v[j].y * w[j]; acc.z += v[j].z * w[j]; acc.w += v[j].w * w[j]; }
+                }
+            }
+            for (; k < ns; ++k) {
+                const float mk = p.part_ml[e0 + k].x;
+                const float w = (mk == -INFINITY) ? 0.f : exp2f(mk - m_all);
+                const float4 v = *(const float4*)(p.part_o + (e0 + k) * D + c4);
+                if (w != 0.f) { acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w; }
+            }
         }
     }
     const float inv = 1.f / l_all;
