@@ -56,7 +56,8 @@ constexpr uint32_t kOffBar = kOffV + 2 * kTileBytes;
 // V stage s: the first two behind the K ring, the third (kStreams only) in the unused second Q tile
 __host__ __device__ constexpr uint32_t v_stage_off(int s) { return s < 2 ? kOffV + s * kTileBytes : kOffQ + kTileBytes; }
 constexpr uint32_t kOffPark = kOffK + 2 * kTileBytes;   // kStreams epilogue: stream 1's O rows (64 KB), then its (m, l)
-constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // + barriers + alignment slack
+constexpr uint32_t kOffCtx = kOffBar + 256;            // what the epilogue needs to know, parked at kernel start
+constexpr uint32_t kSmemBytes = kOffBar + 512 + 1024;  // + barriers + epilogue context + alignment slack
 constexpr float kRescaleThreshold = 8.0f;              // log2 units
 // Of every 8 column pairs, this many take the polynomial 2^x instead of the special-function unit.
 // Measured on B200 (P = 30720, q = 2048): 0 -> 950 us, 1 -> 957, 2 -> 964, 4 -> 982: the extra FMA-pipe
@@ -186,6 +187,16 @@ __device__ __forceinline__ int find_seq(const AttnParams& p, int item) {
 struct TileItem {
     int g, G, P, q, rows, row0, split, nsplit, n_tiles, kv_begin, kv_end, vis_end, q_row0, seq_index;
 };
+// Everything the epilogue needs, kept in shared memory: kernel parameters reached through a pointer are
+// slow to read, and registers are too precious across the main loop.
+struct EpiCtx {
+    TileItem it;
+    int part_base, hq;
+    void* out;
+    float* part_o;
+    float2* part_ml;
+    float* lse;
+};
 template <bool kStreams>
 __device__ __forceinline__ TileItem locate_item(const AttnParams& p, int block) {
     constexpr int kRowsPerCta = Sched<kStreams>::kRows;
@@ -216,16 +227,18 @@ __device__ __forceinline__ TileItem locate_item(const AttnParams& p, int block) 
 // workspace for the combine kernel.  Kept out of line, and re-deriving its indices from the block index,
 // so that nothing but its few arguments has to stay alive across the register-hungry main loop.
 template <bool kStreams>
-__device__ __noinline__ void tile_epilogue(const AttnParams& p, unsigned char* smem, uint32_t tO, float m_ref, float l_run, bool ok) {
+__device__ __noinline__ void tile_epilogue(unsigned char* smem, uint32_t tO, float m_ref, float l_run, bool ok) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const TileItem it = locate_item<kStreams>(p, blockIdx.x);
+    const EpiCtx cx = *(const EpiCtx*)(smem + kOffCtx);
+    const TileItem& it = cx.it;
+    const bool warp_has_rows = it.row0 + ((warp & 3) << 5) + (kStreams ? 0 : ((warp - 4) >> 2) * 128) < it.rows;
     float w_own = 1.f, w_other = 0.f;   // kStreams: weights of the two streams' accumulators
     if (kStreams) {
         // Stream 1 (warps 8-11) parks its rows in shared memory; stream 0 (warps 4-7) adds them to its own.
         const int rt = ((warp & 3) << 5) + lane;
         unsigned char* park = smem + kOffPark + rt * 512;
         float2* park_ml = (float2*)(smem + kOffPark + 128 * 512);
-        if (warp >= 8 && ok) {
+        if (warp >= 8 && ok && warp_has_rows) {
             tc_fence_after();
             uint32_t oreg[32];
 #pragma unroll
@@ -240,7 +253,7 @@ __device__ __noinline__ void tile_epilogue(const AttnParams& p, unsigned char* s
         }
         // every softmax thread reaches this barrier, also after a bounded wait gave up somewhere in the CTA
         asm volatile("bar.sync 1, 256;\n" ::: "memory");
-        if (warp >= 8 || !ok || *(volatile int*)(smem + kOffBar + BAR_COUNT * 8)) return;
+        if (warp >= 8 || !ok || !warp_has_rows || *(volatile int*)(smem + kOffBar + BAR_COUNT * 8)) return;
         const float2 other = park_ml[rt];
         const float m_new = fmaxf(m_ref, other.x);
         w_own = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_new);
@@ -248,7 +261,7 @@ __device__ __noinline__ void tile_epilogue(const AttnParams& p, unsigned char* s
         l_run = l_run * w_own + other.y * w_other;
         m_ref = m_new;
     }
-    const SeqPlan& sp = p.seq[find_seq(p, blockIdx.x)];
+    if (!warp_has_rows) return;
     unsigned char* stage = smem + kOffK + (warp - 4) * 16384;    // [32 rows][512 B], 16-byte units XOR-swizzled by row
     const int r_warp0 = it.row0 + (warp - 4) * 32;               // first row of this warp
     const uint64_t magic = (0x100000000ull + it.G - 1) / it.G;   // (row * magic) >> 32 == row / G exactly for rows < 2^22
@@ -286,9 +299,9 @@ __device__ __noinline__ void tile_epilogue(const AttnParams& p, unsigned char* s
         if (r < it.rows) {
             const int i = (int)(((uint64_t)(uint32_t)r * magic) >> 32), h = it.g * it.G + (r - i * it.G);
             if (single) {
-                if (p.lse) p.lse[(long long)(it.q_row0 + i) * p.hq + h] = (m_ref + log2f(l_run)) * 0.6931471805599453f;
+                if (cx.lse) cx.lse[(long long)(it.q_row0 + i) * cx.hq + h] = (m_ref + log2f(l_run)) * 0.6931471805599453f;
             } else {
-                p.part_ml[(long long)sp.part_base + ((long long)i * p.hq + h) * it.nsplit + it.split] = make_float2(m_ref, l_run);
+                cx.part_ml[(long long)cx.part_base + ((long long)i * cx.hq + h) * it.nsplit + it.split] = make_float2(m_ref, l_run);
             }
         }
     }
@@ -304,10 +317,10 @@ __device__ __noinline__ void tile_epilogue(const AttnParams& p, unsigned char* s
             uint2 pk;
             pk.x = pack_bf16(__uint_as_float(v.x), __uint_as_float(v.y));
             pk.y = pack_bf16(__uint_as_float(v.z), __uint_as_float(v.w));
-            *(uint2*)((unsigned char*)p.out + (((long long)(it.q_row0 + io) * p.hq + ho) * 256 + lane * 8)) = pk;
+            *(uint2*)((unsigned char*)cx.out + (((long long)(it.q_row0 + io) * cx.hq + ho) * 256 + lane * 8)) = pk;
         } else {
-            const long long e = (long long)sp.part_base + ((long long)io * p.hq + ho) * it.nsplit + it.split;
-            *(uint4*)((unsigned char*)(p.part_o + e * kD) + lane * 16) = v;
+            const long long e = (long long)cx.part_base + ((long long)io * cx.hq + ho) * it.nsplit + it.split;
+            *(uint4*)((unsigned char*)(cx.part_o + e * kD) + lane * 16) = v;
         }
     }
 }
@@ -373,10 +386,13 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             cp_async_16(smem_base + kOffQ + tile * kTileBytes + half * kHalfBytes + rt * 128 + ((u ^ (rt & 7)) << 4), src, valid ? 16u : 0u);
         }
     }
+    // Barriers initialised, TMEM address published.  Warp 0 (which set the barriers up and needs nothing
+    // from the others) only signals and goes straight to the page table and its first K/V copies.
     tc_fence_before();
-    __syncthreads();   // barriers initialised, TMEM address published
+    if (warp == 0) { __syncwarp(); asm volatile("bar.arrive 2, %0;\n" ::"n"(kThreads) : "memory"); }
+    else asm volatile("bar.sync 2, %0;\n" ::"n"(kThreads) : "memory");
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_base = (warp == 0) ? 0u : *tmem_slot;
     if (warp >= 2) {
         asm volatile("cp.async.wait_all;\n" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
@@ -548,6 +564,11 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
         }
         __syncwarp();
+    } else if (tid == 32 * 3) {   // an otherwise idle warp parks the epilogue's context
+        EpiCtx* cx = (EpiCtx*)(smem + kOffCtx);
+        cx->it = locate_item<kStreams>(p, blockIdx.x);
+        cx->part_base = sp.part_base; cx->hq = p.hq;
+        cx->out = p.out; cx->part_o = p.part_o; cx->part_ml = p.part_ml; cx->lse = p.lse;
     }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsHigh));
@@ -567,11 +588,18 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         float m_ref = -INFINITY;
         float l_run = 0.f;                                   // running row sum, relative to m_ref
         bool ok = true;
-        for (int t = kStreams ? x : 0; t < n_tiles; t += kStreams ? 2 : 1) {
-            const int j = kStreams ? (t >> 1) : t;           // this warpgroup's j-th tile
+        constexpr int kStep = kStreams ? 2 : 1;
+        const int t_first = kStreams ? x : 0;
+        if (!warp_has_rows) {   // keep S_FULL / P_READY in step, nothing else
+            for (int t = t_first; t < n_tiles && ok; t += kStep) {
+                ok = mbar_wait(bar(BAR_S_FULL + x), ((t - t_first) / kStep) & 1, abort_flag, p.status);
+                if (ok) mbar_arrive(bar(BAR_P_READY + x));
+            }
+        } else
+        for (int t = t_first; t < n_tiles; t += kStep) {
+            const int j = (t - t_first) / kStep;             // this warpgroup's j-th tile
             ok = mbar_wait(bar(BAR_S_FULL + x), j & 1, abort_flag, p.status);
             if (!ok) break;
-            if (!warp_has_rows) { mbar_arrive(bar(BAR_P_READY + x)); continue; }
             tc_fence_after();
             uint32_t sreg[128];
 #pragma unroll
@@ -673,7 +701,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             mbar_arrive(bar(BAR_P_READY + x));
         }
         if (ok) ok = mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
-        if (ok || kStreams) tile_epilogue<kStreams>(p, smem, tO, m_ref, l_run, ok);
+        if (ok || kStreams) tile_epilogue<kStreams>(smem, tO, m_ref, l_run, ok);
     }
     // ---- teardown
     tc_fence_before();
