@@ -21,6 +21,7 @@ struct agx_handle {
     int small_min_split;    // tokens; tuning knob (env AGX_SMALL_MIN_SPLIT)
     int force_mma_sync;     // route large q through the mma.sync kernel (env AGX_FORCE_MMA_SYNC)
     int debug_plan;         // print launch plans to stderr (env AGX_DEBUG_PLAN)
+    int small_kw;           // pages per pipeline stage of the warp-MMA kernel, 4 or 8 (env AGX_SMALL_KW)
     int stream_min_tokens;  // context length from which blocks of <= 64 rows take the tensor-core stream schedule (env AGX_STREAM_MIN_TOKENS)
     std::vector<int32_t> cu_host;  // staging for agx_verify_step_host (lives until its final sync)
     char err[512];
@@ -102,7 +103,7 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
         std::vector<long long> per_seq_items(seqs.size());
         if (k == KIND_SIMT) { unit = 64; min_split = 256; target = h->sm_count * 16; }
         else if (k == KIND_TILE || k == KIND_STREAM) { unit = 128; min_split = k == KIND_TILE ? 512 : 256; target = h->sm_count; }
-        else { unit = 64; min_split = h->small_min_split; target = h->sm_count * (k == KIND_SMALL4 ? 1 : 2); }
+        else { unit = 64; min_split = h->small_min_split; target = h->sm_count * ((k == KIND_SMALL4 || h->small_kw == 8) ? 1 : 2); }
         const int rows_per_chunk = (k == KIND_SMALL1) ? 16 : (k == KIND_SMALL2) ? 32 : (k == KIND_SMALL4) ? 64 : (k == KIND_STREAM) ? 128 : 256;
         long long work = 0;
         for (size_t n = 0; n < seqs.size(); ++n) {
@@ -221,6 +222,8 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     h->force_mma_sync = env ? atoi(env) : 0;
     env = getenv("AGX_STREAM_MIN_TOKENS");
     h->stream_min_tokens = env ? atoi(env) : 8192;
+    env = getenv("AGX_SMALL_KW");
+    h->small_kw = (env && atoi(env) == 4) ? 4 : 8;
     env = getenv("AGX_DEBUG_PLAN");
     h->debug_plan = env ? atoi(env) : 0;
     cudaError_t e = cudaGetDevice(&h->device);
@@ -316,9 +319,9 @@ agx_status agx_attn_prefixed(agx_handle* h, const void* q_block, const void* k_p
         for (int i = 0; i < p.num_seqs; ++i) { p.seq[i] = ln.seqs[i]; split |= ln.seqs[i].nsplit > 1; }
         cudaError_t e;
         switch (ln.kind) {
-            case KIND_SMALL1: e = launch_attn_small_bf16(p, 1, stream); break;
-            case KIND_SMALL2: e = launch_attn_small_bf16(p, 2, stream); break;
-            case KIND_SMALL4: e = launch_attn_small_bf16(p, 4, stream); break;
+            case KIND_SMALL1: e = launch_attn_small_bf16(p, 1, h->small_kw, stream); break;
+            case KIND_SMALL2: e = launch_attn_small_bf16(p, 2, h->small_kw, stream); break;
+            case KIND_SMALL4: e = launch_attn_small_bf16(p, 4, 4, stream); break;
             case KIND_SIMT: e = launch_attn_simt_f32(p, stream); break;
             case KIND_TILE: e = launch_attn_tile_bf16(p, false, stream); break;
             case KIND_STREAM: e = launch_attn_tile_bf16(p, true, stream); break;

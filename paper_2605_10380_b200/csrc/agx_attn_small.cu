@@ -7,14 +7,16 @@
 // dimension of warp-level bf16 tensor-core MMAs (m16n8k16, fp32 accumulate): the kernel stays
 // bandwidth-bound and verifying 8 tokens costs the same bytes as decoding 1.
 //
-// Work item = (sequence, KV head, KV split).  A CTA of 4 * MT warps: warp (mt, kg) owns query rows
-// [16 mt, 16 mt + 16) and, in every 64-token stage, page kg.  K/V pages stream through a
-// multi-stage ring filled by TMA (per page two [16 tokens][64 dims] boxes for K and for V,
-// SWIZZLE_128B so ldmatrix is conflict-free; page ids come from the page table, prefetched 32 at a
-// time) and handed over with full/empty mbarriers, so no thread spends instructions on addresses and
-// warps never meet at a CTA-wide barrier inside the loop; the four KV groups keep private
-// online-softmax states that are merged through shared memory at the end.  Splits write fp32 (m, l, O) partials; a combine kernel merges them in fixed order, so
-// results are bit-reproducible run to run.
+// Work item = (sequence, KV head, KV split).  A CTA of KW * MT warps (KW = 4 or 8 KV groups): warp (mt, kg)
+// owns query rows [16 mt, 16 mt + 16) and, in every stage of KW pages, page kg.  K/V pages stream through a
+// 3-stage ring filled by TMA (per page two [16 tokens][64 dims] boxes for K and for V, SWIZZLE_128B so
+// ldmatrix is conflict-free; page ids come from the page table, prefetched 32 at a time) and handed over
+// with full/empty mbarriers, so no thread spends instructions on addresses and warps never meet at a
+// CTA-wide barrier inside the loop; the KV groups keep private online-softmax states that are merged
+// through shared memory at the end.  KW = 8 (16 warps for a 32-row verify block, one CTA per SM) halves the
+// number of dependent page steps per warp, which is what a 4k-token context is bounded by.  Splits write
+// fp32 (m, l, O) partials; a combine kernel merges them in fixed order, so results are bit-reproducible
+// run to run.
 #include <math.h>
 
 #include "agx_internal.cuh"
@@ -26,9 +28,7 @@ namespace {
 
 constexpr int kD = 128;                    // head dim of the bf16 kernels
 constexpr int kRowBytes = kD * 2;          // one (token, head) row
-constexpr int kKW = 4;                     // KV groups (pages per stage)
-constexpr int kStageTokens = kKW * kPage;  // 64
-constexpr int kStageBytes = 2 * kStageTokens * kRowBytes;  // K + V = 32 KB
+// KW = KV groups = pages per pipeline stage (4 or 8): stage = KW * 16 tokens, K + V = KW * 8 KB
 constexpr int kMergeStride = 136;          // floats per merged row (conflict-free float2 stores)
 
 
@@ -62,13 +62,16 @@ __device__ __forceinline__ int find_seq(const AttnParams& p, int item) {
 
 }  // namespace
 
-template <int MT, int NS>
-__global__ void __launch_bounds__(128 * MT, (MT <= 2) ? 2 : 1)
+template <int MT, int KW, int NS>
+__global__ void __launch_bounds__(32 * MT * KW, (MT * KW <= 8) ? 2 : 1)
 attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v) {
     extern __shared__ unsigned char smem_raw[];
-    constexpr int kThreads = 128 * MT;
-    constexpr int kWarps = 4 * MT;
+    constexpr int kKW = KW;
+    constexpr int kStageTokens = kKW * kPage;
+    constexpr int kStageBytes = 2 * kStageTokens * kRowBytes;
+    constexpr int kThreads = 32 * MT * KW;
+    constexpr int kWarps = MT * KW;
     constexpr int kRingBytes = NS * kStageBytes;
     constexpr int kMergeBytes = MT * kKW * 16 * (kMergeStride * 4 + 8);
     constexpr int kRegion = kRingBytes > kMergeBytes ? kRingBytes : kMergeBytes;
@@ -561,35 +564,35 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
 
 // --------------------------------------------------------------------------------------------
 namespace {
-template <int MT, int NS>
+template <int MT, int KW, int NS>
 cudaError_t launch_small(const AttnParams& p, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
-    constexpr int kMergeBytes = MT * kKW * 16 * (kMergeStride * 4 + 8);
-    constexpr int kRing = NS * kStageBytes;
+    constexpr int kMergeBytes = MT * KW * 16 * (kMergeStride * 4 + 8);
+    constexpr int kRing = NS * 2 * KW * kPage * kRowBytes;
     // [ring | merge region][Q tile][2 * NS barriers + abort flag] + slack for the 1024-byte alignment
     constexpr int kSmem = (kRing > kMergeBytes ? kRing : kMergeBytes) + MT * 16 * kRowBytes + 2 * NS * 8 + 16 + 1024;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attn_small_bf16_kernel<MT, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+        cudaError_t e = cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    attn_small_bf16_kernel<MT, NS><<<p.num_items, 128 * MT, kSmem, stream>>>(p, map_k, map_v);
+    attn_small_bf16_kernel<MT, KW, NS><<<p.num_items, 32 * MT * KW, kSmem, stream>>>(p, map_k, map_v);
     return cudaGetLastError();
 }
 }  // namespace
 
-int attn_small_bf16_kv_tile() { return kStageTokens; }
-
-cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, cudaStream_t stream) {
+cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, int kw, cudaStream_t stream) {
     if (p.num_items == 0) return cudaSuccess;
     if ((long long)p.num_pages * p.hkv * kPage > 0x7FFFFFFFll) return cudaErrorInvalidValue;
     alignas(64) CUtensorMap map_k, map_v;
     if (!make_pool_map(&map_k, p.k_pool, p.num_pages, p.hkv) || !make_pool_map(&map_v, p.v_pool, p.num_pages, p.hkv))
         return cudaErrorNotSupported;
-    switch (mt) {
-        case 1: return launch_small<1, 3>(p, map_k, map_v, stream);
-        case 2: return launch_small<2, 3>(p, map_k, map_v, stream);
-        case 4: return launch_small<4, 5>(p, map_k, map_v, stream);
+    switch (mt * 16 + kw) {
+        case 1 * 16 + 4: return launch_small<1, 4, 3>(p, map_k, map_v, stream);
+        case 2 * 16 + 4: return launch_small<2, 4, 3>(p, map_k, map_v, stream);
+        case 1 * 16 + 8: return launch_small<1, 8, 3>(p, map_k, map_v, stream);
+        case 2 * 16 + 8: return launch_small<2, 8, 3>(p, map_k, map_v, stream);
+        case 4 * 16 + 4: return launch_small<4, 4, 5>(p, map_k, map_v, stream);
         default: return cudaErrorInvalidValue;
     }
 }

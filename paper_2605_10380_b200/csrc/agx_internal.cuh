@@ -50,9 +50,9 @@ cudaError_t launch_kv_append(int dtype, void* k_pool, void* v_pool, long long nu
                              const int* cu_q, int B, int total_q, int hkv, int head_dim, int* status,
                              cudaStream_t stream);
 
-// Small-q split-KV kernel (bf16, d = 128, tensor-core mma.sync); mt = m-tiles of 16 rows (1, 2, 4).
-cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, cudaStream_t stream);
-int attn_small_bf16_kv_tile();  // tokens per pipeline stage
+// Small-q split-KV kernel (bf16, d = 128, tensor-core mma.sync); mt = m-tiles of 16 rows (1, 2, 4), kw = KV groups
+// (4 or 8 pages per pipeline stage; 8 only with mt <= 2): CTA = 32 * mt * kw threads.
+cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, int kw, cudaStream_t stream);
 // Scalar fp32-math kernel for AGX_F32 pools (any q, d in {64, 128}).
 cudaError_t launch_attn_simt_f32(const AttnParams& p, cudaStream_t stream);
 // Merge of split partials into out / lse.
