@@ -252,6 +252,26 @@ AGX_API agx_status agx_verify_step_host(agx_handle* handle, void* k_pool, void* 
                                         int32_t* h_seq_lens, void* workspace,
                                         size_t workspace_bytes, void* stream);
 
+/*
+ * agx_verify_step_host_enqueue - the same step (Sec. 2.3: append, attention, acceptance) and the same
+ * arguments as agx_verify_step_host, but the call returns as soon as the copies and kernels are enqueued.
+ * A model calls it once per layer and synchronises the stream once per step, so the copies of one layer
+ * overlap the kernels of another.  Until the caller has synchronised the stream, the host input buffers
+ * must stay unchanged when they are pinned memory (pageable buffers are staged before the call returns),
+ * the host outputs are not valid, and the workspace belongs to the calls in flight (calls on one stream
+ * may share it: they run in order).
+ */
+AGX_API agx_status agx_verify_step_host_enqueue(agx_handle* handle, void* k_pool, void* v_pool,
+                                                int64_t num_pages, const int32_t* page_table,
+                                                int32_t page_table_stride, const int32_t* h_prefix_len,
+                                                const int32_t* h_q_len, int32_t B, const void* h_q_block,
+                                                const void* h_k_new, const void* h_v_new,
+                                                const void* h_logits, int32_t logits_dtype,
+                                                int64_t row_stride, int32_t vocab, const int32_t* h_drafts,
+                                                void* h_out, int32_t* h_accept_len, int32_t* h_next_token,
+                                                int32_t* h_seq_lens, void* workspace,
+                                                size_t workspace_bytes, void* stream);
+
 /* Number of kernels the last agx_attn_prefixed / agx_accept_greedy / agx_kv_append call on this
  * handle launched (for launch accounting in benchmarks). */
 AGX_API int32_t agx_last_launch_count(const agx_handle* handle);

@@ -25,7 +25,8 @@ EXPORTS = (
     "agx_create", "agx_destroy", "agx_status_string", "agx_last_error", "agx_kv_append",
     "agx_attn_workspace_bytes", "agx_attn_prefixed", "agx_accept_workspace_bytes",
     "agx_accept_greedy", "agx_get_status", "agx_last_launch_count",
-    "agx_verify_step_host_workspace_bytes", "agx_verify_step_host", "agx_accept_greedy_static",
+    "agx_verify_step_host_workspace_bytes", "agx_verify_step_host", "agx_verify_step_host_enqueue",
+    "agx_accept_greedy_static",
 )
 
 
@@ -84,6 +85,8 @@ def load() -> ctypes.CDLL:
                                          vp, vp, vp, vp,                        # host outputs
                                          vp, ctypes.c_size_t, vp]
     lib.agx_verify_step_host.restype = i32
+    lib.agx_verify_step_host_enqueue.argtypes = lib.agx_verify_step_host.argtypes
+    lib.agx_verify_step_host_enqueue.restype = i32
     lib.agx_accept_greedy_static.argtypes = [vp, i32, i64, i32, vp, vp, i32, i32, vp, vp, vp, vp, vp]
     lib.agx_accept_greedy_static.restype = i32
     _lib = lib
@@ -223,13 +226,17 @@ class Handle:
     # -- agx_verify_step_host (host tensors: pinned torch tensors or numpy arrays)
     def verify_step_host(self, k_pool, v_pool, page_table, h_prefix_len, h_q_len, h_q_block, h_k_new, h_v_new,
                          h_logits, logits_dtype: str, row_stride: int, vocab: int, h_drafts, h_out, h_accept_len,
-                         h_next_token, h_seq_lens, workspace, stream=None):
+                         h_next_token, h_seq_lens, workspace, stream=None, enqueue_only: bool = False):
+        """agx_verify_step_host, or agx_verify_step_host_enqueue when ``enqueue_only`` (the caller then
+        synchronises the stream before reading the host outputs and keeps ``h_prefix_len``/``h_q_len`` and the
+        pinned inputs alive until then)."""
         P, Q = _h_i32(h_prefix_len), _h_i32(h_q_len)
         ws_bytes = workspace.numel() * workspace.element_size()
-        st = self._lib.agx_verify_step_host(self._h, _ptr(k_pool), _ptr(v_pool), int(k_pool.shape[0]),
-                                            _ptr(page_table), int(page_table.shape[1]), _ptr(P), _ptr(Q),
-                                            int(P.shape[0]), _ptr(h_q_block), _ptr(h_k_new), _ptr(h_v_new),
-                                            _ptr(h_logits), DTYPES[logits_dtype], int(row_stride), int(vocab),
-                                            _ptr(h_drafts), _ptr(h_out), _ptr(h_accept_len), _ptr(h_next_token),
-                                            _ptr(h_seq_lens), _ptr(workspace), ws_bytes, _stream_ptr(stream))
-        self._check(st, "agx_verify_step_host")
+        fn = self._lib.agx_verify_step_host_enqueue if enqueue_only else self._lib.agx_verify_step_host
+        st = fn(self._h, _ptr(k_pool), _ptr(v_pool), int(k_pool.shape[0]),
+                _ptr(page_table), int(page_table.shape[1]), _ptr(P), _ptr(Q),
+                int(P.shape[0]), _ptr(h_q_block), _ptr(h_k_new), _ptr(h_v_new),
+                _ptr(h_logits), DTYPES[logits_dtype], int(row_stride), int(vocab),
+                _ptr(h_drafts), _ptr(h_out), _ptr(h_accept_len), _ptr(h_next_token),
+                _ptr(h_seq_lens), _ptr(workspace), ws_bytes, _stream_ptr(stream))
+        self._check(st, "agx_verify_step_host_enqueue" if enqueue_only else "agx_verify_step_host")

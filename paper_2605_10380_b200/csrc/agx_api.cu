@@ -458,12 +458,12 @@ int64_t agx_verify_step_host_workspace_bytes(agx_handle* h, int32_t B, const int
     return st != AGX_OK ? (int64_t)st : (int64_t)L.total;
 }
 
-agx_status agx_verify_step_host(agx_handle* h, void* k_pool, void* v_pool, int64_t num_pages,
+static agx_status verify_step_host_impl(agx_handle* h, void* k_pool, void* v_pool, int64_t num_pages,
                                 const int32_t* page_table, int32_t pt_stride, const int32_t* P, const int32_t* Q,
                                 int32_t B, const void* h_q, const void* h_k, const void* h_v, const void* h_logits,
                                 int32_t logits_dtype, int64_t row_stride, int32_t vocab, const int32_t* h_drafts,
                                 void* h_out, int32_t* h_accept, int32_t* h_next, int32_t* h_seq_lens, void* workspace,
-                                size_t workspace_bytes, void* stream_v) {
+                                size_t workspace_bytes, void* stream_v, bool sync) {
     if (!h) return AGX_E_INVAL;
     HostStepLayout L;
     agx_status st = host_step_layout(h, B, P, Q, logits_dtype, row_stride, vocab, L);
@@ -516,10 +516,32 @@ agx_status agx_verify_step_host(agx_handle* h, void* k_pool, void* v_pool, int64
     if (with_accept) {
         d2h(h_accept, L.acc, (size_t)B * 4); d2h(h_next, L.next, (size_t)B * 4); d2h(h_seq_lens, L.seqlen, (size_t)B * 4);
     }
-    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e == cudaSuccess && sync) e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return cuda_fail(h, e, "host step: download");
     h->last_launches = launches;
     return AGX_OK;
+}
+
+agx_status agx_verify_step_host(agx_handle* h, void* k_pool, void* v_pool, int64_t num_pages,
+                                const int32_t* page_table, int32_t pt_stride, const int32_t* P, const int32_t* Q,
+                                int32_t B, const void* h_q, const void* h_k, const void* h_v, const void* h_logits,
+                                int32_t logits_dtype, int64_t row_stride, int32_t vocab, const int32_t* h_drafts,
+                                void* h_out, int32_t* h_accept, int32_t* h_next, int32_t* h_seq_lens, void* workspace,
+                                size_t workspace_bytes, void* stream) {
+    return verify_step_host_impl(h, k_pool, v_pool, num_pages, page_table, pt_stride, P, Q, B, h_q, h_k, h_v, h_logits,
+                                 logits_dtype, row_stride, vocab, h_drafts, h_out, h_accept, h_next, h_seq_lens, workspace,
+                                 workspace_bytes, stream, true);
+}
+
+agx_status agx_verify_step_host_enqueue(agx_handle* h, void* k_pool, void* v_pool, int64_t num_pages,
+                                        const int32_t* page_table, int32_t pt_stride, const int32_t* P, const int32_t* Q,
+                                        int32_t B, const void* h_q, const void* h_k, const void* h_v,
+                                        const void* h_logits, int32_t logits_dtype, int64_t row_stride, int32_t vocab,
+                                        const int32_t* h_drafts, void* h_out, int32_t* h_accept, int32_t* h_next,
+                                        int32_t* h_seq_lens, void* workspace, size_t workspace_bytes, void* stream) {
+    return verify_step_host_impl(h, k_pool, v_pool, num_pages, page_table, pt_stride, P, Q, B, h_q, h_k, h_v, h_logits,
+                                 logits_dtype, row_stride, vocab, h_drafts, h_out, h_accept, h_next, h_seq_lens, workspace,
+                                 workspace_bytes, stream, false);
 }
 
 }  // extern "C"

@@ -241,6 +241,35 @@ def test_accept_many_rows_and_unaligned_rows():
         assert np.array_equal(g, r)
 
 
+# ------------------------------------------------------------------ whole step from host buffers
+@pytest.mark.parametrize("enqueue_only", [False, True])
+def test_verify_step_host_matches_oracle(enqueue_only):
+    """Append + attention + accept through the host-buffer entry points (pinned inputs, results back in
+    host memory); the enqueue variant returns before the work is done and is synchronised by the caller."""
+    w = W.make_attn_workload("host_step", 77, "bf16", 32, 8, 128, [1000, 517, 40], [8, 4, 1], spare_pages=2)
+    aw = W.make_planted_accept("host_step_accept", 78, "bf16", 128256, w.q_len, w.prefix_len)
+    b = DeviceBatch(w)
+    pin = lambda a, bf=False: (torch.from_numpy(np.ascontiguousarray(a)).view(torch.bfloat16) if bf else torch.from_numpy(np.ascontiguousarray(a))).pin_memory()
+    hq, hk, hv = pin(w.q_block, True), pin(w.k_new, True), pin(w.v_new, True)
+    hl, hd = pin(aw.logits, True), pin(aw.drafts)
+    h_out = torch.zeros((w.total_q, 32, 128), dtype=torch.bfloat16).pin_memory()
+    h_acc = torch.full((3,), -7, dtype=torch.int32).pin_memory()
+    h_nxt = torch.full((3,), -7, dtype=torch.int32).pin_memory()
+    h_sl = torch.full((3,), -7, dtype=torch.int32).pin_memory()
+    n = b.h.verify_step_host_workspace_bytes(w.prefix_len, w.q_len, "bf16", 128256, 128256)
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+    b.h.verify_step_host(b.k_pool, b.v_pool, b.page_table, w.prefix_len, w.q_len, hq, hk, hv, hl, "bf16", 128256, 128256,
+                         hd, h_out, h_acc, h_nxt, h_sl, ws, enqueue_only=enqueue_only)
+    torch.cuda.synchronize()
+    assert b.status() == 0
+    kp, vp = oracle_pools_after_append(w)
+    assert np.array_equal(host_storage(b.k_pool, "bf16"), kp) and np.array_equal(host_storage(b.v_pool, "bf16"), vp)
+    ref, _ = oracle.attn_paged_batch(w.q_block, kp, vp, w.page_table, "bf16", w.prefix_len, w.q_len, w.cu_q)
+    check_attention(h_out.to(torch.float64).numpy(), ref, "host step")
+    am, al, nt, sl = oracle.accept_greedy(aw.logits, "bf16", aw.vocab, aw.drafts, aw.cu_q, aw.prefix_len)
+    assert np.array_equal(h_acc.numpy(), al) and np.array_equal(h_nxt.numpy(), nt) and np.array_equal(h_sl.numpy(), sl)
+
+
 # ------------------------------------------------------------------ argument errors (host side)
 def test_argument_errors_are_reported_not_faulted():
     w = W.make_attn_workload("err", 6, "bf16", 32, 8, 128, [100], [4])
