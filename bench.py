@@ -35,6 +35,9 @@ if ROOT not in sys.path:
 METRIC = "prefix-cached attn query tok/s"
 UNIT = "query tok/s (per attention-layer call)"
 C2 = dict(P=4096, q=8, hq=32, hkv=8, d=128, vocab=128256, layers=32)
+# DRAM bytes of one attention call of this workload (attention kernel 16,957,696 + combine kernel 2,304,768), from the
+# ncu capture summarised under profiles/; set to None whenever one of the two kernels changes until it is re-captured
+NCU_TRAFFIC_BYTES = 16957696 + 2304768
 
 
 # --------------------------------------------------------------------------- peaks / clocks
@@ -428,9 +431,11 @@ def run_agx(args):
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_max,
                 "path": "agx_verify_step_host_enqueue per layer (pinned host q/k_new/v_new/logits in, out/accept results back), one stream synchronisation per step"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES, "peak_source": peaks["source"],
                      "frac_of_nominal_8000": achieved / 8000.0,
-                     "kernel": "attn_small_bf16_kernel<2,3> + attn_combine_kernel (one agx_attn_prefixed call)",
+                     "kernel": "attn_small_bf16_kernel<2,8,3> + attn_combine_kernel (one agx_attn_prefixed call)",
+                     "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of both kernels, one launch each, "
+                                       "profiles/attn_small_combine_c2_decode_verify.txt",
                      "algorithmic_bytes_per_launch": by, "us_per_launch": ms_attn * 1e3},
         "clocks": clocks,
     }
