@@ -8,8 +8,8 @@ with seeded projections around it.
 
 The n-gram table follows Sec. 4.3: slide a window of n tokens over a token stream, key = the
 first n-1 tokens, value = the successor seen most often with that key.  The paper does not
-say which successor wins a count tie; here the one that reached the winning count first
-(earliest in the stream) wins.
+say which successor wins a count tie; here the lowest token id wins (a rule that does not
+depend on the order in which windows are visited).
 """
 from __future__ import annotations
 
@@ -54,41 +54,34 @@ class ToyLM:
 
 
 def build_ngram_table(stream, n: int = 3) -> dict:
-    """Sec. 4.3: key = n-1 consecutive tokens, value = their most frequent successor."""
-    counts: "OrderedDict[tuple, OrderedDict[int, int]]" = OrderedDict()
+    """Sec. 4.3: slide a window of n tokens over the stream; key = its first n-1 tokens, value = the
+    successor recorded most often with that key.  Equal counts: the lowest token id wins."""
     stream = [int(t) for t in stream]
+    counts: dict = {}
     for i in range(len(stream) - n + 1):
         key = tuple(stream[i:i + n - 1])
         nxt = stream[i + n - 1]
-        bucket = counts.setdefault(key, OrderedDict())
+        bucket = counts.setdefault(key, {})
         bucket[nxt] = bucket.get(nxt, 0) + 1
     table = {}
     for key, bucket in counts.items():
         top = max(bucket.values())
-        # replay the stream: the successor that reaches the winning count first wins a tie
-        run = {}
-        for i in range(len(stream) - n + 1):
-            if tuple(stream[i:i + n - 1]) != key:
-                continue
-            nxt = stream[i + n - 1]
-            run[nxt] = run.get(nxt, 0) + 1
-            if run[nxt] == top:
-                table[key] = nxt
-                break
+        table[key] = min(tok for tok, c in bucket.items() if c == top)
     return table
 
 
-def ngram_drafts(table: dict, history, k: int, n: int, rng: np.random.Generator, vocab: int):
+def ngram_drafts(table: dict, history, k: int, n: int, rng=None, vocab: int = 0, fill=None):
     """Sec. 4.3: chain k drafts from the last n-1 tokens.  Returns None when the FIRST lookup
-    misses (selective fallback to a plain one-token step); later misses guess a random token."""
+    misses (selective fallback to a plain one-token step); a later miss guesses a token: ``fill[i]``
+    when given, else a draw from ``rng``."""
     ctx = [int(t) for t in history[-(n - 1):]]
     if len(ctx) < n - 1 or tuple(ctx) not in table:
         return None
     out = []
-    for _ in range(k):
+    for i in range(k):
         tok = table.get(tuple(ctx))
         if tok is None:
-            tok = int(rng.integers(0, vocab))
+            tok = int(fill[i]) if fill is not None else int(rng.integers(0, vocab))
         out.append(int(tok))
-        ctx = ctx[1:] + [int(tok)]
+        ctx = (ctx + [int(tok)])[1:] if n > 1 else []
     return out

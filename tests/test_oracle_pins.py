@@ -428,9 +428,44 @@ def test_ngram_table_most_frequent_successor():
     stream = [1, 2, 3, 1, 2, 4, 1, 2, 4, 9, 9, 9]
     t = build_ngram_table(stream, 3)
     assert t[(1, 2)] == 4 and t[(9, 9)] == 9 and (2, 9) not in t
-    assert build_ngram_table([5, 6, 7, 5, 6, 8], 3)[(5, 6)] == 7  # count tie: first to reach it
+    assert build_ngram_table([5, 6, 8, 5, 6, 7], 3)[(5, 6)] == 7  # count tie: lowest token id
+    assert build_ngram_table([5, 6, 7, 5, 6, 8], 3)[(5, 6)] == 7
     rng = np.random.default_rng(0)
     assert ngram_drafts(t, [7, 7], 4, 3, rng, 10) is None  # first lookup misses -> fallback
     d = ngram_drafts(t, [0, 1, 2], 3, 3, rng, 10)
     assert d[0] == 4 and d[1] == 1 and len(d) == 3  # (1,2)->4, (2,4)->1, (4,1)->2
     assert d[2] == 2
+
+
+def _naive_ngram(stream, n):
+    """Independent restatement with collections.Counter: most common successor, ties to the lowest id."""
+    from collections import Counter, defaultdict
+    succ = defaultdict(Counter)
+    for w in zip(*[stream[i:] for i in range(n)]):
+        succ[tuple(int(t) for t in w[:-1])][int(w[-1])] += 1
+    return {k: sorted(c.items(), key=lambda kv: (-kv[1], kv[0]))[0][0] for k, c in succ.items()}
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4])
+def test_ngram_table_against_counter_brute_force(n):
+    from oracle.toy_lm import build_ngram_table
+    rng = np.random.default_rng(100 + n)
+    for length, alphabet in [(0, 3), (n - 1, 3), (n, 3), (50, 2), (400, 5), (3000, 40)]:
+        stream = rng.integers(0, alphabet, size=max(length, 0)).tolist()
+        assert build_ngram_table(stream, n) == _naive_ngram(stream, n)
+
+
+def test_ngram_drafts_reproduce_a_periodic_stream_and_fall_back_on_unknown_context():
+    """Closed form: on a stream that repeats a block of distinct tokens every bigram has one successor, so
+    the trigram chain continues the stream exactly; an unseen context gives no drafts at all (Sec. 4.3,
+    selective decoding), a context that goes unknown mid-chain takes the supplied guesses."""
+    from oracle.toy_lm import build_ngram_table, ngram_drafts
+    block = [11, 4, 7, 300, 2, 9]
+    stream = block * 5
+    t = build_ngram_table(stream, 3)
+    assert len(t) == len(block)
+    assert ngram_drafts(t, stream[:8], 9, 3, fill=[0] * 9) == (block * 4)[8 % 6:8 % 6 + 9]
+    assert ngram_drafts(t, [4, 11], 3, 3, fill=[0] * 3) is None
+    open_ended = build_ngram_table([1, 2, 3, 4], 3)          # (1,2)->3, (2,3)->4, nothing after (3,4)
+    assert ngram_drafts(open_ended, [1, 2], 4, 3, fill=[50, 51, 52, 53]) == [3, 4, 52, 53]
+    assert ngram_drafts(build_ngram_table([5, 5, 6, 5, 7, 5, 6], 2), [5], 2, 2, fill=[0, 0]) == [6, 5]  # bigram: 5 -> 6 twice
