@@ -67,7 +67,8 @@ enum { AGX_BF16 = 0, AGX_F32 = 1 };
 /* Bits of the device status word (sticky until agx_get_status clears them). */
 enum {
     AGX_DEV_BAD_PAGE = 1,    /* a page id outside [0, num_pages) was met; the access was skipped */
-    AGX_DEV_WAIT_TIMEOUT = 2 /* a bounded in-kernel wait gave up; results of that launch are invalid */
+    AGX_DEV_WAIT_TIMEOUT = 2, /* a bounded in-kernel wait gave up; results of that launch are invalid */
+    AGX_DEV_BAD_TOKEN = 4     /* agx_ngram_build met a token id outside [0, 2^21); its windows were skipped */
 };
 
 typedef struct agx_config {
@@ -271,6 +272,44 @@ AGX_API agx_status agx_verify_step_host_enqueue(agx_handle* handle, void* k_pool
                                                 void* h_out, int32_t* h_accept_len, int32_t* h_next_token,
                                                 int32_t* h_seq_lens, void* workspace,
                                                 size_t workspace_bytes, void* stream);
+
+/*
+ * agx_ngram_build - the draft table of example-based speculative decoding, built on the device.
+ * Sec. 4.3: a window of n consecutive tokens slides over one token stream (the prompt's examples and
+ * the query); the first n-1 tokens of a window are a key, and the key's value is the token that follows
+ * it most often in the stream.  The paper does not say which successor wins when counts are equal:
+ * here the lowest token id does.
+ *   stream_tokens : device int32 [num_tokens], ids in [0, 2^21); a window holding any other id is
+ *                   skipped and sets AGX_DEV_BAD_TOKEN
+ *   n             : 2 or 3 (3, the trigram table, is the paper's choice)
+ *   lut           : device, >= agx_ngram_lut_bytes(num_tokens) bytes, 16-byte aligned; opaque, valid
+ *                   until overwritten; read by agx_ngram_draft
+ *   workspace     : device, >= agx_ngram_workspace_bytes(num_tokens) bytes, 16-byte aligned
+ * num_tokens < n builds an empty table.  Errors: AGX_E_INVAL, AGX_E_UNSUPPORTED (n), AGX_E_RANGE
+ * (num_tokens > 2^24), AGX_E_CUDA.
+ */
+AGX_API int64_t agx_ngram_lut_bytes(int32_t max_stream_tokens);
+AGX_API int64_t agx_ngram_workspace_bytes(int32_t stream_tokens);
+AGX_API agx_status agx_ngram_build(agx_handle* handle, const int32_t* stream_tokens, int32_t num_tokens,
+                                   int32_t n, void* lut, size_t lut_bytes, void* workspace,
+                                   size_t workspace_bytes, void* stream);
+
+/*
+ * agx_ngram_draft - k draft tokens per sequence by chained table lookups (Sec. 4.3).
+ * Draft 1 is the table's value for the sequence's last n-1 tokens, draft 2 the value for the last n-2
+ * tokens followed by draft 1, and so on.  Selective decoding: has_draft[s] = 0 when the FIRST lookup
+ * misses - the caller then runs a plain one-token step (q_len = 1) instead of paying for a verify block
+ * that cannot be accepted; after a first hit, a later miss takes the caller's guess fill[s][i] (the
+ * paper's "random token", drawn by the caller) and the chain goes on from it.
+ *   lut        : device, built by agx_ngram_build
+ *   context    : device int32 [B][n-1], the most recent n-1 tokens of each sequence, oldest first
+ *   fill       : device int32 [B][k]
+ *   drafts     : device int32 [B][k] (written in any case); has_draft : device int32 [B] (written)
+ * Errors: AGX_E_INVAL (null pointers, B < 0, k < 0), AGX_E_CUDA.
+ */
+AGX_API agx_status agx_ngram_draft(agx_handle* handle, const void* lut, const int32_t* context,
+                                   const int32_t* fill, int32_t B, int32_t k, int32_t* drafts,
+                                   int32_t* has_draft, void* stream);
 
 /* Number of kernels the last agx_attn_prefixed / agx_accept_greedy / agx_kv_append call on this
  * handle launched (for launch accounting in benchmarks). */

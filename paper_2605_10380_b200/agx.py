@@ -15,7 +15,7 @@ import numpy as np
 
 AGX_OK = 0
 AGX_BF16, AGX_F32 = 0, 1
-AGX_DEV_BAD_PAGE, AGX_DEV_WAIT_TIMEOUT = 1, 2
+AGX_DEV_BAD_PAGE, AGX_DEV_WAIT_TIMEOUT, AGX_DEV_BAD_TOKEN = 1, 2, 4
 DTYPES = {"bf16": AGX_BF16, "f32": AGX_F32}
 
 _LIB_PATH = Path(__file__).resolve().parent / "lib" / "libagx.so"
@@ -26,7 +26,7 @@ EXPORTS = (
     "agx_attn_workspace_bytes", "agx_attn_prefixed", "agx_accept_workspace_bytes",
     "agx_accept_greedy", "agx_get_status", "agx_last_launch_count",
     "agx_verify_step_host_workspace_bytes", "agx_verify_step_host", "agx_verify_step_host_enqueue",
-    "agx_accept_greedy_static",
+    "agx_accept_greedy_static", "agx_ngram_lut_bytes", "agx_ngram_workspace_bytes", "agx_ngram_build", "agx_ngram_draft",
 )
 
 
@@ -40,6 +40,14 @@ class AgxError(RuntimeError):
     def __init__(self, status: int, where: str, detail: str = ""):
         self.status = status
         super().__init__(f"{where}: status {status} ({status_string(status)}) {detail}".rstrip())
+
+
+def ngram_lut_bytes(max_stream_tokens: int) -> int:
+    return int(load().agx_ngram_lut_bytes(int(max_stream_tokens)))
+
+
+def ngram_workspace_bytes(stream_tokens: int) -> int:
+    return int(load().agx_ngram_workspace_bytes(int(stream_tokens)))
 
 
 def lib_path() -> Path:
@@ -89,6 +97,14 @@ def load() -> ctypes.CDLL:
     lib.agx_verify_step_host_enqueue.restype = i32
     lib.agx_accept_greedy_static.argtypes = [vp, i32, i64, i32, vp, vp, i32, i32, vp, vp, vp, vp, vp]
     lib.agx_accept_greedy_static.restype = i32
+    lib.agx_ngram_lut_bytes.argtypes = [i32]
+    lib.agx_ngram_lut_bytes.restype = i64
+    lib.agx_ngram_workspace_bytes.argtypes = [i32]
+    lib.agx_ngram_workspace_bytes.restype = i64
+    lib.agx_ngram_build.argtypes = [vp, vp, i32, i32, vp, ctypes.c_size_t, vp, ctypes.c_size_t, vp]
+    lib.agx_ngram_build.restype = i32
+    lib.agx_ngram_draft.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp]
+    lib.agx_ngram_draft.restype = i32
     _lib = lib
     return lib
 
@@ -204,6 +220,18 @@ class Handle:
                                          _ptr(next_token), _ptr(argmax), _ptr(seq_lens), _ptr(workspace), ws_bytes,
                                          _stream_ptr(stream))
         self._check(st, "agx_accept_greedy")
+
+    # -- agx_ngram_build / agx_ngram_draft (device int32 tensors; lut and workspace are uint8 tensors)
+    def ngram_build(self, stream_tokens, n: int, lut, workspace, stream=None):
+        st = self._lib.agx_ngram_build(self._h, _ptr(stream_tokens), int(stream_tokens.numel()), int(n), _ptr(lut),
+                                       lut.numel() * lut.element_size(), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+        self._check(st, "agx_ngram_build")
+
+    def ngram_draft(self, lut, context, fill, k: int, drafts, has_draft, stream=None):
+        st = self._lib.agx_ngram_draft(self._h, _ptr(lut), _ptr(context), _ptr(fill), int(has_draft.shape[0]), int(k),
+                                       _ptr(drafts), _ptr(has_draft), _stream_ptr(stream))
+        self._check(st, "agx_ngram_draft")
 
     # -- agx_get_status
     def get_status(self, stream=None, raise_on_error: bool = False) -> int:

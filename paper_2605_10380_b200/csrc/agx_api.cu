@@ -544,4 +544,45 @@ agx_status agx_verify_step_host_enqueue(agx_handle* h, void* k_pool, void* v_poo
                                  workspace_bytes, stream, false);
 }
 
+int64_t agx_ngram_lut_bytes(int32_t max_stream_tokens) {
+    if (max_stream_tokens < 0 || max_stream_tokens > (1 << 24)) return AGX_E_RANGE;
+    return (int64_t)ngram_lut_bytes(max_stream_tokens);
+}
+
+int64_t agx_ngram_workspace_bytes(int32_t stream_tokens) {
+    if (stream_tokens < 0 || stream_tokens > (1 << 24)) return AGX_E_RANGE;
+    return (int64_t)ngram_workspace_bytes(stream_tokens);
+}
+
+agx_status agx_ngram_build(agx_handle* h, const int32_t* stream_tokens, int32_t num_tokens, int32_t n, void* lut,
+                           size_t lut_bytes, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!h) return AGX_E_INVAL;
+    h->last_launches = 0;
+    if (n != 2 && n != 3) return fail(h, AGX_E_UNSUPPORTED, "n-gram order %d (2 and 3 are built)", n);
+    if (num_tokens < 0) return fail(h, AGX_E_INVAL, "negative num_tokens");
+    if (num_tokens > (1 << 24)) return fail(h, AGX_E_RANGE, "more than 2^24 stream tokens");
+    if (!lut || !workspace || (!stream_tokens && num_tokens > 0)) return fail(h, AGX_E_INVAL, "null pointer");
+    if (!aligned(lut, 16) || !aligned(workspace, 16)) return fail(h, AGX_E_INVAL, "lut/workspace must be 16-byte aligned");
+    if ((long long)lut_bytes < ngram_lut_bytes(num_tokens) || (long long)workspace_bytes < ngram_workspace_bytes(num_tokens))
+        return fail(h, AGX_E_INVAL, "lut (%lld needed) or workspace (%lld needed) too small", ngram_lut_bytes(num_tokens),
+                    ngram_workspace_bytes(num_tokens));
+    cudaError_t e = launch_ngram_build(stream_tokens, num_tokens, n, lut, workspace, h->d_status, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "n-gram build");
+    h->last_launches = num_tokens >= n ? 3 : 1;
+    return AGX_OK;
+}
+
+agx_status agx_ngram_draft(agx_handle* h, const void* lut, const int32_t* context, const int32_t* fill, int32_t B, int32_t k,
+                           int32_t* drafts, int32_t* has_draft, void* stream) {
+    if (!h) return AGX_E_INVAL;
+    h->last_launches = 0;
+    if (B < 0 || k < 0) return fail(h, AGX_E_INVAL, "negative B or k");
+    if (B == 0) return AGX_OK;
+    if (!lut || !context || !has_draft || (k > 0 && (!fill || !drafts))) return fail(h, AGX_E_INVAL, "null pointer");
+    cudaError_t e = launch_ngram_draft(lut, context, fill, B, k, drafts, has_draft, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "n-gram draft");
+    h->last_launches = 1;
+    return AGX_OK;
+}
+
 }  // extern "C"

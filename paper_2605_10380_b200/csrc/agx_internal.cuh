@@ -69,4 +69,12 @@ cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_st
                           int* seq_lens, unsigned long long* partials, int chunks, unsigned int* ticket,
                           cudaStream_t stream);
 
+// n-gram draft table (Sec. 4.3): sizes, build (three memsets + three small kernels) and chained lookups.
+long long ngram_lut_bytes(int max_stream_tokens);
+long long ngram_workspace_bytes(int stream_tokens);
+cudaError_t launch_ngram_build(const int* stream_tokens, int num_tokens, int n, void* lut, void* workspace, int* status,
+                               cudaStream_t stream);
+cudaError_t launch_ngram_draft(const void* lut, const int* context, const int* fill, int B, int k, int* drafts,
+                               int* has_draft, cudaStream_t stream);
+
 }  // namespace agx

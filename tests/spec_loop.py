@@ -45,6 +45,73 @@ class OracleBackend:
         return self.step(q, k, v, drafts)
 
 
+class CudaBackend:
+    """The same cache and step on the GPU: agx_kv_append, agx_attn_prefixed and agx_accept_greedy through the
+    C ABI (float32 pools); the toy model's projections around them stay in numpy."""
+
+    def __init__(self, lm, max_tokens=512, seed=5):
+        import torch
+        from paper_2605_10380_b200 import agx
+        self.torch, self.lm = torch, lm
+        self.h = agx.Handle(lm.hq, lm.hkv, lm.d, "f32")
+        n_pages = (max_tokens + 15) // 16
+        rng = np.random.default_rng(seed)
+        self.page_row = rng.permutation(n_pages + 8).astype(np.int32)[:n_pages]
+        self.page_table = torch.from_numpy(self.page_row[None, :].copy()).cuda()
+        self.k_pool = torch.zeros((n_pages + 8, lm.hkv, 16, lm.d), dtype=torch.float32, device="cuda")
+        self.v_pool = torch.zeros_like(self.k_pool)
+        self.length = 0
+
+    def run_block(self, tokens, drafts):
+        torch = self.torch
+        n, P = len(tokens), self.length
+        x = self.lm.embed(tokens, np.arange(P, P + n))
+        q, k, v = self.lm.qkv(x)
+        dq, dk, dv = (torch.from_numpy(a).cuda() for a in (q, k, v))
+        cu = torch.tensor([0, n], dtype=torch.int32, device="cuda")
+        pl = torch.tensor([P], dtype=torch.int32, device="cuda")
+        self.h.kv_append(self.k_pool, self.v_pool, dk, dv, self.page_table, pl, cu)
+        out = torch.empty_like(dq)
+        Pn, Qn = np.array([P], np.int32), np.array([n], np.int32)
+        nws = self.h.attn_workspace_bytes(Pn, Qn)
+        ws = torch.empty(max(nws, 256), dtype=torch.uint8, device="cuda") if nws else None
+        self.h.attn_prefixed(dq, self.k_pool, self.v_pool, self.page_table, Pn, Qn, out, None, ws)
+        logits = torch.from_numpy(self.lm.logits(x, out.cpu().numpy().astype(np.float64))).cuda()
+        dd = torch.tensor(list(drafts) if len(drafts) else [0], dtype=torch.int32, device="cuda")
+        acc = torch.zeros(1, dtype=torch.int32, device="cuda"); nxt = torch.zeros(1, dtype=torch.int32, device="cuda")
+        sl = pl.clone()
+        aws = torch.empty(self.h.accept_workspace_bytes(n, self.lm.vocab), dtype=torch.uint8, device="cuda")
+        self.h.accept_greedy(logits, "f32", self.lm.vocab, dd, cu, acc, nxt, None, sl, aws)
+        torch.cuda.synchronize()
+        self.length = int(sl.item())
+        return int(acc.item()), int(nxt.item())
+
+
+class DeviceNgramDrafts:
+    """Draft source on the GPU: agx_ngram_build once over the prompt, agx_ngram_draft per round
+    (Sec. 4.3, with the selective fallback)."""
+
+    def __init__(self, prompt, n=3, seed=3, vocab=512):
+        import torch
+        from paper_2605_10380_b200 import agx
+        self.torch, self.n, self.vocab = torch, n, vocab
+        self.h = agx.Handle(4, 2, 64, "f32")
+        st = torch.tensor([int(t) for t in prompt], dtype=torch.int32, device="cuda")
+        self.lut = torch.empty(agx.ngram_lut_bytes(len(prompt)), dtype=torch.uint8, device="cuda")
+        ws = torch.empty(agx.ngram_workspace_bytes(len(prompt)), dtype=torch.uint8, device="cuda")
+        self.h.ngram_build(st, n, self.lut, ws)
+        self.rng = np.random.default_rng(seed)
+
+    def __call__(self, history, k):
+        torch = self.torch
+        ctx = torch.tensor([int(t) for t in history[-(self.n - 1):]], dtype=torch.int32, device="cuda").reshape(1, self.n - 1)
+        fill = torch.from_numpy(self.rng.integers(0, self.vocab, size=(1, k)).astype(np.int32)).cuda()
+        drafts = torch.zeros((1, k), dtype=torch.int32, device="cuda")
+        has = torch.zeros(1, dtype=torch.int32, device="cuda")
+        self.h.ngram_draft(self.lut, ctx, fill, k, drafts, has)
+        return drafts[0].tolist() if has.item() else None
+
+
 def generate(backend, prompt, n_new, draft_fn=None, k=4):
     """Greedy generation.  ``draft_fn(history, k)`` returns k draft tokens or None (plain step).
     Returns (emitted tokens, number of model calls, list of accept lengths)."""

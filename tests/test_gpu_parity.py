@@ -270,6 +270,88 @@ def test_verify_step_host_matches_oracle(enqueue_only):
     assert np.array_equal(h_acc.numpy(), al) and np.array_equal(h_nxt.numpy(), nt) and np.array_equal(h_sl.numpy(), sl)
 
 
+# ------------------------------------------------------------------ n-gram draft table (Sec. 4.3)
+def _ngram_case(h, stream, n, contexts, k, fill):
+    from oracle.toy_lm import build_ngram_table, ngram_drafts
+    st = torch.tensor(stream, dtype=torch.int32, device="cuda")
+    lut = torch.empty(agx.ngram_lut_bytes(len(stream)), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(agx.ngram_workspace_bytes(len(stream)), dtype=torch.uint8, device="cuda")
+    h.ngram_build(st, n, lut, ws)
+    B = len(contexts)
+    ctx = torch.tensor(contexts, dtype=torch.int32, device="cuda").reshape(B, n - 1)
+    fl = torch.tensor(fill, dtype=torch.int32, device="cuda").reshape(B, max(k, 1))[:, :k].contiguous()
+    drafts = torch.full((B, max(k, 1)), -7, dtype=torch.int32, device="cuda")[:, :k].contiguous()
+    has = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    h.ngram_draft(lut, ctx, fl, k, drafts, has)
+    torch.cuda.synchronize()
+    table = build_ngram_table(stream, n)
+    got_d, got_h = drafts.cpu().numpy(), has.cpu().numpy()
+    for s in range(B):
+        ref = ngram_drafts(table, contexts[s], k, n, fill=fill[s])
+        if tuple(contexts[s]) not in table:
+            assert ref is None and got_h[s] == 0     # selective fallback: no verify block for this sequence
+        else:
+            assert got_h[s] == 1 and got_d[s].tolist() == ref
+    return table
+
+
+@pytest.mark.parametrize("n", [2, 3])
+def test_ngram_table_and_draft_chains_match_oracle(n):
+    h = agx.Handle(32, 8, 128, "bf16")
+    rng = np.random.default_rng(7 + n)
+    ids = rng.choice(1 << 21, size=60, replace=False)            # a small alphabet of large ids: many repeats and count ties
+    for length, alphabet in [(0, 4), (n - 1, 4), (n, 4), (37, 3), (1000, 12), (5000, 60), (120000, 60)]:
+        stream = ids[rng.integers(0, alphabet, size=length)].tolist()
+        k = 5
+        known = [list(stream[i:i + n - 1]) for i in rng.integers(0, max(length - n + 1, 1), size=40)] if length >= n else []
+        unknown = [[int(ids[59])] * (n - 1), [0] * (n - 1), [(1 << 21) - 1] * (n - 1), [-5] * (n - 1)]
+        contexts = known + unknown
+        fill = ids[rng.integers(0, alphabet, size=(len(contexts), k))].tolist()
+        table = _ngram_case(h, stream, n, contexts, k, fill)
+        if length >= 1000:   # every key of the table, one lookup each
+            keys = [list(key) for key in table]
+            _ngram_case(h, stream, n, keys, 1, [[0]] * len(keys))
+    assert h.get_status() == 0
+
+
+def test_ngram_build_flags_tokens_outside_its_range_and_skips_their_windows():
+    h = agx.Handle(32, 8, 128, "bf16")
+    stream = [5, 6, 7, 1 << 21, 5, 6, 9, -1, 5, 6, 9]
+    from oracle.toy_lm import build_ngram_table
+    st = torch.tensor(stream, dtype=torch.int32, device="cuda")
+    lut = torch.empty(agx.ngram_lut_bytes(len(stream)), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(agx.ngram_workspace_bytes(len(stream)), dtype=torch.uint8, device="cuda")
+    h.ngram_build(st, 3, lut, ws)
+    ctx = torch.tensor([[5, 6], [6, 7]], dtype=torch.int32, device="cuda")
+    fl = torch.zeros((2, 1), dtype=torch.int32, device="cuda")
+    d = torch.zeros((2, 1), dtype=torch.int32, device="cuda"); hs = torch.zeros(2, dtype=torch.int32, device="cuda")
+    h.ngram_draft(lut, ctx, fl, 1, d, hs)
+    torch.cuda.synchronize()
+    assert h.get_status() & agx.AGX_DEV_BAD_TOKEN
+    assert d[0, 0].item() == 9 and hs.tolist() == [1, 0]     # (5,6)->9 twice, ->7 once; (6,7,bad) skipped
+    with pytest.raises(agx.AgxError):
+        h.ngram_build(st, 4, lut, ws)
+
+
+def test_speculative_loop_on_gpu_emits_the_tokens_of_plain_greedy_decoding():
+    """Greedy speculative decoding (verify blocks through agx_kv_append / agx_attn_prefixed / agx_accept_greedy,
+    drafts from the device-side trigram table with its selective fallback) emits exactly the stream of
+    one-token-at-a-time greedy decoding, on the GPU and in the oracle (Sec. 2.3, Sec. 4.3)."""
+    from oracle.toy_lm import ToyLM
+    from tests.spec_loop import CudaBackend, DeviceNgramDrafts, OracleBackend, generate
+    lm = ToyLM(seed=11)
+    rng = np.random.default_rng(21)
+    motif = rng.integers(0, lm.vocab, size=12).tolist()
+    prompt = (motif * 4)[:40]
+    T = 48
+    base, calls0, _ = generate(OracleBackend(lm), prompt, T)
+    plain, calls1, _ = generate(CudaBackend(lm), prompt, T)
+    spec, calls2, acc = generate(CudaBackend(lm), prompt, T, DeviceNgramDrafts(prompt, 3, vocab=lm.vocab), k=4)
+    wrong, calls3, acc_w = generate(CudaBackend(lm), prompt, T, lambda hist, k: [(hist[-1] + 1 + i) % lm.vocab for i in range(k)], k=4)
+    assert plain == base and spec == base and wrong == base
+    assert calls1 == T and calls2 <= T and calls3 <= T
+
+
 # ------------------------------------------------------------------ argument errors (host side)
 def test_argument_errors_are_reported_not_faulted():
     w = W.make_attn_workload("err", 6, "bf16", 32, 8, 128, [100], [4])
