@@ -8,6 +8,7 @@
 // (ticket counter) folds the per-chunk keys, compares drafts and writes the results, so no second
 // launch and no host round trip is needed.
 #include "agx_internal.cuh"
+#include "agx_sm100.cuh"
 
 namespace agx {
 
@@ -50,6 +51,8 @@ accept_kernel(const void* __restrict__ logits, long long row_stride, int vocab, 
               int* __restrict__ accept_len, int* __restrict__ next_token, int* __restrict__ argmax,
               int* __restrict__ seq_lens, unsigned long long* partials, int* tokens, unsigned int* ticket) {
     constexpr int kVecElems = kBf16 ? 8 : 4;
+    pdl_launch_dependents();
+    pdl_wait();
     const int row = blockIdx.y;
     const int chunk = blockIdx.x;
     const unsigned int begin = (unsigned int)chunk * (unsigned int)chunk_elems;
@@ -159,14 +162,15 @@ cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_st
     const bool vec = ((uintptr_t)logits % 16 == 0) && ((row_stride * esz) % 16 == 0);
     int* tokens = (int*)(partials + (size_t)total_q * chunks);
     dim3 grid(chunks, total_q);
+    cudaError_t err = cudaSuccess;
 #define AGX_LAUNCH_ACCEPT(BF, VEC)                                                                              \
-    accept_kernel<BF, VEC><<<grid, 256, 0, stream>>>(logits, row_stride, vocab, chunk_elems, chunks, drafts,    \
-                                                     cu_q, B, total_q, accept_len, next_token, argmax, seq_lens, \
-                                                     partials, tokens, ticket)
+    err = launch_chained(accept_kernel<BF, VEC>, grid, dim3(256), 0, stream, logits, row_stride, vocab, chunk_elems,  \
+                         chunks, drafts, cu_q, B, total_q, accept_len, next_token, argmax, seq_lens, partials, tokens, \
+                         ticket)
     if (bf16) { if (vec) AGX_LAUNCH_ACCEPT(true, true); else AGX_LAUNCH_ACCEPT(true, false); }
     else      { if (vec) AGX_LAUNCH_ACCEPT(false, true); else AGX_LAUNCH_ACCEPT(false, false); }
 #undef AGX_LAUNCH_ACCEPT
-    return cudaGetLastError();
+    return err;
 }
 
 }  // namespace agx

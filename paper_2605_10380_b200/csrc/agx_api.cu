@@ -135,6 +135,7 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
                 const long long cost = waves * (std::min(c_tokens, round_up(max_len, unit)) / unit + 3);
                 if (best_cost < 0 || cost < best_cost) { best_cost = cost; C = c_tokens; }
             }
+            if (const char* force = getenv("AGX_TILE_SPLIT_TOKENS")) { if (atoi(force) >= unit) C = atoi(force) / unit * unit; }
             if (h->debug_plan)
                 fprintf(stderr, "agx plan: tile kernel, %lld row chunks, longest sequence %d tokens -> KV splits of %d tokens, %lld CTAs\n",
                         base_items, max_len, C, count_items(C));

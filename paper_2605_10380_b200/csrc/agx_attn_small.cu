@@ -115,6 +115,8 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&map_k) : "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&map_v) : "memory");
     }
+    pdl_launch_dependents();
+    pdl_wait();   // from here on global memory written by the launch before this one is read
     // ---- Q tile -> shared (rows beyond q*G are zero)
     for (int c = tid; c < MT * 16 * 16; c += kThreads) {
         const int r = c >> 4, ch = c & 15;
@@ -381,6 +383,8 @@ template <int D>
 __global__ void __launch_bounds__(128)
 attn_simt_f32_kernel(const __grid_constant__ AttnParams p) {
     constexpr int kPer = D / 32;
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int si = find_seq(p, blockIdx.x);
     const SeqPlan sp = p.seq[si];
@@ -456,6 +460,8 @@ attn_simt_f32_kernel(const __grid_constant__ AttnParams p) {
 template <bool kBf16Out>
 __global__ void __launch_bounds__(128)
 attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int rh = blockIdx.x * 4 + (threadIdx.x >> 5);  // index over (local row, head) of the launch's sequences
     if (rh >= total_rows * p.hq) return;
@@ -576,8 +582,7 @@ cudaError_t launch_small(const AttnParams& p, const CUtensorMap& map_k, const CU
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    attn_small_bf16_kernel<MT, KW, NS><<<p.num_items, 32 * MT * KW, kSmem, stream>>>(p, map_k, map_v);
-    return cudaGetLastError();
+    return launch_chained(attn_small_bf16_kernel<MT, KW, NS>, dim3(p.num_items), dim3(32 * MT * KW), kSmem, stream, p, map_k, map_v);
 }
 }  // namespace
 
@@ -599,19 +604,17 @@ cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, int kw, cudaStre
 
 cudaError_t launch_attn_simt_f32(const AttnParams& p, cudaStream_t stream) {
     if (p.num_items == 0) return cudaSuccess;
-    if (p.head_dim == 64) attn_simt_f32_kernel<64><<<p.num_items, 128, 0, stream>>>(p);
-    else if (p.head_dim == 128) attn_simt_f32_kernel<128><<<p.num_items, 128, 0, stream>>>(p);
-    else return cudaErrorInvalidValue;
-    return cudaGetLastError();
+    if (p.head_dim == 64) return launch_chained(attn_simt_f32_kernel<64>, dim3(p.num_items), dim3(128), 0, stream, p);
+    if (p.head_dim == 128) return launch_chained(attn_simt_f32_kernel<128>, dim3(p.num_items), dim3(128), 0, stream, p);
+    return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, cudaStream_t stream) {
     const long long n = (long long)total_rows * p.hq;
     if (n == 0) return cudaSuccess;
     const int blocks = (int)((n + 3) / 4);
-    if (dtype == AGX_BF16) attn_combine_kernel<true><<<blocks, 128, 0, stream>>>(p, total_rows);
-    else attn_combine_kernel<false><<<blocks, 128, 0, stream>>>(p, total_rows);
-    return cudaGetLastError();
+    if (dtype == AGX_BF16) return launch_chained(attn_combine_kernel<true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+    return launch_chained(attn_combine_kernel<false>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
 }
 
 }  // namespace agx

@@ -348,8 +348,10 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
     const int split = it.split, g = it.g, G = it.G, P = it.P, q = it.q, L = P + q, rows = it.rows, row0 = it.row0;
     const int kv_begin = it.kv_begin, kv_end = it.kv_end, n_tiles = it.n_tiles;
 
+    pdl_launch_dependents();
     if (n_tiles == 0) {  // nothing visible in this split (nsplit > 1 by construction): publish (m, l) = (-inf, 0);
                          // the combine kernel does not read the O rows of such entries
+        pdl_wait();
         for (int rl = tid; rl < kRowsPerCta; rl += kThreads) {
             const int r = row0 + rl;
             if (r >= rows) break;
@@ -372,6 +374,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
+    pdl_wait();   // from here on global memory written by the launch before this one is read (Q, page table, K/V)
     // Q: 256 rows x 256 B by 16-byte cp.async (all of a thread's copies in flight at once), written in
     // the 128-byte-swizzled K-major operand layout; rows past q * G are zero-filled.
     if (warp >= 2) {
@@ -757,8 +760,7 @@ cudaError_t launch_tile(const AttnParams& p, const CUtensorMap& map_k, const CUt
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    attn_tile_bf16_kernel<kStreams><<<p.num_items, kThreads, kSmemBytes, stream>>>(p, map_k, map_v);
-    return cudaGetLastError();
+    return launch_chained(attn_tile_bf16_kernel<kStreams>, dim3(p.num_items), dim3(kThreads), kSmemBytes, stream, p, map_k, map_v);
 }
 }  // namespace
 

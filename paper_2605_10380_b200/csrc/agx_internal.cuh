@@ -44,6 +44,22 @@ struct AttnParams {
     SeqPlan seq[kMaxSeqs];
 };
 
+// Launch with programmatic stream serialisation: the kernel may start while the launch before it in the
+// stream is still draining, so its launch latency and set-up overlap that kernel's tail.  Every kernel
+// launched this way calls pdl_wait() before its first global-memory access.  AGX_NO_PDL=1 turns it off.
+bool pdl_enabled();
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Launchers (each returns the cudaError_t of its launch).
 cudaError_t launch_kv_append(int dtype, void* k_pool, void* v_pool, long long num_pages, const void* k_new,
                              const void* v_new, const int* page_table, int pt_stride, const int* prefix_len,

@@ -4,7 +4,10 @@
 // HBM-bound copy: 2 * 2 * rows * Hkv * d * elem bytes (read + write, K and V).  One thread moves
 // 16 bytes of K and 16 bytes of V; a (token, kv head) row is `vec_per_row` consecutive threads, so
 // loads and stores are fully coalesced 128-bit accesses.
+#include <stdlib.h>
+
 #include "agx_internal.cuh"
+#include "agx_sm100.cuh"
 
 namespace agx {
 
@@ -13,6 +16,8 @@ kv_append_kernel(uint4* __restrict__ k_pool, uint4* __restrict__ v_pool, long lo
                  const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
                  const int* __restrict__ page_table, int pt_stride, const int* __restrict__ prefix_len,
                  const int* __restrict__ cu_q, int B, int total_q, int hkv, int vec_per_row, int* status) {
+    pdl_launch_dependents();
+    pdl_wait();
     const long long n_vec = (long long)total_q * hkv * vec_per_row;
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < n_vec;
          idx += (long long)gridDim.x * blockDim.x) {
@@ -51,10 +56,14 @@ cudaError_t launch_kv_append(int dtype, void* k_pool, void* v_pool, long long nu
     if (n_vec == 0) return cudaSuccess;
     long long blocks = (n_vec + 255) / 256;
     if (blocks > 148 * 8) blocks = 148 * 8;
-    kv_append_kernel<<<(int)blocks, 256, 0, stream>>>((uint4*)k_pool, (uint4*)v_pool, num_pages, (const uint4*)k_new,
-                                                      (const uint4*)v_new, page_table, pt_stride, prefix_len, cu_q,
-                                                      B, total_q, hkv, vec_per_row, status);
-    return cudaGetLastError();
+    return launch_chained(kv_append_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, (uint4*)k_pool, (uint4*)v_pool, num_pages,
+                          (const uint4*)k_new, (const uint4*)v_new, page_table, pt_stride, prefix_len, cu_q, B, total_q, hkv,
+                          vec_per_row, status);
+}
+
+bool pdl_enabled() {
+    static const bool on = [] { const char* e = getenv("AGX_NO_PDL"); return !(e && atoi(e) != 0); }();
+    return on;
 }
 
 }  // namespace agx
