@@ -301,6 +301,46 @@ def extra_workloads(torch, agx, W, peaks, steps, warmup):
         torch.cuda.empty_cache()
     except Exception as e:  # keep the headline line alive
         out["c5_long_context_verify"] = {"error": repr(e)}
+    # accept step alone: one read of the logits; 64 distinct buffers rotated inside one graph so they come from HBM
+    try:
+        acc = {}
+        for name, q_list in (("c2_accept_8x128256", [8]), ("c5_accept_32x128256", [8] * 4)):
+            h = agx.Handle(32, 8, 128, "bf16")
+            rows, B, V = sum(q_list), len(q_list), 128256
+            bufs = [torch.randn(rows, V, device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(64)]
+            drafts = torch.randint(0, V, (max(rows - B, 1),), device="cuda", dtype=torch.int32)
+            cu = torch.from_numpy(W.cu_from_q(q_list)).cuda()
+            al = torch.zeros(B, dtype=torch.int32, device="cuda"); nt = torch.zeros(B, dtype=torch.int32, device="cuda")
+            ws = torch.empty(h.accept_workspace_bytes(rows, V), dtype=torch.uint8, device="cuda")
+
+            def run():
+                for x in bufs:
+                    h.accept_greedy(x, "bf16", V, drafts, cu, al, nt, None, None, ws)
+            g = capture(torch, run)
+            ms = time_graph(torch, g, max(steps // 10, 10), max(warmup, 3)) / len(bufs)
+            by = rows * V * 2
+            acc[name] = {"us": ms * 1e3, "GB/s": by / (ms * 1e-3) / 1e9, "frac_of_measured_hbm": by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                         "roofline_us": by / peaks["hbm_gbs"] / 1e3}
+            del bufs, g
+            torch.cuda.empty_cache()
+        out["accept_step"] = acc
+    except Exception as e:
+        out["accept_step"] = {"error": repr(e)}
+    # KV append alone: the 512-token suffix of the prefill config (1 MB of K and of V, read + write)
+    try:
+        lv = LayeredVerify(torch, agx, W, [3072], [512], 24, 8, 128, 8, 0, 13)
+
+        def run_append():
+            for l in range(lv.layers):
+                lv.h.kv_append(lv.k_pools[l], lv.v_pools[l], lv.k_new[l], lv.v_new[l], lv.page_table, lv.prefix_dev, lv.cu_dev)
+        g = capture(torch, run_append)
+        ms = time_graph(torch, g, max(steps // 10, 10), max(warmup, 3)) / lv.layers
+        by = 2 * 2 * 512 * 8 * 128 * 2
+        out["kv_append_512_tokens"] = {"us": ms * 1e3, "GB/s": by / (ms * 1e-3) / 1e9}
+        del lv, g
+        torch.cuda.empty_cache()
+    except Exception as e:
+        out["kv_append_512_tokens"] = {"error": repr(e)}
     # multi-token tax: one attention call verifying q = 8 tokens against decoding q = 1 over the same context
     # (the paper measures 1.86x for q = 2 with its stock attention; the point of the small-q kernels is ~1.0)
     try:

@@ -341,7 +341,7 @@ agx_status agx_attn_prefixed(agx_handle* h, const void* q_block, const void* k_p
 
 static int accept_chunks(const agx_handle* h, int total_q, int vocab, int dtype) {
     const int vec = 16 / elem_size(dtype);
-    const int target = 2 * h->sm_count;
+    const int target = 8 * h->sm_count;   // enough CTAs that every thread needs a single trip of two 16-byte loads
     int want = std::max(1, (target + total_q - 1) / total_q);
     const int max_chunks = std::max(1, (vocab + 256 * vec * 2 - 1) / (256 * vec * 2));  // >= 2 vectors per thread
     want = std::min(want, max_chunks);
