@@ -163,7 +163,7 @@ class Handle:
     def close(self):
         if getattr(self, "_h", None) and self._h.value:
             self._lib.agx_destroy(self._h)
-            self._h = ctypes.c_void_p()
+            self._h = None   # (at interpreter shutdown the ctypes module may already be gone)
 
     __del__ = close
 

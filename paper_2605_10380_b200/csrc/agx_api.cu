@@ -489,9 +489,18 @@ static agx_status verify_step_host_impl(agx_handle* h, void* k_pool, void* v_poo
         h2d(L.logits, h_logits, L.logits_bytes);
         h2d(L.drafts, h_drafts, (size_t)(L.total_q - B) * 4);
     }
-    h2d(L.prefix, P, (size_t)B * 4);
-    h2d(L.seqlen, P, (size_t)B * 4);
-    h2d(L.cu, cu.data(), (size_t)(B + 1) * 4);
+    if (B <= kMaxSeqs) {   // as kernel arguments: no pageable copies, which would each synchronise the stream first
+        StepMeta meta;
+        meta.B = B;
+        for (int s = 0; s < B; ++s) { meta.prefix[s] = P[s]; meta.cu[s] = cu[s]; }
+        meta.cu[B] = cu[B];
+        if (e == cudaSuccess)
+            e = launch_write_meta(meta, (int*)(ws + L.prefix), (int*)(ws + L.seqlen), (int*)(ws + L.cu), stream);
+    } else {
+        h2d(L.prefix, P, (size_t)B * 4);
+        h2d(L.seqlen, P, (size_t)B * 4);
+        h2d(L.cu, cu.data(), (size_t)(B + 1) * 4);
+    }
     if (e != cudaSuccess) return cuda_fail(h, e, "host step: upload");
     int launches = 0;
     st = agx_kv_append(h, k_pool, v_pool, num_pages, ws + L.k, ws + L.v, page_table, pt_stride,

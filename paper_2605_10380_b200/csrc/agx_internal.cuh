@@ -60,6 +60,14 @@ cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// Lengths of a batch of at most kMaxSeqs sequences, passed to write_meta_kernel by value.
+struct StepMeta {
+    int B;
+    int prefix[kMaxSeqs];
+    int cu[kMaxSeqs + 1];
+};
+cudaError_t launch_write_meta(const StepMeta& m, int* prefix, int* seq_lens, int* cu_q, cudaStream_t stream);
+
 // Launchers (each returns the cudaError_t of its launch).
 cudaError_t launch_kv_append(int dtype, void* k_pool, void* v_pool, long long num_pages, const void* k_new,
                              const void* v_new, const int* page_table, int pt_stride, const int* prefix_len,

@@ -61,6 +61,20 @@ cudaError_t launch_kv_append(int dtype, void* k_pool, void* v_pool, long long nu
                           vec_per_row, status);
 }
 
+// Lengths of a small batch travel as kernel arguments instead of three pageable host-to-device copies (each
+// of which would first synchronise the stream): prefix_len, the committed lengths and the row offsets.
+__global__ void write_meta_kernel(const __grid_constant__ StepMeta m, int* prefix, int* seq_lens, int* cu_q) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int i = threadIdx.x;
+    if (i < m.B) { prefix[i] = m.prefix[i]; seq_lens[i] = m.prefix[i]; }
+    if (i <= m.B) cu_q[i] = m.cu[i];
+}
+
+cudaError_t launch_write_meta(const StepMeta& m, int* prefix, int* seq_lens, int* cu_q, cudaStream_t stream) {
+    return launch_chained(write_meta_kernel, dim3(1), dim3(64), 0, stream, m, prefix, seq_lens, cu_q);
+}
+
 bool pdl_enabled() {
     static const bool on = [] { const char* e = getenv("AGX_NO_PDL"); return !(e && atoi(e) != 0); }();
     return on;
