@@ -35,9 +35,11 @@ if ROOT not in sys.path:
 METRIC = "prefix-cached attn query tok/s"
 UNIT = "query tok/s (per attention-layer call)"
 C2 = dict(P=4096, q=8, hq=32, hkv=8, d=128, vocab=128256, layers=32)
-# DRAM bytes of one attention call of this workload (attention kernel 16,957,696 + combine kernel 2,304,768), from the
+WORKLOAD = ("decode verification (c2): batch 1, cached context 4096, q=8, GQA 32/8, d=128, bf16, "
+            "page 16 shuffled, 32 per-layer KV pools + accept on bf16 logits [8,128256]")
+# DRAM bytes of one attention call of this workload (attention kernel 16,957,696 + combine kernel 2,305,280), from the
 # ncu capture summarised under profiles/; set to None whenever one of the two kernels changes until it is re-captured
-NCU_TRAFFIC_BYTES = 16957696 + 2304768
+NCU_TRAFFIC_BYTES = 16957696 + 2305280
 
 
 # --------------------------------------------------------------------------- peaks / clocks
@@ -276,7 +278,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "decode verification (c2): P=4096 q=8 GQA 32/8 d=128 bf16 storage", "sample": sample},
+            "config": {"workload": WORKLOAD, "sample": sample},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -461,8 +463,7 @@ def run_agx(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": "decode verification (c2): batch 1, cached context 4096, q=8, GQA 32/8, d=128, bf16, "
-                               "page 16 shuffled, 32 per-layer KV pools + accept on bf16 logits [8,128256]",
+        "config": {"workload": WORKLOAD,
                    "step": "32 x (agx_kv_append + agx_attn_prefixed) + 1 x agx_accept_greedy, one CUDA graph",
                    "l2": "inputs larger than L2: 32 distinct layer pools = 553 MB, each read once per step",
                    "parallelism": f"{world} independent replica(s), no collective"},
