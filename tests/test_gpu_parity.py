@@ -241,6 +241,48 @@ def test_accept_many_rows_and_unaligned_rows():
         assert np.array_equal(g, r)
 
 
+# ------------------------------------------------------------------ invariants of the definition, on the GPU
+def _attend(w):
+    b = DeviceBatch(w); b.append(); out, lse = b.attend()
+    assert b.status() == 0
+    return out, lse
+
+
+@pytest.mark.parametrize("P,q", [(700, 8), (9000, 8), (1500, 200)])
+def test_gpu_output_is_unchanged_by_a_joint_permutation_of_the_cached_prefix(P, q):
+    """No positional term inside the library: shuffling the cached prefix's (K, V) tokens together leaves every
+    output row unchanged up to summation order (small-q, stream and tile kernels)."""
+    w = W.make_attn_workload("perm", 71, "bf16", 32, 8, 128, [P], [q])
+    a, lse_a = _attend(w)
+    K = W.gather_contiguous(w.k_pool, w.page_table[0], P); V = W.gather_contiguous(w.v_pool, w.page_table[0], P)
+    perm = np.random.default_rng(5).permutation(P)
+    w2 = W.make_attn_workload("perm", 71, "bf16", 32, 8, 128, [P], [q])
+    W.scatter_contiguous(w2.k_pool, w2.page_table[0], 0, K[perm]); W.scatter_contiguous(w2.v_pool, w2.page_table[0], 0, V[perm])
+    b, lse_b = _attend(w2)
+    assert np.max(np.abs(a - b)) <= 4e-3 and np.max(np.abs(lse_a - lse_b)) <= 1e-3
+
+
+def test_gpu_gqa_equals_mha_with_replicated_kv_heads_and_ignores_pages_beyond_the_sequence():
+    w = W.make_attn_workload("gqa", 72, "bf16", 8, 2, 128, [1000], [8], spare_pages=9)
+    a, _ = _attend(w)
+    rep = lambda x: np.repeat(x, 4, axis=1)
+    w2 = W.AttnWorkload("mha", "bf16", 8, 8, 128, w.prefix_len, w.q_len, w.cu_q, w.page_table, w.num_pages,
+                        rep(w.k_pool), rep(w.v_pool), w.q_block, rep(w.k_new), rep(w.v_new))
+    b, _ = _attend(w2)
+    assert np.array_equal(a, b)   # same kernel, same per-head arithmetic
+    # a longer page table whose extra entries point at pages full of NaN changes nothing
+    w3 = W.make_attn_workload("gqa", 72, "bf16", 8, 2, 128, [1000], [8], spare_pages=9)
+    table = np.full((1, w3.page_table.shape[1] + 4), -1, dtype=np.int32)
+    table[0, :w3.page_table.shape[1]] = w3.page_table[0]
+    used = set(w3.page_table[0].tolist())
+    spare = [pg for pg in range(w3.num_pages) if pg not in used][:4]
+    table[0, w3.page_table.shape[1]:] = spare
+    w3.k_pool[spare] = 0x7FC0; w3.v_pool[spare] = 0x7FC0
+    w3.page_table = table
+    c, _ = _attend(w3)
+    assert np.array_equal(a, c)
+
+
 # ------------------------------------------------------------------ whole step from host buffers
 @pytest.mark.parametrize("enqueue_only", [False, True])
 def test_verify_step_host_matches_oracle(enqueue_only):
