@@ -68,7 +68,7 @@ __global__ void ngram_count_kernel(const int* __restrict__ stream, int num_token
 }
 
 __global__ void ngram_select_kernel(const unsigned long long* __restrict__ win_keys, const unsigned int* __restrict__ win_counts,
-                                    unsigned int win_capacity, LutHeader* hdr, LutSlot* lut, unsigned int lut_capacity) {
+                                    unsigned int win_capacity, LutSlot* lut, unsigned int lut_capacity) {
     for (unsigned int s = blockIdx.x * blockDim.x + threadIdx.x; s < win_capacity; s += gridDim.x * blockDim.x) {
         const unsigned long long key = win_keys[s];
         if (key == kEmpty) continue;
@@ -161,7 +161,7 @@ cudaError_t launch_ngram_build(const int* stream_tokens, int num_tokens, int n, 
         const int blocks = (windows + 255) / 256 < 1184 ? (windows + 255) / 256 : 1184;
         ngram_count_kernel<<<blocks, 256, 0, stream>>>(stream_tokens, num_tokens, n, win_keys, win_counts, cap, status);
         const int blocks2 = (int)((cap + 255) / 256 < 1184 ? (cap + 255) / 256 : 1184);
-        ngram_select_kernel<<<blocks2, 256, 0, stream>>>(win_keys, win_counts, cap, hdr, slots, cap);
+        ngram_select_kernel<<<blocks2, 256, 0, stream>>>(win_keys, win_counts, cap, slots, cap);
     }
     return cudaGetLastError();
 }
