@@ -313,6 +313,48 @@ AGX_API agx_status agx_ngram_draft(agx_handle* handle, const void* lut, const in
                                    const int32_t* fill, int32_t B, int32_t k, int32_t* drafts,
                                    int32_t* has_draft, void* stream);
 
+/*
+ * agx_pw_select_combinations - which cluster combinations to precompute (Algorithm 1, Sec. 4.2).  HOST code.
+ * A sample is the ordered sequence of clusters a training query activates.  The coverage of a cached set
+ * is, summed over samples, the length of the longest prefix of the sample that is cached.  Starting from
+ * the empty set, `budget` times the candidate that raises the coverage most is added; candidates are the
+ * samples' prefixes that are a single cluster or a cached sequence extended by one cluster.  Equal gains
+ * (the paper is silent): the shorter candidate, then the lexicographically smaller one.  The selection
+ * ends early when no candidate is left.
+ *   samples      : host int32 [num_samples][max_len], cluster ids >= 0, rows padded with -1
+ *   selected     : host int32 [budget][max_len] (written, padded with -1), in the order of selection
+ *   selected_len : host int32 [budget]; gains : host int32 [budget] or NULL (coverage gained by each step)
+ *   num_selected : host int32 (written)
+ * Errors: AGX_E_INVAL.
+ */
+AGX_API agx_status agx_pw_select_combinations(const int32_t* samples, int32_t num_samples, int32_t max_len,
+                                              int32_t budget, int32_t* selected, int32_t* selected_len,
+                                              int32_t* gains, int32_t* num_selected);
+
+/*
+ * agx_pw_longest_prefix - online lookup with tail cut (Sec. 4.2).  HOST code.
+ * Among the stored combinations, the one that shares the longest run of leading clusters with the query;
+ * the stored combination may go on after the run (its tail is cut off: only the KV of the run is reused).
+ * Equal runs: the first stored combination.  *index = -1, *length = 0 when nothing matches.
+ *   stored : host int32 [num_stored][max_len]; stored_len : host int32 [num_stored]; query : host int32 [query_len]
+ */
+AGX_API agx_status agx_pw_longest_prefix(const int32_t* stored, const int32_t* stored_len, int32_t num_stored,
+                                         int32_t max_len, const int32_t* query, int32_t query_len,
+                                         int32_t* index, int32_t* length);
+
+/*
+ * agx_kv_copy_pages - private copies of KV pages.  Sec. 4.2: a reused prefix may be cut anywhere (the
+ * mismatched tail of a stored combination is dropped), so its last page can be partly valid and still
+ * shared with other sequences; a sequence that appends behind the cut needs that page for itself.  The
+ * caller points the first prefix_len / 16 entries of the new page-table row at the stored pages, copies
+ * page prefix_len / 16 with this call when prefix_len % 16 != 0, and uses fresh pages after it.
+ *   k_pool, v_pool : device pools (pages dst[i] are overwritten with pages src[i], K and V, all heads)
+ *   src, dst       : device int32 [count]; ids outside [0, num_pages) set AGX_DEV_BAD_PAGE and are skipped
+ * Errors: AGX_E_INVAL, AGX_E_CUDA.
+ */
+AGX_API agx_status agx_kv_copy_pages(agx_handle* handle, void* k_pool, void* v_pool, int64_t num_pages,
+                                     const int32_t* src, const int32_t* dst, int32_t count, void* stream);
+
 /* Number of kernels the last agx_attn_prefixed / agx_accept_greedy / agx_kv_append call on this
  * handle launched (for launch accounting in benchmarks). */
 AGX_API int32_t agx_last_launch_count(const agx_handle* handle);

@@ -27,6 +27,7 @@ EXPORTS = (
     "agx_accept_greedy", "agx_get_status", "agx_last_launch_count",
     "agx_verify_step_host_workspace_bytes", "agx_verify_step_host", "agx_verify_step_host_enqueue",
     "agx_accept_greedy_static", "agx_ngram_lut_bytes", "agx_ngram_workspace_bytes", "agx_ngram_build", "agx_ngram_draft",
+    "agx_pw_select_combinations", "agx_pw_longest_prefix", "agx_kv_copy_pages",
 )
 
 
@@ -48,6 +49,40 @@ def ngram_lut_bytes(max_stream_tokens: int) -> int:
 
 def ngram_workspace_bytes(stream_tokens: int) -> int:
     return int(load().agx_ngram_workspace_bytes(int(stream_tokens)))
+
+
+def pw_select_combinations(samples, budget: int):
+    """samples: list of cluster-id sequences.  Returns (list of selected tuples in order, list of gains)."""
+    lib = load()
+    n = len(samples)
+    max_len = max([len(s) for s in samples] + [1])
+    arr = np.full((max(n, 1), max_len), -1, dtype=np.int32)
+    for i, s in enumerate(samples):
+        arr[i, :len(s)] = np.asarray(s, dtype=np.int32)
+    sel = np.full((max(budget, 1), max_len), -1, dtype=np.int32)
+    sel_len = np.zeros(max(budget, 1), dtype=np.int32); gains = np.zeros(max(budget, 1), dtype=np.int32)
+    cnt = ctypes.c_int32(0)
+    st = lib.agx_pw_select_combinations(_ptr(arr), n, max_len, int(budget), _ptr(sel), _ptr(sel_len), _ptr(gains), ctypes.byref(cnt))
+    if st != AGX_OK:
+        raise AgxError(st, "agx_pw_select_combinations")
+    k = int(cnt.value)
+    return [tuple(int(c) for c in sel[i, :sel_len[i]]) for i in range(k)], gains[:k].tolist()
+
+
+def pw_longest_prefix(stored, query):
+    """stored: list of cluster-id sequences; query: one sequence.  Returns (index, length)."""
+    lib = load()
+    max_len = max([len(s) for s in stored] + [1])
+    arr = np.full((max(len(stored), 1), max_len), -1, dtype=np.int32)
+    lens = np.zeros(max(len(stored), 1), dtype=np.int32)
+    for i, s in enumerate(stored):
+        arr[i, :len(s)] = np.asarray(s, dtype=np.int32); lens[i] = len(s)
+    q = np.asarray(list(query) if len(query) else [0], dtype=np.int32)
+    idx, ln = ctypes.c_int32(0), ctypes.c_int32(0)
+    st = lib.agx_pw_longest_prefix(_ptr(arr), _ptr(lens), len(stored), max_len, _ptr(q), len(query), ctypes.byref(idx), ctypes.byref(ln))
+    if st != AGX_OK:
+        raise AgxError(st, "agx_pw_longest_prefix")
+    return int(idx.value), int(ln.value)
 
 
 def lib_path() -> Path:
@@ -105,6 +140,12 @@ def load() -> ctypes.CDLL:
     lib.agx_ngram_build.restype = i32
     lib.agx_ngram_draft.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp]
     lib.agx_ngram_draft.restype = i32
+    lib.agx_pw_select_combinations.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
+    lib.agx_pw_select_combinations.restype = i32
+    lib.agx_pw_longest_prefix.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
+    lib.agx_pw_longest_prefix.restype = i32
+    lib.agx_kv_copy_pages.argtypes = [vp, vp, vp, i64, vp, vp, i32, vp]
+    lib.agx_kv_copy_pages.restype = i32
     _lib = lib
     return lib
 
@@ -220,6 +261,12 @@ class Handle:
                                          _ptr(next_token), _ptr(argmax), _ptr(seq_lens), _ptr(workspace), ws_bytes,
                                          _stream_ptr(stream))
         self._check(st, "agx_accept_greedy")
+
+    # -- agx_kv_copy_pages (src, dst: device int32 tensors)
+    def kv_copy_pages(self, k_pool, v_pool, src, dst, stream=None):
+        st = self._lib.agx_kv_copy_pages(self._h, _ptr(k_pool), _ptr(v_pool), int(k_pool.shape[0]), _ptr(src), _ptr(dst),
+                                         int(src.numel()), _stream_ptr(stream))
+        self._check(st, "agx_kv_copy_pages")
 
     # -- agx_ngram_build / agx_ngram_draft (device int32 tensors; lut and workspace are uint8 tensors)
     def ngram_build(self, stream_tokens, n: int, lut, workspace, stream=None):

@@ -595,4 +595,19 @@ agx_status agx_ngram_draft(agx_handle* h, const void* lut, const int32_t* contex
     return AGX_OK;
 }
 
+agx_status agx_kv_copy_pages(agx_handle* h, void* k_pool, void* v_pool, int64_t num_pages, const int32_t* src,
+                             const int32_t* dst, int32_t count, void* stream) {
+    if (!h) return AGX_E_INVAL;
+    h->last_launches = 0;
+    if (count < 0) return fail(h, AGX_E_INVAL, "negative count");
+    if (count == 0) return AGX_OK;
+    if (!k_pool || !v_pool || !src || !dst || num_pages < 1) return fail(h, AGX_E_INVAL, "null pointer or no pages");
+    if (!aligned(k_pool, 16) || !aligned(v_pool, 16)) return fail(h, AGX_E_INVAL, "pools must be 16-byte aligned");
+    cudaError_t e = launch_copy_pages(h->cfg.dtype, k_pool, v_pool, num_pages, src, dst, count, h->cfg.num_kv_heads,
+                                      h->cfg.head_dim, h->d_status, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "page copy");
+    h->last_launches = 1;
+    return AGX_OK;
+}
+
 }  // extern "C"

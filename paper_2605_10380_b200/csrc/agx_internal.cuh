@@ -93,6 +93,10 @@ cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_st
                           int* seq_lens, unsigned long long* partials, int chunks, unsigned int* ticket,
                           cudaStream_t stream);
 
+// Private copies of KV pages (a reused prefix that is cut inside a page, Sec. 4.2).
+cudaError_t launch_copy_pages(int dtype, void* k_pool, void* v_pool, long long num_pages, const int* src, const int* dst,
+                              int count, int hkv, int head_dim, int* status, cudaStream_t stream);
+
 // n-gram draft table (Sec. 4.3): sizes, build (three memsets + three small kernels) and chained lookups.
 long long ngram_lut_bytes(int max_stream_tokens);
 long long ngram_workspace_bytes(int stream_tokens);

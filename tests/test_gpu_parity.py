@@ -283,6 +283,50 @@ def test_gpu_gqa_equals_mha_with_replicated_kv_heads_and_ignores_pages_beyond_th
     assert np.array_equal(a, c)
 
 
+# ------------------------------------------------------------------ reusing a stored prefix that is cut inside a page
+def test_prefix_reuse_with_tail_cut_shares_full_pages_and_copies_the_cut_page():
+    """Sec. 4.2: a request matches only the leading part of a stored combination, so the reused KV ends in the
+    middle of a page.  The new sequence shares the full pages, gets a private copy of the cut page
+    (agx_kv_copy_pages), appends its own block behind the cut, and must see exactly prefix + block; the stored
+    sequence's pages are untouched."""
+    P_stored, P_cut, q = 200, 37 * 3 + 5, 24            # cut at token 116: 7 full pages shared, page 7 copied
+    w = W.make_attn_workload("stored", 81, "bf16", 32, 8, 128, [P_stored], [q], spare_pages=12)
+    h = agx.Handle(32, 8, 128, "bf16")
+    k_pool, v_pool = dev(w.k_pool, "bf16"), dev(w.v_pool, "bf16")
+    k_before = host_storage(k_pool, "bf16").copy()
+    stored_row = w.page_table[0]
+    used = set(stored_row.tolist())
+    fresh = [pg for pg in range(w.num_pages) if pg not in used]
+    n_full = P_cut // 16
+    new_row = np.full(stored_row.shape[0], -1, dtype=np.int32)
+    new_row[:n_full] = stored_row[:n_full]                           # shared, read only
+    need = (P_cut + q + 15) // 16 - n_full
+    new_row[n_full:n_full + need] = fresh[:need]
+    h.kv_copy_pages(k_pool, v_pool, dev(np.array([stored_row[n_full]], np.int32)), dev(np.array([new_row[n_full]], np.int32)))
+    table = dev(new_row[None, :].copy())
+    h.kv_append(k_pool, v_pool, dev(w.k_new, "bf16"), dev(w.v_new, "bf16"), table, dev(np.array([P_cut], np.int32)),
+                dev(np.array([0, q], np.int32)))
+    out = torch.zeros((q, 32, 128), dtype=torch.bfloat16, device="cuda")
+    Pn, Qn = np.array([P_cut], np.int32), np.array([q], np.int32)
+    n = h.attn_workspace_bytes(Pn, Qn)
+    ws = torch.empty(max(n, 256), dtype=torch.uint8, device="cuda") if n else None
+    h.attn_prefixed(dev(w.q_block, "bf16"), k_pool, v_pool, table, Pn, Qn, out, None, ws)
+    torch.cuda.synchronize()
+    assert h.get_status() == 0
+    # oracle: contiguous K/V = the first P_cut tokens of the stored sequence, then the block
+    K = np.concatenate([W.gather_contiguous(w.k_pool, stored_row, P_cut), w.k_new])
+    V = np.concatenate([W.gather_contiguous(w.v_pool, stored_row, P_cut), w.v_new])
+    ref, _, _ = oracle.attn_contiguous(w.q_block, K, V, "bf16", P_cut)
+    check_attention(out.to(torch.float64).cpu().numpy(), ref, "tail cut")
+    k_after = host_storage(k_pool, "bf16")
+    assert np.array_equal(k_after[stored_row[:(P_stored + 15) // 16]], k_before[stored_row[:(P_stored + 15) // 16]])
+    assert np.array_equal(k_after[new_row[n_full], :, :P_cut % 16], k_before[stored_row[n_full], :, :P_cut % 16])
+    # bad page ids are flagged, not followed
+    h.kv_copy_pages(k_pool, v_pool, dev(np.array([w.num_pages + 3], np.int32)), dev(np.array([0], np.int32)))
+    torch.cuda.synchronize()
+    assert h.get_status() & agx.AGX_DEV_BAD_PAGE
+
+
 # ------------------------------------------------------------------ whole step from host buffers
 @pytest.mark.parametrize("enqueue_only", [False, True])
 def test_verify_step_host_matches_oracle(enqueue_only):
