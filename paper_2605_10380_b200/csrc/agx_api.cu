@@ -22,7 +22,7 @@ struct agx_handle {
     int force_mma_sync;     // route large q through the mma.sync kernel (env AGX_FORCE_MMA_SYNC)
     int debug_plan;         // print launch plans to stderr (env AGX_DEBUG_PLAN)
     int small_kw;           // pages per pipeline stage of the warp-MMA kernel, 4 or 8 (env AGX_SMALL_KW)
-    int stream_min_tokens;  // context length from which blocks of <= 64 rows take the tensor-core stream schedule (env AGX_STREAM_MIN_TOKENS)
+    int stream_min_tokens;  // context length from which blocks of <= 32 rows take the tensor-core stream schedule (env AGX_STREAM_MIN_TOKENS)
     std::vector<int32_t> cu_host;  // staging for agx_verify_step_host (lives until its final sync)
     char err[512];
 };
@@ -84,9 +84,10 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
         else {
             const int rows = Q[s] * G;
             const bool tile_ok = !h->force_mma_sync && attn_tile_available();
-            // up to 128 rows over a long context: one Q tile per CTA, KV tiles alternating between two softmax
-            // warpgroups (HBM-bound streaming on the tcgen05 pipe); short contexts stay with the warp-MMA kernel
-            if (tile_ok && rows <= 128 && (rows > kSmallRowsMax || P[s] + Q[s] >= h->stream_min_tokens)) k = KIND_STREAM;
+            // up to 128 rows: one Q tile per CTA, KV tiles alternating between two softmax warpgroups (HBM-bound
+            // streaming on the tcgen05 pipe); blocks of at most 32 rows over short contexts stay with the warp-MMA
+            // kernel, whose start-up is shorter (measured cross-over: 8k-16k tokens at 32 rows, none above 32 rows)
+            if (tile_ok && rows <= 128 && (rows > 32 || P[s] + Q[s] >= h->stream_min_tokens)) k = KIND_STREAM;
             else if (rows <= 16) k = KIND_SMALL1;
             else if (rows <= 32) k = KIND_SMALL2;
             else if (rows <= kSmallRowsMax || h->force_mma_sync || !attn_tile_available()) k = KIND_SMALL4;
@@ -222,7 +223,7 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     env = getenv("AGX_FORCE_MMA_SYNC");
     h->force_mma_sync = env ? atoi(env) : 0;
     env = getenv("AGX_STREAM_MIN_TOKENS");
-    h->stream_min_tokens = env ? atoi(env) : 8192;
+    h->stream_min_tokens = env ? atoi(env) : 12288;
     env = getenv("AGX_SMALL_KW");
     h->small_kw = (env && atoi(env) == 4) ? 4 : 8;
     env = getenv("AGX_DEBUG_PLAN");
