@@ -355,6 +355,26 @@ AGX_API agx_status agx_pw_longest_prefix(const int32_t* stored, const int32_t* s
 AGX_API agx_status agx_kv_copy_pages(agx_handle* handle, void* k_pool, void* v_pool, int64_t num_pages,
                                      const int32_t* src, const int32_t* dst, int32_t count, void* stream);
 
+/*
+ * agx_kv_import_pages - bring precomputed KV pages from host memory into the pool.
+ * Sec. 4.2 / Sec. 5.1: the KV caches of the static prefix and of the selected cluster combinations are computed
+ * once, kept in storage and loaded when a request reuses them (the paper loads from SSD into unified
+ * memory; here the stored pages sit in host memory and cross to the GPU).  Two host-to-device copies into
+ * a staging area and one scatter kernel, all on `stream`: issued on a stream of its own, an import
+ * overlaps attention that runs on other streams over pages already resident.
+ *   h_k_pages, h_v_pages : HOST, [count][num_kv_heads][16][head_dim] of the handle's element type (pinned
+ *                          memory makes the copies asynchronous)
+ *   dst_pages            : device int32 [count]: pool page that receives imported page i; ids outside
+ *                          [0, num_pages) set AGX_DEV_BAD_PAGE and are skipped
+ *   staging              : device, >= agx_kv_import_staging_bytes(count) bytes, 16-byte aligned; busy until the
+ *                          scatter kernel has run
+ * Errors: AGX_E_INVAL, AGX_E_CUDA.
+ */
+AGX_API int64_t agx_kv_import_staging_bytes(const agx_handle* handle, int32_t count);
+AGX_API agx_status agx_kv_import_pages(agx_handle* handle, void* k_pool, void* v_pool, int64_t num_pages,
+                                       const void* h_k_pages, const void* h_v_pages, const int32_t* dst_pages,
+                                       int32_t count, void* staging, size_t staging_bytes, void* stream);
+
 /* Number of kernels the last agx_attn_prefixed / agx_accept_greedy / agx_kv_append call on this
  * handle launched (for launch accounting in benchmarks). */
 AGX_API int32_t agx_last_launch_count(const agx_handle* handle);

@@ -28,6 +28,7 @@ EXPORTS = (
     "agx_verify_step_host_workspace_bytes", "agx_verify_step_host", "agx_verify_step_host_enqueue",
     "agx_accept_greedy_static", "agx_ngram_lut_bytes", "agx_ngram_workspace_bytes", "agx_ngram_build", "agx_ngram_draft",
     "agx_pw_select_combinations", "agx_pw_longest_prefix", "agx_kv_copy_pages",
+    "agx_kv_import_staging_bytes", "agx_kv_import_pages",
 )
 
 
@@ -146,6 +147,10 @@ def load() -> ctypes.CDLL:
     lib.agx_pw_longest_prefix.restype = i32
     lib.agx_kv_copy_pages.argtypes = [vp, vp, vp, i64, vp, vp, i32, vp]
     lib.agx_kv_copy_pages.restype = i32
+    lib.agx_kv_import_staging_bytes.argtypes = [vp, i32]
+    lib.agx_kv_import_staging_bytes.restype = i64
+    lib.agx_kv_import_pages.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, vp, ctypes.c_size_t, vp]
+    lib.agx_kv_import_pages.restype = i32
     _lib = lib
     return lib
 
@@ -267,6 +272,16 @@ class Handle:
         st = self._lib.agx_kv_copy_pages(self._h, _ptr(k_pool), _ptr(v_pool), int(k_pool.shape[0]), _ptr(src), _ptr(dst),
                                          int(src.numel()), _stream_ptr(stream))
         self._check(st, "agx_kv_copy_pages")
+
+    # -- agx_kv_import_pages (h_k, h_v: pinned host tensors or numpy arrays; dst_pages: device int32; staging: device uint8)
+    def kv_import_staging_bytes(self, count: int) -> int:
+        return int(self._lib.agx_kv_import_staging_bytes(self._h, int(count)))
+
+    def kv_import_pages(self, k_pool, v_pool, h_k, h_v, dst_pages, staging, stream=None):
+        st = self._lib.agx_kv_import_pages(self._h, _ptr(k_pool), _ptr(v_pool), int(k_pool.shape[0]), _ptr(h_k), _ptr(h_v),
+                                           _ptr(dst_pages), int(dst_pages.numel()), _ptr(staging),
+                                           staging.numel() * staging.element_size(), _stream_ptr(stream))
+        self._check(st, "agx_kv_import_pages")
 
     # -- agx_ngram_build / agx_ngram_draft (device int32 tensors; lut and workspace are uint8 tensors)
     def ngram_build(self, stream_tokens, n: int, lut, workspace, stream=None):

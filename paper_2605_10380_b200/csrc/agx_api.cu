@@ -611,4 +611,31 @@ agx_status agx_kv_copy_pages(agx_handle* h, void* k_pool, void* v_pool, int64_t 
     return AGX_OK;
 }
 
+int64_t agx_kv_import_staging_bytes(const agx_handle* h, int32_t count) {
+    if (!h || count < 0) return AGX_E_INVAL;
+    return 2ll * count * h->cfg.num_kv_heads * kPage * h->cfg.head_dim * elem_size(h->cfg.dtype);
+}
+
+agx_status agx_kv_import_pages(agx_handle* h, void* k_pool, void* v_pool, int64_t num_pages, const void* h_k, const void* h_v,
+                               const int32_t* dst_pages, int32_t count, void* staging, size_t staging_bytes, void* stream_v) {
+    if (!h) return AGX_E_INVAL;
+    h->last_launches = 0;
+    if (count < 0) return fail(h, AGX_E_INVAL, "negative count");
+    if (count == 0) return AGX_OK;
+    if (!k_pool || !v_pool || !h_k || !h_v || !dst_pages || !staging || num_pages < 1) return fail(h, AGX_E_INVAL, "null pointer or no pages");
+    if (!aligned(k_pool, 16) || !aligned(v_pool, 16) || !aligned(staging, 16)) return fail(h, AGX_E_INVAL, "pools and staging must be 16-byte aligned");
+    const size_t half = (size_t)agx_kv_import_staging_bytes(h, count) / 2;
+    if (staging_bytes < 2 * half) return fail(h, AGX_E_INVAL, "staging too small: %zu < %zu", staging_bytes, 2 * half);
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    char* st = (char*)staging;
+    cudaError_t e = cudaMemcpyAsync(st, h_k, half, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(st + half, h_v, half, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess)
+        e = launch_scatter_pages(h->cfg.dtype, k_pool, v_pool, num_pages, st, st + half, dst_pages, count, h->cfg.num_kv_heads,
+                                 h->cfg.head_dim, h->d_status, stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "page import");
+    h->last_launches = 1;
+    return AGX_OK;
+}
+
 }  // extern "C"

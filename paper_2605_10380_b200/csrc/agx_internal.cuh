@@ -97,6 +97,10 @@ cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_st
 cudaError_t launch_copy_pages(int dtype, void* k_pool, void* v_pool, long long num_pages, const int* src, const int* dst,
                               int count, int hkv, int head_dim, int* status, cudaStream_t stream);
 
+cudaError_t launch_scatter_pages(int dtype, void* k_pool, void* v_pool, long long num_pages, const void* k_stage,
+                                 const void* v_stage, const int* dst, int count, int hkv, int head_dim, int* status,
+                                 cudaStream_t stream);
+
 // n-gram draft table (Sec. 4.3): sizes, build (three memsets + three small kernels) and chained lookups.
 long long ngram_lut_bytes(int max_stream_tokens);
 long long ngram_workspace_bytes(int stream_tokens);

@@ -3,6 +3,8 @@
 //     short sequences, run once offline);
 //   * the online lookup - the stored combination that shares the longest run of leading clusters with a
 //     request, the mismatched tail of the stored one being cut off;
+//   * bringing stored KV pages from host memory into the pool (two large copies into a staging area, one
+//     scatter kernel), on whatever stream the caller chooses so that it overlaps attention elsewhere;
 //   * the page copy a cut needs: a reused prefix that ends inside a page shares the full pages before it
 //     and gets a private copy of that last page, so that the new sequence can append behind the cut.
 #include <algorithm>
@@ -29,6 +31,33 @@ copy_pages_kernel(uint4* __restrict__ k_pool, uint4* __restrict__ v_pool, long l
     }
     if (s == d) return;
     for (long long i = threadIdx.x; i < vec_per_page; i += blockDim.x) pool[d * vec_per_page + i] = pool[s * vec_per_page + i];
+}
+
+// Scatter pages from a packed staging area (page i of the import) to pool pages dst[i]: one CTA per (page, K or V).
+__global__ void __launch_bounds__(256)
+scatter_pages_kernel(uint4* __restrict__ k_pool, uint4* __restrict__ v_pool, long long num_pages, const uint4* __restrict__ k_stage,
+                     const uint4* __restrict__ v_stage, const int* __restrict__ dst, long long vec_per_page, int* status) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int i = blockIdx.x >> 1;
+    const bool is_v = blockIdx.x & 1;
+    const long long d = dst[i];
+    if (d < 0 || d >= num_pages) {
+        if (threadIdx.x == 0) atomicOr(status, AGX_DEV_BAD_PAGE);
+        return;
+    }
+    uint4* pool = is_v ? v_pool : k_pool;
+    const uint4* stage = is_v ? v_stage : k_stage;
+    for (long long j = threadIdx.x; j < vec_per_page; j += blockDim.x) pool[d * vec_per_page + j] = stage[(long long)i * vec_per_page + j];
+}
+
+cudaError_t launch_scatter_pages(int dtype, void* k_pool, void* v_pool, long long num_pages, const void* k_stage,
+                                 const void* v_stage, const int* dst, int count, int hkv, int head_dim, int* status,
+                                 cudaStream_t stream) {
+    if (count == 0) return cudaSuccess;
+    const long long vec_per_page = (long long)hkv * kPage * head_dim * (dtype == AGX_BF16 ? 2 : 4) / 16;
+    return launch_chained(scatter_pages_kernel, dim3(2 * count), dim3(256), 0, stream, (uint4*)k_pool, (uint4*)v_pool, num_pages,
+                          (const uint4*)k_stage, (const uint4*)v_stage, dst, vec_per_page, status);
 }
 
 cudaError_t launch_copy_pages(int dtype, void* k_pool, void* v_pool, long long num_pages, const int* src, const int* dst,

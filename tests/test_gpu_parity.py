@@ -327,6 +327,38 @@ def test_prefix_reuse_with_tail_cut_shares_full_pages_and_copies_the_cut_page():
     assert h.get_status() & agx.AGX_DEV_BAD_PAGE
 
 
+def test_import_of_stored_pages_from_host_memory_overlapping_attention_on_another_stream():
+    """Stored KV pages (Sec. 4.2) come from pinned host memory into scattered pool pages, bit for bit, on a stream
+    of their own while attention over resident pages runs on another; a sequence then attends over the imported
+    prefix."""
+    w = W.make_attn_workload("import", 91, "bf16", 32, 8, 128, [3072], [64], spare_pages=4)
+    h = agx.Handle(32, 8, 128, "bf16")
+    n_imp = 3072 // 16
+    rows = w.page_table[0, :n_imp].astype(np.int64)
+    h_k = torch.from_numpy(w.k_pool[rows].copy()).pin_memory(); h_v = torch.from_numpy(w.v_pool[rows].copy()).pin_memory()
+    kp, vp = w.k_pool.copy(), w.v_pool.copy()
+    kp[rows] = 0; vp[rows] = 0                                       # the pool does not hold the prefix yet
+    k_pool, v_pool = dev(kp, "bf16"), dev(vp, "bf16")
+    other = DeviceBatch(W.make_attn_workload("busy", 92, "bf16", 32, 8, 128, [20000], [8]))   # resident work for the other stream
+    staging = torch.empty(h.kv_import_staging_bytes(n_imp), dtype=torch.uint8, device="cuda")
+    dst = dev(w.page_table[0, :n_imp].copy())
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        h.kv_import_pages(k_pool, v_pool, h_k, h_v, dst, staging, stream=side)
+    other.append(); other.attend()                                   # enqueued on the current stream meanwhile
+    side.synchronize(); torch.cuda.synchronize()
+    assert h.get_status() == 0 and other.status() == 0
+    assert np.array_equal(host_storage(k_pool, "bf16"), w.k_pool) and np.array_equal(host_storage(v_pool, "bf16"), w.v_pool)
+    b = DeviceBatch(w); b.k_pool, b.v_pool = k_pool, v_pool
+    b.append(); out, _ = b.attend()
+    kref, vref = oracle_pools_after_append(w)
+    rng = np.random.default_rng(1)
+    si = rng.integers(0, 64, 30).astype(np.int32); sh = rng.integers(0, 32, 30).astype(np.int32)
+    ref, _, _ = oracle.attn_paged(w.q_block, kref, vref, w.page_table[0], "bf16", 3072, select=(si, sh))
+    check_attention(out[si, sh], ref, "imported prefix")
+
+
 # ------------------------------------------------------------------ whole step from host buffers
 @pytest.mark.parametrize("enqueue_only", [False, True])
 def test_verify_step_host_matches_oracle(enqueue_only):
