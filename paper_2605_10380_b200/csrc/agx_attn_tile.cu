@@ -301,21 +301,31 @@ __device__ __noinline__ void tile_epilogue(unsigned char* smem, uint32_t tO, flo
         }
     }
     __syncwarp();
-    // a warp writes one row per instruction: lane j moves 16-byte unit j (fp32) or converts it to 8 bytes of bf16
-#pragma unroll 8
-    for (int rl = 0; rl < 32; ++rl) {
-        const int ro = r_warp0 + rl;
-        if (ro >= it.rows) break;
-        const int io = (int)(((uint64_t)(uint32_t)ro * magic) >> 32), ho = it.g * it.G + (ro - io * it.G);
-        const uint4 v = *(const uint4*)(stage + rl * 512 + ((lane ^ rl) << 4));
-        if (single) {
-            uint2 pk;
-            pk.x = pack_bf16(__uint_as_float(v.x), __uint_as_float(v.y));
-            pk.y = pack_bf16(__uint_as_float(v.z), __uint_as_float(v.w));
-            *(uint2*)((unsigned char*)cx.out + (((long long)(it.q_row0 + io) * cx.hq + ho) * 256 + lane * 8)) = pk;
-        } else {
-            const long long e = (long long)cx.part_base + ((long long)io * cx.hq + ho) * it.nsplit + it.split;
-            *(uint4*)((unsigned char*)(cx.part_o + e * kD) + lane * 16) = v;
+    // a warp writes one row per instruction: lane j moves 16-byte unit j (fp32) or converts it to 8 bytes of bf16;
+    // eight rows' loads are in flight before the first store
+    const int n_valid = min(32, it.rows - r_warp0);
+    for (int rl0 = 0; rl0 < n_valid; rl0 += 8) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int rl = rl0 + u;
+            v[u] = *(const uint4*)(stage + (rl & 31) * 512 + ((lane ^ (rl & 31)) << 4));
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int rl = rl0 + u;
+            if (rl >= n_valid) break;
+            const int ro = r_warp0 + rl;
+            const int io = (int)(((uint64_t)(uint32_t)ro * magic) >> 32), ho = it.g * it.G + (ro - io * it.G);
+            if (single) {
+                uint2 pk;
+                pk.x = pack_bf16(__uint_as_float(v[u].x), __uint_as_float(v[u].y));
+                pk.y = pack_bf16(__uint_as_float(v[u].z), __uint_as_float(v[u].w));
+                *(uint2*)((unsigned char*)cx.out + (((long long)(it.q_row0 + io) * cx.hq + ho) * 256 + lane * 8)) = pk;
+            } else {
+                const long long e = (long long)cx.part_base + ((long long)io * cx.hq + ho) * it.nsplit + it.split;
+                *(uint4*)((unsigned char*)(cx.part_o + e * kD) + lane * 16) = v[u];
+            }
         }
     }
 }
