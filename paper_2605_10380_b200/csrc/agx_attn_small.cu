@@ -576,7 +576,11 @@ cudaError_t launch_small(const AttnParams& p, const CUtensorMap& map_k, const CU
     constexpr int kRing = NS * 2 * KW * kPage * kRowBytes;
     // [ring | merge region][Q tile][2 * NS barriers + abort flag] + slack for the 1024-byte alignment
     constexpr int kSmem = (kRing > kMergeBytes ? kRing : kMergeBytes) + MT * 16 * kRowBytes + 2 * NS * 8 + 16 + 1024;
-    static bool configured = false;
+    // the attribute is per device: remember which devices have it (a process normally drives one GPU)
+    static bool configured_on[64] = {false};
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    bool& configured = configured_on[device];
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
         if (e != cudaSuccess) return e;

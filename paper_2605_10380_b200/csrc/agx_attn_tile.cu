@@ -759,7 +759,11 @@ bool make_pool_map(CUtensorMap* map, const void* pool, long long num_pages, int 
 namespace {
 template <bool kStreams>
 cudaError_t launch_tile(const AttnParams& p, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
-    static bool configured = false;
+    // the attribute is per device: remember which devices have it (a process normally drives one GPU)
+    static bool configured_on[64] = {false};
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    bool& configured = configured_on[device];
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(attn_tile_bf16_kernel<kStreams>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
         if (e != cudaSuccess) return e;
