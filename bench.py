@@ -2,7 +2,7 @@
 """Benchmark of the prefix-cached block-attention / greedy-accept hot path on B200.
 
 One JSON line on stdout (rank 0).  A *step* is one pass of the whole hot path over one batch:
-for every layer ``agx_kv_append`` + ``agx_attn_prefixed``, then one ``agx_accept_greedy``.
+for every layer ``agx_attn_prefixed_append`` (KV append + attention), then one ``agx_accept_greedy``.
 
 Default workload = "decode verification": batch 1, cached context 4096, q = 8 (7 drafts + the last
 emitted token), GQA 32/8, head_dim 128, bf16, page size 16 with shuffled pages, 32 independent
@@ -176,11 +176,12 @@ class LayeredVerify:
     def step(self, attn_only=False):
         n = 0
         for l in range(self.layers):
-            if not attn_only:
-                self.h.kv_append(self.k_pools[l], self.v_pools[l], self.k_new[l], self.v_new[l], self.page_table,
-                                 self.prefix_dev, self.cu_dev)
+            if attn_only:
+                n += self.attn_layer(l)
+            else:   # the block's K/V rows are written by the attention kernel's CTAs before they read them
+                self.h.attn_prefixed_append(self.q_block[l], self.k_new[l], self.v_new[l], self.k_pools[l], self.v_pools[l],
+                                            self.page_table, self.P, self.Q, self.out[l], None, self.ws)
                 n += self.h.last_launch_count()
-            n += self.attn_layer(l)
         if not attn_only and self.vocab:
             self.seq_lens.copy_(self.prefix_dev)
             self.h.accept_greedy(self.logits, "bf16", self.vocab, self.drafts, self.cu_dev, self.acc, self.nxt, None,
@@ -464,7 +465,7 @@ def run_agx(args):
         "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": WORKLOAD,
-                   "step": "32 x (agx_kv_append + agx_attn_prefixed) + 1 x agx_accept_greedy, one CUDA graph",
+                   "step": "32 x agx_attn_prefixed_append (KV append + attention) + 1 x agx_accept_greedy, one CUDA graph",
                    "l2": "inputs larger than L2: 32 distinct layer pools = 553 MB, each read once per step",
                    "parallelism": f"{world} independent replica(s), no collective"},
         "gpu_launches": launches,

@@ -147,6 +147,26 @@ AGX_API agx_status agx_attn_prefixed(agx_handle* handle, const void* q_block, co
                              const int32_t* h_q_len, int32_t B, void* out, float* lse,
                              void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * agx_attn_prefixed_append - agx_kv_append and agx_attn_prefixed of the same block as one call.
+ * Sec. 2.3: the block's K/V rows join the cache (after the cached prefix) and the block then attends to
+ * prefix plus block.  Results, in the pools and in `out`, are those of the two calls made one after the
+ * other.  Where every sequence of a launch has at most 256 query rows per KV head (q_len * G; bf16 handles), the
+ * rows are written inside the attention kernel: each CTA stores the rows of its own KV head that fall into
+ * its own KV split before it reads them, which saves the append launch of a decode or verify step.
+ * Longer blocks and fp32 handles get an append launch in front of the attention launch.
+ *   k_new, v_new : device, [total_q][num_kv_heads][head_dim], 16-byte aligned (rows in the order of q_block)
+ *   k_pool, v_pool : device pools (written, then read); the other arguments as for agx_attn_prefixed
+ * Errors: those of agx_attn_prefixed; a page id outside [0, num_pages) sets AGX_DEV_BAD_PAGE, the row is
+ * not written and reads as zeros.
+ */
+AGX_API agx_status agx_attn_prefixed_append(agx_handle* handle, const void* q_block, const void* k_new,
+                                            const void* v_new, void* k_pool, void* v_pool, int64_t num_pages,
+                                            const int32_t* page_table, int32_t page_table_stride,
+                                            const int32_t* h_prefix_len, const int32_t* h_q_len, int32_t B,
+                                            void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                            void* stream);
+
 /* Scratch bytes agx_accept_greedy needs for total_q logits rows. */
 AGX_API int64_t agx_accept_workspace_bytes(agx_handle* handle, int32_t total_q, int32_t vocab);
 

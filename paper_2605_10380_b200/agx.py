@@ -23,7 +23,7 @@ _lib = None
 
 EXPORTS = (
     "agx_create", "agx_destroy", "agx_status_string", "agx_last_error", "agx_kv_append",
-    "agx_attn_workspace_bytes", "agx_attn_prefixed", "agx_accept_workspace_bytes",
+    "agx_attn_workspace_bytes", "agx_attn_prefixed", "agx_attn_prefixed_append", "agx_accept_workspace_bytes",
     "agx_accept_greedy", "agx_get_status", "agx_last_launch_count",
     "agx_verify_step_host_workspace_bytes", "agx_verify_step_host", "agx_verify_step_host_enqueue",
     "agx_accept_greedy_static", "agx_ngram_lut_bytes", "agx_ngram_workspace_bytes", "agx_ngram_build", "agx_ngram_draft",
@@ -114,6 +114,8 @@ def load() -> ctypes.CDLL:
     lib.agx_attn_workspace_bytes.restype = i64
     lib.agx_attn_prefixed.argtypes = [vp, vp, vp, vp, i64, vp, i32, vp, vp, i32, vp, vp, vp, ctypes.c_size_t, vp]
     lib.agx_attn_prefixed.restype = i32
+    lib.agx_attn_prefixed_append.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, i32, vp, vp, i32, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.agx_attn_prefixed_append.restype = i32
     lib.agx_accept_workspace_bytes.argtypes = [vp, i32, i32]
     lib.agx_accept_workspace_bytes.restype = i64
     lib.agx_accept_greedy.argtypes = [vp, vp, i32, i64, i32, vp, vp, i32, i32, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
@@ -247,6 +249,17 @@ class Handle:
                                          int(P.shape[0]), _ptr(out), _ptr(lse), _ptr(workspace), ws_bytes,
                                          _stream_ptr(stream))
         self._check(st, "agx_attn_prefixed")
+
+    # -- agx_attn_prefixed_append
+    def attn_prefixed_append(self, q_block, k_new, v_new, k_pool, v_pool, page_table, h_prefix_len, h_q_len, out, lse=None,
+                             workspace=None, stream=None):
+        P, Q = _h_i32(h_prefix_len), _h_i32(h_q_len)
+        ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        st = self._lib.agx_attn_prefixed_append(self._h, _ptr(q_block), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool),
+                                                int(k_pool.shape[0]), _ptr(page_table), int(page_table.shape[1]), _ptr(P),
+                                                _ptr(Q), int(P.shape[0]), _ptr(out), _ptr(lse), _ptr(workspace), ws_bytes,
+                                                _stream_ptr(stream))
+        self._check(st, "agx_attn_prefixed_append")
 
     # -- agx_accept_workspace_bytes
     def accept_workspace_bytes(self, total_q: int, vocab: int) -> int:

@@ -281,15 +281,20 @@ int64_t agx_attn_workspace_bytes(agx_handle* h, int32_t B, const int32_t* P, con
     return (int64_t)(part_ml_bytes(plan.part_entries) + (size_t)plan.part_entries * h->cfg.head_dim * sizeof(float));
 }
 
-agx_status agx_attn_prefixed(agx_handle* h, const void* q_block, const void* k_pool, const void* v_pool,
-                             int64_t num_pages, const int32_t* page_table, int32_t pt_stride, const int32_t* P,
-                             const int32_t* Q, int32_t B, void* out, float* lse, void* workspace,
-                             size_t workspace_bytes, void* stream_v) {
+// Attention, optionally preceded by the append of the block's own K/V rows (k_new != NULL).  Launches whose
+// sequences all fit one row chunk write those rows in the attention kernel's prologue (each CTA the rows of its own
+// KV split and head); the others (blocks of more than 256 rows, fp32 handles) get a separate append launch in front.
+static agx_status attn_impl(agx_handle* h, const void* q_block, const void* k_new, const void* v_new, const void* k_pool,
+                            const void* v_pool, int64_t num_pages, const int32_t* page_table, int32_t pt_stride,
+                            const int32_t* P, const int32_t* Q, int32_t B, void* out, float* lse, void* workspace,
+                            size_t workspace_bytes, void* stream_v) {
     if (!h) return AGX_E_INVAL;
     h->last_launches = 0;
     if (B < 0) return fail(h, AGX_E_INVAL, "negative B");
     if (B == 0) return AGX_OK;
     if (!q_block || !k_pool || !v_pool || !page_table || !P || !Q || !out) return fail(h, AGX_E_INVAL, "null pointer");
+    if (k_new && (!v_new || !aligned(k_new, 16) || !aligned(v_new, 16)))
+        return fail(h, AGX_E_INVAL, "k_new/v_new must both be given and 16-byte aligned");
     if (!aligned(q_block, 16) || !aligned(out, 16) || !aligned(k_pool, 256) || !aligned(v_pool, 256))
         return fail(h, AGX_E_INVAL, "q_block/out must be 16-byte and pools 256-byte aligned");
     if (num_pages < 1 || pt_stride < 1) return fail(h, AGX_E_INVAL, "num_pages and page_table_stride must be >= 1");
@@ -318,8 +323,23 @@ agx_status agx_attn_prefixed(agx_handle* h, const void* q_block, const void* k_p
         p.num_seqs = (int)ln.seqs.size();
         p.num_items = ln.num_items;
         bool split = false;
-        for (int i = 0; i < p.num_seqs; ++i) { p.seq[i] = ln.seqs[i]; split |= ln.seqs[i].nsplit > 1; }
+        bool one_chunk = true;
+        for (int i = 0; i < p.num_seqs; ++i) {
+            p.seq[i] = ln.seqs[i];
+            split |= ln.seqs[i].nsplit > 1;
+            one_chunk &= ln.seqs[i].row_chunks == 1;
+        }
         cudaError_t e;
+        p.k_new = p.v_new = nullptr;
+        if (k_new) {
+            p.k_new = k_new; p.v_new = v_new;
+            if (ln.kind == KIND_SIMT || !one_chunk) {
+                e = launch_kv_append_plan(p, h->cfg.dtype, ln.total_rows, stream);
+                if (e != cudaSuccess) return cuda_fail(h, e, "append launch");
+                h->last_launches++;
+                p.k_new = p.v_new = nullptr;
+            }
+        }
         switch (ln.kind) {
             case KIND_SMALL1: e = launch_attn_small_bf16(p, 1, h->small_kw, stream); break;
             case KIND_SMALL2: e = launch_attn_small_bf16(p, 2, h->small_kw, stream); break;
@@ -338,6 +358,23 @@ agx_status agx_attn_prefixed(agx_handle* h, const void* q_block, const void* k_p
         }
     }
     return AGX_OK;
+}
+
+agx_status agx_attn_prefixed(agx_handle* h, const void* q_block, const void* k_pool, const void* v_pool,
+                             int64_t num_pages, const int32_t* page_table, int32_t pt_stride, const int32_t* P,
+                             const int32_t* Q, int32_t B, void* out, float* lse, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    return attn_impl(h, q_block, nullptr, nullptr, k_pool, v_pool, num_pages, page_table, pt_stride, P, Q, B, out, lse,
+                     workspace, workspace_bytes, stream);
+}
+
+agx_status agx_attn_prefixed_append(agx_handle* h, const void* q_block, const void* k_new, const void* v_new, void* k_pool,
+                                    void* v_pool, int64_t num_pages, const int32_t* page_table, int32_t pt_stride,
+                                    const int32_t* P, const int32_t* Q, int32_t B, void* out, float* lse,
+                                    void* workspace, size_t workspace_bytes, void* stream) {
+    if (h && B > 0 && (!k_new || !v_new)) return fail(h, AGX_E_INVAL, "null pointer");
+    return attn_impl(h, q_block, k_new, v_new, k_pool, v_pool, num_pages, page_table, pt_stride, P, Q, B, out, lse,
+                     workspace, workspace_bytes, stream);
 }
 
 static int accept_chunks(const agx_handle* h, int total_q, int vocab, int dtype) {
@@ -504,12 +541,9 @@ static agx_status verify_step_host_impl(agx_handle* h, void* k_pool, void* v_poo
     }
     if (e != cudaSuccess) return cuda_fail(h, e, "host step: upload");
     int launches = 0;
-    st = agx_kv_append(h, k_pool, v_pool, num_pages, ws + L.k, ws + L.v, page_table, pt_stride,
-                       (const int32_t*)(ws + L.prefix), (const int32_t*)(ws + L.cu), B, L.total_q, stream);
-    if (st != AGX_OK) return st;
-    launches += h->last_launches;
-    st = agx_attn_prefixed(h, ws + L.q, k_pool, v_pool, num_pages, page_table, pt_stride, P, Q, B, ws + L.out, nullptr,
-                           L.attn_ws_bytes ? ws + L.attn_ws : nullptr, L.attn_ws_bytes, stream);
+    st = agx_attn_prefixed_append(h, ws + L.q, ws + L.k, ws + L.v, k_pool, v_pool, num_pages, page_table, pt_stride, P, Q,
+                                  B, ws + L.out, nullptr, L.attn_ws_bytes ? ws + L.attn_ws : nullptr, L.attn_ws_bytes,
+                                  stream);
     if (st != AGX_OK) return st;
     launches += h->last_launches;
     if (with_accept) {

@@ -117,6 +117,7 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     }
     pdl_launch_dependents();
     pdl_wait();   // from here on global memory written by the launch before this one is read
+    if (p.k_new) append_rows_bf16(p, sp, g, tok_begin, tok_begin + sp.split_tokens, tid, kThreads);   // fused append (row_chunks == 1)
     // ---- Q tile -> shared (rows beyond q*G are zero)
     for (int c = tid; c < MT * 16 * 16; c += kThreads) {
         const int r = c >> 4, ch = c & 15;

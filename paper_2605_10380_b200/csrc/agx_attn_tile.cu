@@ -380,6 +380,8 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
     pdl_wait();   // from here on global memory written by the launch before this one is read (Q, page table, K/V)
+    // fused append (one row chunk per sequence): the block's own K/V rows of this split go into the pages first
+    if (p.k_new && warp >= 2) append_rows_bf16(p, sp, g, kv_begin, kv_begin + sp.split_tokens, tid - 64, kQLoadThreads);
     // Q: 256 rows x 256 B by 16-byte cp.async (all of a thread's copies in flight at once), written in
     // the 128-byte-swizzled K-major operand layout; rows past q * G are zero-filled.
     if (warp >= 2) {
@@ -397,7 +399,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
     // Barriers initialised, TMEM address published.  Warp 0 (which set the barriers up and needs nothing
     // from the others) only signals and goes straight to the page table and its first K/V copies.
     tc_fence_before();
-    if (warp == 0) { __syncwarp(); asm volatile("bar.arrive 2, %0;\n" ::"n"(kThreads) : "memory"); }
+    if (warp == 0 && !p.k_new) { __syncwarp(); asm volatile("bar.arrive 2, %0;\n" ::"n"(kThreads) : "memory"); }   // (a fused append must land first)
     else asm volatile("bar.sync 2, %0;\n" ::"n"(kThreads) : "memory");
     tc_fence_after();
     const uint32_t tmem_base = (warp == 0) ? 0u : *tmem_slot;

@@ -35,6 +35,8 @@ struct AttnParams {
     float* part_o;   // [entries][head_dim] fp32, un-normalised, relative to part_ml.x
     float2* part_ml; // [entries] (running max in log2 units, sum)
     int* status;
+    const void* k_new;   // fused append (agx_attn_prefixed_append): the block's K/V rows [total_q][hkv][d], or NULL
+    const void* v_new;
     long long num_pages;
     int pt_stride;
     int hq, hkv, head_dim;
@@ -67,6 +69,9 @@ struct StepMeta {
     int cu[kMaxSeqs + 1];
 };
 cudaError_t launch_write_meta(const StepMeta& m, int* prefix, int* seq_lens, int* cu_q, cudaStream_t stream);
+
+// Append of the launch's sequences with the plans taken from the kernel arguments (no device-side lengths needed).
+cudaError_t launch_kv_append_plan(const AttnParams& p, int dtype, int total_rows, cudaStream_t stream);
 
 // Launchers (each returns the cudaError_t of its launch).
 cudaError_t launch_kv_append(int dtype, void* k_pool, void* v_pool, long long num_pages, const void* k_new,

@@ -61,6 +61,39 @@ cudaError_t launch_kv_append(int dtype, void* k_pool, void* v_pool, long long nu
                           vec_per_row, status);
 }
 
+// The same scatter for the sequences of one attention launch, lengths and row offsets taken from the launch's plans.
+__global__ void __launch_bounds__(256)
+kv_append_plan_kernel(const __grid_constant__ AttnParams p, int vec_per_row, int total_rows) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const long long n_vec = (long long)total_rows * p.hkv * vec_per_row;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < n_vec; idx += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(idx % vec_per_row);
+        const long long row = idx / vec_per_row;
+        const int g = (int)(row % p.hkv);
+        int lr = (int)(row / p.hkv);   // row within the launch: sequences back to back
+        int si = 0;
+        while (si + 1 < p.num_seqs && lr >= p.seq[si].q_len) { lr -= p.seq[si].q_len; ++si; }
+        const SeqPlan& sp = p.seq[si];
+        const int tok = sp.prefix_len + lr;
+        const long long page = (tok >> 4) < p.pt_stride ? __ldg(p.page_table + (long long)sp.seq_index * p.pt_stride + (tok >> 4)) : -1;
+        if (page < 0 || page >= p.num_pages) { if (c == 0 && g == 0) atomicOr(p.status, AGX_DEV_BAD_PAGE); continue; }
+        const long long src = ((long long)(sp.q_row0 + lr) * p.hkv + g) * vec_per_row + c;
+        const long long dst = ((page * p.hkv + g) * kPage + (tok & 15)) * vec_per_row + c;
+        ((uint4*)p.k_pool)[dst] = ((const uint4*)p.k_new)[src];
+        ((uint4*)p.v_pool)[dst] = ((const uint4*)p.v_new)[src];
+    }
+}
+
+cudaError_t launch_kv_append_plan(const AttnParams& p, int dtype, int total_rows, cudaStream_t stream) {
+    const int vec_per_row = p.head_dim * (dtype == AGX_BF16 ? 2 : 4) / 16;
+    const long long n_vec = (long long)total_rows * p.hkv * vec_per_row;
+    if (n_vec == 0) return cudaSuccess;
+    long long blocks = (n_vec + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    return launch_chained(kv_append_plan_kernel, dim3((unsigned)blocks), dim3(256), 0, stream, p, vec_per_row, total_rows);
+}
+
 // Lengths of a small batch travel as kernel arguments instead of three pageable host-to-device copies (each
 // of which would first synchronise the stream): prefix_len, the committed lengths and the row offsets.
 __global__ void write_meta_kernel(const __grid_constant__ StepMeta m, int* prefix, int* seq_lens, int* cu_q) {

@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include "agx.h"
+#include "agx_internal.cuh"
 
 namespace agx {
 
@@ -61,6 +62,28 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 // before it has completed and its writes are visible.  Both are no-ops for launches without the attribute.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+
+// Fused KV append (bf16, d = 128): the CTA that will read tokens [t_lo, t_hi) of KV head g writes the block's own
+// rows in that range into the sequence's pages first (Sec. 2.3: the block's KV joins the cache before it is attended
+// to), then makes them visible to the TMA copies that follow: a generic-proxy fence here, a CTA barrier at the caller.
+__device__ __forceinline__ void append_rows_bf16(const AttnParams& p, const SeqPlan& sp, int g, int t_lo, int t_hi, int tid,
+                                                 int nthreads) {
+    const int lo = max(t_lo, sp.prefix_len), hi = min(t_hi, sp.prefix_len + sp.q_len);
+    if (hi > lo) {
+        const int* pt_row = p.page_table + (long long)sp.seq_index * p.pt_stride;
+        for (int idx = tid; idx < (hi - lo) * 32; idx += nthreads) {
+            const int tok = lo + (idx >> 5), is_v = (idx >> 4) & 1, c = idx & 15;
+            const long long page = (tok >> 4) < p.pt_stride ? __ldg(pt_row + (tok >> 4)) : -1;
+            if (page < 0 || page >= p.num_pages) { if (c == 0) atomicOr(p.status, AGX_DEV_BAD_PAGE); continue; }
+            const unsigned char* src = (const unsigned char*)(is_v ? p.v_new : p.k_new) +
+                                       (((long long)(sp.q_row0 + tok - sp.prefix_len) * p.hkv + g) * 256 + c * 16);
+            unsigned char* dst = (unsigned char*)(is_v ? p.v_pool : p.k_pool) + (((page * p.hkv + g) * kPage + (tok & 15)) * 256 + c * 16);
+            *(uint4*)dst = __ldg((const uint4*)src);
+        }
+        __threadfence();
+        asm volatile("fence.proxy.async;\n" ::: "memory");
+    }
+}
 
 __device__ __forceinline__ float ex2(float x) {
     float y;

@@ -60,6 +60,15 @@ class DeviceBatch:
         torch.cuda.synchronize()
         return host_f64(self.out), host_f64(self.lse)
 
+    def attend_append(self):
+        """Append and attention of the block as the one fused call."""
+        w = self.w
+        self.h.attn_prefixed_append(self.q_block, self.k_new, self.v_new, self.k_pool, self.v_pool, self.page_table,
+                                    w.prefix_len, w.q_len, self.out, self.lse, self.ws)
+        self.launches = self.h.last_launch_count()
+        torch.cuda.synchronize()
+        return host_f64(self.out), host_f64(self.lse)
+
     def status(self):
         return self.h.get_status()
 

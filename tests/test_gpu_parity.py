@@ -16,7 +16,7 @@ from tests.gpu_util import (DeviceBatch, check_attention, dev, host_storage, ora
 pytestmark = pytest.mark.gpu
 
 
-def run_and_check(w, sample=None, poison=False, strict=False):
+def run_and_check(w, sample=None, poison=False, strict=False, fused=False):
     b = DeviceBatch(w)
     if poison:  # slots past P + q in every sequence's last page hold NaN: they must never be read
         nanbits = 0x7FC0 if w.dtype == "bf16" else np.float32(np.nan)
@@ -27,8 +27,11 @@ def run_and_check(w, sample=None, poison=False, strict=False):
                 kp = host_storage(b.k_pool, w.dtype); vp = host_storage(b.v_pool, w.dtype)
                 kp[pg, :, L % 16:, :] = nanbits; vp[pg, :, L % 16:, :] = nanbits
                 b.k_pool.copy_(dev(kp, w.dtype)); b.v_pool.copy_(dev(vp, w.dtype))
-    b.append()
-    out, lse = b.attend()
+    if fused:
+        out, lse = b.attend_append()
+    else:
+        b.append()
+        out, lse = b.attend()
     assert b.status() == 0
     kp, vp = oracle_pools_after_append(w)
     # append parity, bit-exact on the touched pages
@@ -516,6 +519,59 @@ def test_stream_schedule_ragged_batch_matches_warp_mma_kernel(monkeypatch):
     assert b.status() == 0 and b2.status() == 0
     assert np.max(np.abs(a - c)) < 2e-2
     run_and_check(w, sample=(7, 12))
+
+
+# ------------------------------------------------------------------ append fused into the attention launch
+FUSED_CASES = [
+    # name, dtype, hq, hkv, d, P, q, stream schedule forced
+    ("decode", "bf16", 32, 8, 128, [0, 1, 15, 16, 4095], [1, 1, 1, 1, 1], False),
+    ("verify_ragged", "bf16", 32, 8, 128, [2048, 2100, 4000, 2063, 9000, 2500, 3001, 250], [1, 2, 4, 8, 16, 3, 5, 30], False),
+    ("verify_split_boundaries", "bf16", 32, 8, 128, [249, 255, 256, 511, 1020], [8, 8, 8, 8, 8], False),
+    ("stream_forced", "bf16", 32, 8, 128, [17, 127, 2049, 5000, 777], [4, 8, 5, 8, 32], True),
+    ("stream_long", "bf16", 32, 8, 128, [20000, 14000], [8, 3], False),
+    ("mid_q", "bf16", 32, 8, 128, [3000, 130], [20, 9], False),
+    ("tile_one_chunk", "bf16", 8, 2, 128, [256, 100, 1000], [64, 50, 33], False),
+    ("tile_many_chunks", "bf16", 24, 8, 128, [1030, 5], [300, 200], False),
+    ("mixed_kinds", "bf16", 32, 8, 128, [2048, 2300, 2055, 4000, 2600, 3000], [8, 200, 1, 130, 16, 513], False),
+    ("fp32", "f32", 8, 2, 64, [256, 30, 0], [4, 1, 7], False),
+]
+
+
+@pytest.mark.parametrize("name,dtype,hq,hkv,d,P,q,stream", FUSED_CASES, ids=[c[0] for c in FUSED_CASES])
+def test_fused_append_attention_equals_the_two_calls_and_the_oracle(name, dtype, hq, hkv, d, P, q, stream, monkeypatch):
+    """agx_attn_prefixed_append: pools and outputs bit-identical to agx_kv_append followed by agx_attn_prefixed
+    (the same kernels do the arithmetic), slots it must not touch unchanged, and parity with the oracle."""
+    if stream:
+        monkeypatch.setenv("AGX_STREAM_MIN_TOKENS", "0")
+    w = W.make_attn_workload("fused_" + name, 7000 + sum(P) + sum(q), dtype, hq, hkv, d, P, q, spare_pages=3)
+    two = DeviceBatch(w); two.append(); out2, lse2 = two.attend()
+    one = DeviceBatch(w); out1, lse1 = one.attend_append()
+    assert one.status() == 0 and two.status() == 0
+    assert torch.equal(one.k_pool, two.k_pool) and torch.equal(one.v_pool, two.v_pool)
+    assert np.array_equal(out1, out2) and np.array_equal(lse1, lse2)
+    run_and_check(w, sample=(3, 40) if max(P) + max(q) > 3000 else None, fused=True)
+
+
+def test_fused_append_saves_the_append_launch_on_a_verify_batch():
+    w = W.c2_decode_verify()
+    b = DeviceBatch(w); b.attend_append()
+    fused = b.launches
+    b2 = DeviceBatch(w); b2.append(); b2.attend()
+    assert fused == b2.launches and b.status() == 0      # attention + combine; the append took a launch of its own before
+    assert torch.equal(b.k_pool, b2.k_pool) and torch.equal(b.out, b2.out)
+
+
+def test_fused_append_reports_a_bad_page_and_skips_the_row():
+    w = W.make_attn_workload("fused_bad_page", 77, "bf16", 32, 8, 128, [40, 300], [8, 8], spare_pages=2)
+    b = DeviceBatch(w)
+    pt = w.page_table.copy(); pt[1, 300 // 16] = w.k_pool.shape[0] + 5
+    b.page_table = dev(pt)
+    before = b.k_pool.clone()
+    b.attend_append()
+    assert b.status() & agx.AGX_DEV_BAD_PAGE
+    touched = (b.k_pool != before).flatten(1).any(1).nonzero().flatten().cpu().numpy()
+    assert int(w.page_table[1, 300 // 16]) not in touched.tolist()      # the row behind the bad id was not written anywhere
+    assert set(touched.tolist()) == {int(w.page_table[0, 2]), int(w.page_table[1, 19])}
 
 
 # ------------------------------------------------------------------ tensor-core tile kernel (large q)
