@@ -471,7 +471,7 @@ def run_agx(args):
         "gpu_launches": launches,
         "e2e": {"value": units_all / (e2e_ms_max * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_max,
-                "path": "agx_verify_step_host_enqueue per layer (pinned host q/k_new/v_new/logits in, out/accept results back), one stream synchronisation per step"},
+                "path": "agx_verify_step_host_enqueue per layer (pinned host q/k_new/v_new/logits in, out/accept results back; the small per-layer buffers are read and written by kernels over the bus, logits and accept results by copy-engine transfers), one stream synchronisation per step"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES, "peak_source": peaks["source"],
                      "frac_of_nominal_8000": achieved / 8000.0,

@@ -248,7 +248,12 @@ AGX_API agx_status agx_get_status(agx_handle* handle, void* stream, int32_t* dev
  *   k_pool, v_pool, page_table : device (as in agx_kv_append)
  *   h_prefix_len, h_q_len      : host int32 [B]
  *   h_q_block, h_k_new, h_v_new: host, element type of the handle (pinned memory makes the
- *                                copies asynchronous; pageable memory works but serialises)
+ *                                copies asynchronous; pageable memory works but serialises).
+ *                                When the three are pinned, mapped into the device's address space
+ *                                (cudaHostAlloc / cudaHostRegister) and together at most 1 MiB, one
+ *                                kernel reads them across the bus instead of three transfers; a
+ *                                pinned, mapped h_out of at most 1 MiB is written by the attention
+ *                                kernels directly.  Results are the same either way.
  *   h_logits                   : host, [total_q][row_stride] of logits_dtype
  *   h_drafts                   : host int32 [total_q - B] (may be NULL when total_q == B)
  *   h_out                      : host, [total_q][num_q_heads][head_dim]

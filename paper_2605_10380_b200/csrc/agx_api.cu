@@ -22,6 +22,7 @@ struct agx_handle {
     int force_mma_sync;     // route large q through the mma.sync kernel (env AGX_FORCE_MMA_SYNC)
     int debug_plan;         // print launch plans to stderr (env AGX_DEBUG_PLAN)
     int small_kw;           // pages per pipeline stage of the warp-MMA kernel, 4 or 8 (env AGX_SMALL_KW)
+    int zero_copy;          // host steps: bit 0 = kernels read small pinned inputs, bit 1 = kernels write `out` into a pinned buffer (env AGX_ZERO_COPY, default 3)
     int stream_min_tokens;  // context length from which blocks of <= 32 rows take the tensor-core stream schedule (env AGX_STREAM_MIN_TOKENS)
     std::vector<int32_t> cu_host;  // staging for agx_verify_step_host (lives until its final sync)
     char err[512];
@@ -224,6 +225,8 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     h->force_mma_sync = env ? atoi(env) : 0;
     env = getenv("AGX_STREAM_MIN_TOKENS");
     h->stream_min_tokens = env ? atoi(env) : 12288;
+    env = getenv("AGX_ZERO_COPY");
+    h->zero_copy = env ? atoi(env) : 3;
     env = getenv("AGX_SMALL_KW");
     h->small_kw = (env && atoi(env) == 4) ? 4 : 8;
     env = getenv("AGX_DEBUG_PLAN");
@@ -443,6 +446,17 @@ int32_t agx_last_launch_count(const agx_handle* h) { return h ? h->last_launches
 }  // extern "C"
 
 namespace {
+constexpr size_t kZeroCopyMaxBytes = 1u << 20;
+
+// Device-side address of a 16-byte-aligned host buffer that is pinned and mapped (cudaHostAlloc / cudaHostRegister
+// under unified addressing), else NULL.
+void* mapped_alias(const void* host) {
+    if (!host || ((uintptr_t)host & 15)) return nullptr;
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
 struct HostStepLayout {
     size_t q, k, v, out, logits, drafts, prefix, cu, acc, next, seqlen, attn_ws, accept_ws, total;
     size_t q_bytes, kv_bytes, logits_bytes, attn_ws_bytes, accept_ws_bytes;
@@ -519,30 +533,52 @@ static agx_status verify_step_host_impl(agx_handle* h, void* k_pool, void* v_poo
     cu.assign(B + 1, 0);
     for (int s = 0; s < B; ++s) cu[s + 1] = cu[s] + Q[s];
     cudaError_t e = cudaSuccess;
+    int launches = 0;
     auto h2d = [&](size_t off, const void* src, size_t bytes) {
         if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(ws + off, src, bytes, cudaMemcpyHostToDevice, stream);
     };
-    h2d(L.q, h_q, L.q_bytes); h2d(L.k, h_k, L.kv_bytes); h2d(L.v, h_v, L.kv_bytes);
+    // Small blocks in pinned, device-mapped host memory cross by one kernel that reads the host buffers and, on the
+    // way back, by the attention kernels writing `out` straight into the host buffer: each copy-engine transfer on
+    // the stream costs several microseconds whatever its size.  Anything else goes through cudaMemcpyAsync.
+    const size_t in_bytes = L.q_bytes + 2 * L.kv_bytes;
+    const void* mq = (h->zero_copy & 1) && in_bytes <= kZeroCopyMaxBytes ? mapped_alias(h_q) : nullptr;
+    const void* mk = mq ? mapped_alias(h_k) : nullptr;
+    const void* mv = mk ? mapped_alias(h_v) : nullptr;
+    void* out_dev = ws + L.out;
+    if ((h->zero_copy & 2) && L.q_bytes <= kZeroCopyMaxBytes)
+        if (void* mo = mapped_alias(h_out)) out_dev = mo;
+    if (mv) {
+        StageCopies sc;
+        sc.src[0] = (const uint4*)mq; sc.src[1] = (const uint4*)mk; sc.src[2] = (const uint4*)mv;
+        sc.dst[0] = (uint4*)(ws + L.q); sc.dst[1] = (uint4*)(ws + L.k); sc.dst[2] = (uint4*)(ws + L.v);
+        sc.units[0] = (unsigned)(L.q_bytes / 16); sc.units[1] = sc.units[2] = (unsigned)(L.kv_bytes / 16);
+        e = launch_stage_in(sc, stream);
+        if (e == cudaSuccess) ++launches;
+    } else {
+        h2d(L.q, h_q, L.q_bytes); h2d(L.k, h_k, L.kv_bytes); h2d(L.v, h_v, L.kv_bytes);
+    }
     if (with_accept) {
         h2d(L.logits, h_logits, L.logits_bytes);
         h2d(L.drafts, h_drafts, (size_t)(L.total_q - B) * 4);
     }
-    if (B <= kMaxSeqs) {   // as kernel arguments: no pageable copies, which would each synchronise the stream first
+    if (!with_accept) {
+        // lengths are needed on the device by the accept step only
+    } else if (B <= kMaxSeqs) {   // as kernel arguments: no pageable copies, which would each synchronise the stream first
         StepMeta meta;
         meta.B = B;
         for (int s = 0; s < B; ++s) { meta.prefix[s] = P[s]; meta.cu[s] = cu[s]; }
         meta.cu[B] = cu[B];
         if (e == cudaSuccess)
             e = launch_write_meta(meta, (int*)(ws + L.prefix), (int*)(ws + L.seqlen), (int*)(ws + L.cu), stream);
+        if (e == cudaSuccess) ++launches;
     } else {
         h2d(L.prefix, P, (size_t)B * 4);
         h2d(L.seqlen, P, (size_t)B * 4);
         h2d(L.cu, cu.data(), (size_t)(B + 1) * 4);
     }
     if (e != cudaSuccess) return cuda_fail(h, e, "host step: upload");
-    int launches = 0;
     st = agx_attn_prefixed_append(h, ws + L.q, ws + L.k, ws + L.v, k_pool, v_pool, num_pages, page_table, pt_stride, P, Q,
-                                  B, ws + L.out, nullptr, L.attn_ws_bytes ? ws + L.attn_ws : nullptr, L.attn_ws_bytes,
+                                  B, out_dev, nullptr, L.attn_ws_bytes ? ws + L.attn_ws : nullptr, L.attn_ws_bytes,
                                   stream);
     if (st != AGX_OK) return st;
     launches += h->last_launches;
@@ -557,7 +593,7 @@ static agx_status verify_step_host_impl(agx_handle* h, void* k_pool, void* v_poo
     auto d2h = [&](void* dst, size_t off, size_t bytes) {
         if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, ws + off, bytes, cudaMemcpyDeviceToHost, stream);
     };
-    d2h(h_out, L.out, L.q_bytes);
+    if (out_dev == ws + L.out) d2h(h_out, L.out, L.q_bytes);
     if (with_accept) {
         d2h(h_accept, L.acc, (size_t)B * 4); d2h(h_next, L.next, (size_t)B * 4); d2h(h_seq_lens, L.seqlen, (size_t)B * 4);
     }

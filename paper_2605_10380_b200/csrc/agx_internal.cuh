@@ -70,6 +70,15 @@ struct StepMeta {
 };
 cudaError_t launch_write_meta(const StepMeta& m, int* prefix, int* seq_lens, int* cu_q, cudaStream_t stream);
 
+// Up to three copies of 16-byte units by one kernel (sources may be pinned host memory mapped into the device's
+// address space: a few hundred KB cross faster this way than as separate copy-engine transfers).
+struct StageCopies {
+    const uint4* src[3];
+    uint4* dst[3];
+    unsigned units[3];
+};
+cudaError_t launch_stage_in(const StageCopies& c, cudaStream_t stream);
+
 // Append of the launch's sequences with the plans taken from the kernel arguments (no device-side lengths needed).
 cudaError_t launch_kv_append_plan(const AttnParams& p, int dtype, int total_rows, cudaStream_t stream);
 

@@ -6,6 +6,8 @@
 // loads and stores are fully coalesced 128-bit accesses.
 #include <stdlib.h>
 
+#include <algorithm>
+
 #include "agx_internal.cuh"
 #include "agx_sm100.cuh"
 
@@ -106,6 +108,24 @@ __global__ void write_meta_kernel(const __grid_constant__ StepMeta m, int* prefi
 
 cudaError_t launch_write_meta(const StepMeta& m, int* prefix, int* seq_lens, int* cu_q, cudaStream_t stream) {
     return launch_chained(write_meta_kernel, dim3(1), dim3(64), 0, stream, m, prefix, seq_lens, cu_q);
+}
+
+__global__ void __launch_bounds__(256) stage_in_kernel(const StageCopies c) {
+    pdl_launch_dependents();
+    pdl_wait();   // the launch before this one may still read the destination
+    const unsigned n0 = c.units[0], n1 = n0 + c.units[1], n2 = n1 + c.units[2];
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n2; i += gridDim.x * blockDim.x) {
+        const int k = i < n0 ? 0 : i < n1 ? 1 : 2;
+        const unsigned j = i - (k == 0 ? 0u : k == 1 ? n0 : n1);
+        c.dst[k][j] = c.src[k][j];
+    }
+}
+
+cudaError_t launch_stage_in(const StageCopies& c, cudaStream_t stream) {
+    const unsigned n = c.units[0] + c.units[1] + c.units[2];
+    if (n == 0) return cudaSuccess;
+    const unsigned blocks = std::min(1024u, (n + 255u) / 256u);
+    return launch_chained(stage_in_kernel, dim3(blocks), dim3(256), 0, stream, c);
 }
 
 bool pdl_enabled() {

@@ -363,17 +363,25 @@ def test_import_of_stored_pages_from_host_memory_overlapping_attention_on_anothe
 
 
 # ------------------------------------------------------------------ whole step from host buffers
-@pytest.mark.parametrize("enqueue_only", [False, True])
-def test_verify_step_host_matches_oracle(enqueue_only):
-    """Append + attention + accept through the host-buffer entry points (pinned inputs, results back in
-    host memory); the enqueue variant returns before the work is done and is synchronised by the caller."""
+n_launch = {}
+
+
+@pytest.mark.parametrize("enqueue_only,memory", [(False, "pinned"), (True, "pinned"), (True, "pageable"), (True, "pinned_copies")])
+def test_verify_step_host_matches_oracle(enqueue_only, memory, monkeypatch):
+    """Append + attention + accept through the host-buffer entry points (results back in host memory); the enqueue
+    variant returns before the work is done and is synchronised by the caller.  Small pinned buffers are read and
+    written by the kernels themselves, pageable ones (and pinned ones with AGX_ZERO_COPY=0) go through copies."""
+    if memory == "pinned_copies":
+        monkeypatch.setenv("AGX_ZERO_COPY", "0")
     w = W.make_attn_workload("host_step", 77, "bf16", 32, 8, 128, [1000, 517, 40], [8, 4, 1], spare_pages=2)
     aw = W.make_planted_accept("host_step_accept", 78, "bf16", 128256, w.q_len, w.prefix_len)
     b = DeviceBatch(w)
-    pin = lambda a, bf=False: (torch.from_numpy(np.ascontiguousarray(a)).view(torch.bfloat16) if bf else torch.from_numpy(np.ascontiguousarray(a))).pin_memory()
+    to_t = lambda a, bf: torch.from_numpy(np.ascontiguousarray(a)).view(torch.bfloat16) if bf else torch.from_numpy(np.ascontiguousarray(a))
+    pin = lambda a, bf=False: to_t(a, bf).pin_memory() if memory != "pageable" else to_t(a, bf).clone()
     hq, hk, hv = pin(w.q_block, True), pin(w.k_new, True), pin(w.v_new, True)
     hl, hd = pin(aw.logits, True), pin(aw.drafts)
-    h_out = torch.zeros((w.total_q, 32, 128), dtype=torch.bfloat16).pin_memory()
+    h_out = torch.zeros((w.total_q, 32, 128), dtype=torch.bfloat16)
+    h_out = h_out.pin_memory() if memory != "pageable" else h_out
     h_acc = torch.full((3,), -7, dtype=torch.int32).pin_memory()
     h_nxt = torch.full((3,), -7, dtype=torch.int32).pin_memory()
     h_sl = torch.full((3,), -7, dtype=torch.int32).pin_memory()
@@ -387,6 +395,9 @@ def test_verify_step_host_matches_oracle(enqueue_only):
     assert np.array_equal(host_storage(b.k_pool, "bf16"), kp) and np.array_equal(host_storage(b.v_pool, "bf16"), vp)
     ref, _ = oracle.attn_paged_batch(w.q_block, kp, vp, w.page_table, "bf16", w.prefix_len, w.q_len, w.cu_q)
     check_attention(h_out.to(torch.float64).numpy(), ref, "host step")
+    n_launch[memory] = b.h.last_launch_count()
+    if "pinned" in n_launch and "pinned_copies" in n_launch:      # the kernel that reads the pinned inputs is the one extra launch
+        assert n_launch["pinned"] == n_launch["pinned_copies"] + 1
     am, al, nt, sl = oracle.accept_greedy(aw.logits, "bf16", aw.vocab, aw.drafts, aw.cu_q, aw.prefix_len)
     assert np.array_equal(h_acc.numpy(), al) and np.array_equal(h_nxt.numpy(), nt) and np.array_equal(h_sl.numpy(), sl)
 
