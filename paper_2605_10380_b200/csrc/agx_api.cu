@@ -22,6 +22,7 @@ struct agx_handle {
     int force_mma_sync;     // route large q through the mma.sync kernel (env AGX_FORCE_MMA_SYNC)
     int debug_plan;         // print launch plans to stderr (env AGX_DEBUG_PLAN)
     int small_kw;           // pages per pipeline stage of the warp-MMA kernel, 4 or 8 (env AGX_SMALL_KW)
+    bool cluster_merge;     // KV splits of the small-q kernel merged inside thread-block clusters where the batch allows (env AGX_CLUSTER_MERGE=0 turns it off)
     int zero_copy;          // host steps: bit 0 = kernels read small pinned inputs, bit 1 = kernels write `out` into a pinned buffer (env AGX_ZERO_COPY, default 3)
     int stream_min_tokens;  // context length from which blocks of <= 32 rows take the tensor-core stream schedule (env AGX_STREAM_MIN_TOKENS)
     std::vector<int32_t> cu_host;  // staging for agx_verify_step_host (lives until its final sync)
@@ -56,6 +57,7 @@ struct Launch {
     Kind kind;
     int total_rows;  // sum of q_len over the launch's sequences
     int num_items;
+    int cluster;     // > 1: CTAs per cluster = KV splits of every sequence of the launch, merged in-kernel (no partials)
     std::vector<SeqPlan> seqs;
 };
 
@@ -144,12 +146,35 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
         } else {
             while (count_items(C) > std::max<long long>(target, base_items)) C += unit;
         }
+        // ---- small-q kernel: when every sequence has one row chunk and the same number of KV splits (2..16), the
+        //      splits of a (sequence, KV head) form a thread-block cluster and are merged through distributed shared
+        //      memory: no partials in global memory, no combine launch.  17..20 splits are squeezed into 16.
+        int cluster = 0;
+        if ((k == KIND_SMALL1 || k == KIND_SMALL2 || k == KIND_SMALL4) && h->cluster_merge && seqs.size() <= (size_t)kMaxSeqs) {
+            int common = -1;
+            bool ok = true;
+            for (size_t n = 0; n < seqs.size() && ok; ++n) {
+                const int L = P[seqs[n]] + Q[seqs[n]];
+                int ns = (L + C - 1) / C;
+                ns = (L + round_up((L + ns - 1) / ns, unit) - 1) / round_up((L + ns - 1) / ns, unit);
+                if (ns > 16 && ns <= 20) ns = 16;
+                ok = per_seq_items[n] == c.num_kv_heads && (common < 0 || ns == common);
+                common = ns;
+            }
+            if (ok && common >= 2 && common <= 16) {
+                const int mt = k == KIND_SMALL1 ? 1 : k == KIND_SMALL2 ? 2 : 4;
+                const int fit = attn_small_max_clusters(mt, mt == 4 ? 4 : h->small_kw, common);
+                if (fit >= base_items) cluster = common;
+                if (h->debug_plan) fprintf(stderr, "agx plan: clusters of %d: %d fit the device, %lld needed\n", common, fit, base_items);
+            }
+        }
         // ---- emit launches of at most kMaxSeqs sequences
         for (size_t a = 0; a < seqs.size(); a += kMaxSeqs) {
             Launch ln;
             ln.kind = (Kind)k;
             ln.total_rows = 0;
             ln.num_items = 0;
+            ln.cluster = cluster;
             for (size_t n = a; n < std::min(seqs.size(), a + kMaxSeqs); ++n) {
                 const int s = seqs[n];
                 const int L = P[s] + Q[s];
@@ -161,10 +186,11 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
                 sp.nsplit = (L + C - 1) / C;
                 sp.split_tokens = round_up((L + sp.nsplit - 1) / sp.nsplit, unit);
                 sp.nsplit = (L + sp.split_tokens - 1) / sp.split_tokens;
+                if (cluster) { sp.nsplit = cluster; sp.split_tokens = round_up((L + cluster - 1) / cluster, kPage); }
                 sp.row_chunks = (k == KIND_SIMT) ? 1 : (Q[s] * G + rows_per_chunk - 1) / rows_per_chunk;
                 sp.item0 = ln.num_items;
                 sp.part_base = 0;
-                if (sp.nsplit > 1) {
+                if (sp.nsplit > 1 && !cluster) {
                     if (plan.part_entries + (long long)Q[s] * c.num_q_heads * sp.nsplit > 0x7FFFFFFFll)
                         return fail(h, AGX_E_RANGE, "split partials exceed 2^31 entries");
                     sp.part_base = (int)plan.part_entries;
@@ -177,6 +203,10 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
                 ln.total_rows += Q[s];
                 ln.seqs.push_back(sp);
             }
+            if (h->debug_plan && k != KIND_TILE && k != KIND_STREAM)
+                fprintf(stderr, "agx plan: kind %d, %zu sequences, %d CTAs, first sequence %d splits of %d tokens%s\n", k,
+                        ln.seqs.size(), ln.num_items, ln.seqs[0].nsplit, ln.seqs[0].split_tokens,
+                        cluster ? ", merged in clusters" : "");
             plan.launches.push_back(std::move(ln));
         }
     }
@@ -225,6 +255,8 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     h->force_mma_sync = env ? atoi(env) : 0;
     env = getenv("AGX_STREAM_MIN_TOKENS");
     h->stream_min_tokens = env ? atoi(env) : 12288;
+    env = getenv("AGX_CLUSTER_MERGE");
+    h->cluster_merge = !(env && atoi(env) == 0);
     env = getenv("AGX_ZERO_COPY");
     h->zero_copy = env ? atoi(env) : 3;
     env = getenv("AGX_SMALL_KW");
@@ -329,10 +361,11 @@ static agx_status attn_impl(agx_handle* h, const void* q_block, const void* k_ne
         bool one_chunk = true;
         for (int i = 0; i < p.num_seqs; ++i) {
             p.seq[i] = ln.seqs[i];
-            split |= ln.seqs[i].nsplit > 1;
+            split |= ln.seqs[i].nsplit > 1 && !ln.cluster;
             one_chunk &= ln.seqs[i].row_chunks == 1;
         }
         cudaError_t e;
+        p.cluster_size = ln.cluster;
         p.k_new = p.v_new = nullptr;
         if (k_new) {
             p.k_new = k_new; p.v_new = v_new;

@@ -74,7 +74,8 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     constexpr int kWarps = MT * KW;
     constexpr int kRingBytes = NS * kStageBytes;
     constexpr int kMergeBytes = MT * kKW * 16 * (kMergeStride * 4 + 8);
-    constexpr int kRegion = kRingBytes > kMergeBytes ? kRingBytes : kMergeBytes;
+    constexpr int kClusterBytes = MT * 16 * (kD * 4 + 8);   // this CTA's (O, m, l) rows, read by the cluster's other CTAs
+    constexpr int kRegion = kRingBytes > kMergeBytes + kClusterBytes ? kRingBytes : kMergeBytes + kClusterBytes;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* ring = smem_raw + (smem_base - smem_u32(smem_raw));   // 1024-aligned: TMA swizzle atoms
     unsigned char* q_smem = ring + kRegion;
@@ -117,20 +118,6 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     }
     pdl_launch_dependents();
     pdl_wait();   // from here on global memory written by the launch before this one is read
-    if (p.k_new) append_rows_bf16(p, sp, g, tok_begin, tok_begin + sp.split_tokens, tid, kThreads);   // fused append (row_chunks == 1)
-    // ---- Q tile -> shared (rows beyond q*G are zero)
-    for (int c = tid; c < MT * 16 * 16; c += kThreads) {
-        const int r = c >> 4, ch = c & 15;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (row0 + r < rows) {
-            const int i = (row0 + r) / G, hg = (row0 + r) - i * G;
-            const long long off = ((long long)(sp.q_row0 + i) * p.hq + g * G + hg) * kRowBytes + ch * 16;
-            v = __ldg((const uint4*)((const unsigned char*)p.q + off));
-        }
-        *(uint4*)(q_smem + swz(r, ch)) = v;
-    }
-    __syncthreads();  // barriers initialised, Q tile visible
-
     // ---- producer state (warp 0; lane 0 issues the TMA copies).  Page ids are fetched 32 at a time,
     //      one group ahead, so the page-table latency never sits in front of a copy.
     const int* pt_row = p.page_table + (long long)sp.seq_index * p.pt_stride;
@@ -174,12 +161,37 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
             }
         }
     };
+    // The producer lane set the barriers up itself, so it needs nothing from the other warps: it fetches the page
+    // ids and issues the first copies at once, while the others bring the Q tile in.  Only a CTA that first writes
+    // rows of its own (fused append) holds its copies back until those rows are in place.
+    const bool early = !(p.k_new && tok_begin < L && tok_begin + sp.split_tokens > P);
     if (warp == 0) {
+        __syncwarp();   // lane 0's barrier initialisation, before the other lanes poll those barriers
         ids_cur = fetch_ids(0);
         ids_next = fetch_ids(1);
+        if (early) {
+#pragma unroll
+            for (int s = 0; s < NS - 1; ++s) produce(s);
+        }
+    }
+    if (p.k_new) append_rows_bf16(p, sp, g, tok_begin, tok_begin + sp.split_tokens, tid, kThreads);   // fused append (row_chunks == 1)
+    // ---- Q tile -> shared (rows beyond q*G are zero), by the warps other than the producer's
+    for (int c = tid - 32; c >= 0 && c < MT * 16 * 16; c += kThreads - 32) {
+        const int r = c >> 4, ch = c & 15;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (row0 + r < rows) {
+            const int i = (row0 + r) / G, hg = (row0 + r) - i * G;
+            const long long off = ((long long)(sp.q_row0 + i) * p.hq + g * G + hg) * kRowBytes + ch * 16;
+            v = __ldg((const uint4*)((const unsigned char*)p.q + off));
+        }
+        *(uint4*)(q_smem + swz(r, ch)) = v;
+    }
+    __syncthreads();  // barriers initialised, Q tile visible
+    if (warp == 0 && !early) {
 #pragma unroll
         for (int s = 0; s < NS - 1; ++s) produce(s);
     }
+
 
     uint32_t qa[8][4];
     {
@@ -340,6 +352,11 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     }
     __syncthreads();
 
+    // With clusters, the KV splits of this (sequence, KV head) are the cluster's CTAs (rank = split): the split
+    // results stay in shared memory and are merged across the cluster below instead of going through global memory.
+    const bool in_cluster = p.cluster_size > 1;
+    float* cl_o = (float*)(ring + kMergeBytes);                       // [MT*16][kD]
+    float2* cl_ml = (float2*)(ring + kMergeBytes + MT * 16 * kD * 4);  // [MT*16]
     // each thread finishes 4 consecutive columns of one row at a time
     for (int idx = tid; idx < MT * 16 * (kD / 4); idx += kThreads) {
         const int r = idx / (kD / 4);
@@ -369,11 +386,52 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
             packed.y = pack_bf16(acc.z * inv, acc.w * inv);
             *(uint2*)((__nv_bfloat16*)p.out + off) = packed;
             if (p.lse && c4 == 0) p.lse[(long long)(sp.q_row0 + i) * p.hq + h] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+        } else if (in_cluster) {
+            *(float4*)(cl_o + r * kD + c4) = acc;
+            if (c4 == 0) cl_ml[r] = make_float2(m_all, l_all);
         } else {
             const long long e = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit + split;
             *(float4*)(p.part_o + e * kD + c4) = acc;
             if (c4 == 0) p.part_ml[e] = make_float2(m_all, l_all);
         }
+    }
+    if (in_cluster && sp.nsplit > 1) {   // (uniform over the cluster: all its CTAs belong to one sequence)
+        cluster_sync();   // every split's rows are in place
+        const int cs = sp.nsplit;
+        const int n_rows = min(rows - row0, MT * 16);
+        // rows are dealt round-robin to the cluster's CTAs; one warp merges one row, lane k < cs holding split k's
+        // (m, l), every lane four columns of each split's O row (all loads in flight at once)
+        for (int r = split + warp * cs; r < n_rows; r += kWarps * cs) {
+            float2 ml = make_float2(-INFINITY, 0.f);
+            if (lane < cs) ml = ld_cluster_f2(cluster_map(smem_u32(cl_ml + r), lane));
+            float m_all = ml.x;
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, d));
+            const float w = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m_all);
+            float l_all = ml.y * w;
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) l_all += __shfl_xor_sync(0xFFFFFFFFu, l_all, d);
+            const uint32_t row_addr = smem_u32(cl_o + r * kD + lane * 4);
+            float4 v[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k)
+                if (k < cs) v[k] = ld_cluster_f4(cluster_map(row_addr, k));
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                const float wk = __shfl_sync(0xFFFFFFFFu, w, k);
+                if (k < cs && wk != 0.f) { acc.x += v[k].x * wk; acc.y += v[k].y * wk; acc.z += v[k].z * wk; acc.w += v[k].w * wk; }
+            }
+            const int i = (row0 + r) / G, hg = (row0 + r) - i * G;
+            const int h = g * G + hg;
+            const float inv = 1.f / l_all;
+            uint2 packed;
+            packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+            packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+            *(uint2*)((__nv_bfloat16*)p.out + ((long long)(sp.q_row0 + i) * p.hq + h) * kD + lane * 4) = packed;
+            if (p.lse && lane == 0) p.lse[(long long)(sp.q_row0 + i) * p.hq + h] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+        }
+        cluster_sync();   // no CTA leaves while its rows may still be read
     }
 }
 
@@ -485,12 +543,17 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
     float m_all, l_all;
     if (ns <= 32) {
         // One round trip to memory: lane k fetches (m, l) of split k while every lane already fetches its
-        // columns of up to 16 splits' O rows; the weights then travel by shuffle, splits in index order.
+        // columns of every split's O row; the weights then travel by shuffle, splits in index order.
         const float2 ml = (lane < ns) ? p.part_ml[e0 + lane] : make_float2(-INFINITY, 0.f);
-        float4 v[16];
+        float4 v[16], v2[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j)
             if (j < ns && c4 < D) v[j] = *(const float4*)(p.part_o + (e0 + j) * D + c4);
+        if (ns > 16) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (16 + j < ns && c4 < D) v2[j] = *(const float4*)(p.part_o + (e0 + 16 + j) * D + c4);
+        }
         m_all = ml.x;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, off));
@@ -507,13 +570,10 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
         }
         if (ns > 16) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
-                if (16 + j < ns && c4 < D) v[j] = *(const float4*)(p.part_o + (e0 + 16 + j) * D + c4);
-#pragma unroll
             for (int j = 0; j < 16; ++j) {
                 const float w = __shfl_sync(0xFFFFFFFFu, w_mine, 16 + j);
                 if (16 + j < ns && w != 0.f && c4 < D) {
-                    acc.x += v[j].x * w; acc.y += v[j].y * w; acc.z += v[j].z * w; acc.w += v[j].w * w;
+                    acc.x += v2[j].x * w; acc.y += v2[j].y * w; acc.z += v2[j].z * w; acc.w += v2[j].w * w;
                 }
             }
         }
@@ -572,11 +632,16 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
 // --------------------------------------------------------------------------------------------
 namespace {
 template <int MT, int KW, int NS>
-cudaError_t launch_small(const AttnParams& p, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
-    constexpr int kMergeBytes = MT * KW * 16 * (kMergeStride * 4 + 8);
+constexpr int small_smem_bytes() {
+    constexpr int kMergeBytes = MT * KW * 16 * (kMergeStride * 4 + 8) + MT * 16 * (kD * 4 + 8);   // + the cluster rows
     constexpr int kRing = NS * 2 * KW * kPage * kRowBytes;
     // [ring | merge region][Q tile][2 * NS barriers + abort flag] + slack for the 1024-byte alignment
-    constexpr int kSmem = (kRing > kMergeBytes ? kRing : kMergeBytes) + MT * 16 * kRowBytes + 2 * NS * 8 + 16 + 1024;
+    return (kRing > kMergeBytes ? kRing : kMergeBytes) + MT * 16 * kRowBytes + 2 * NS * 8 + 16 + 1024;
+}
+
+template <int MT, int KW, int NS>
+cudaError_t launch_small(const AttnParams& p, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
+    constexpr int kSmem = small_smem_bytes<MT, KW, NS>();
     // the attribute is per device: remember which devices have it (a process normally drives one GPU)
     static bool configured_on[64] = {false};
     int device = 0;
@@ -585,11 +650,51 @@ cudaError_t launch_small(const AttnParams& p, const CUtensorMap& map_k, const CU
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
         if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);   // clusters of up to 16
+        if (e != cudaSuccess) return e;
         configured = true;
     }
+    if (p.cluster_size > 1)
+        return launch_chained_cluster(attn_small_bf16_kernel<MT, KW, NS>, dim3(p.num_items), dim3(32 * MT * KW), kSmem,
+                                      (unsigned)p.cluster_size, stream, p, map_k, map_v);
     return launch_chained(attn_small_bf16_kernel<MT, KW, NS>, dim3(p.num_items), dim3(32 * MT * KW), kSmem, stream, p, map_k, map_v);
 }
+
+template <int MT, int KW, int NS>
+int max_clusters(int cluster) {
+    static int cached[64][17];   // 0 = not asked yet, else 1 + answer
+    int device = 0;
+    if (cluster < 2 || cluster > 16 || cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return 0;
+    if (cached[device][cluster]) return cached[device][cluster] - 1;
+    constexpr int kSmem = small_smem_bytes<MT, KW, NS>();
+    int n = 0;
+    if (cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) == cudaSuccess &&
+        cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(cluster * 64); cfg.blockDim = dim3(32 * MT * KW); cfg.dynamicSmemBytes = kSmem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        if (cudaOccupancyMaxActiveClusters(&n, attn_small_bf16_kernel<MT, KW, NS>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+    } else {
+        (void)cudaGetLastError();
+    }
+    cached[device][cluster] = n + 1;
+    return n;
+}
 }  // namespace
+
+int attn_small_max_clusters(int mt, int kw, int cluster) {
+    switch (mt * 16 + kw) {
+        case 1 * 16 + 4: return max_clusters<1, 4, 3>(cluster);
+        case 2 * 16 + 4: return max_clusters<2, 4, 3>(cluster);
+        case 1 * 16 + 8: return max_clusters<1, 8, 3>(cluster);
+        case 2 * 16 + 8: return max_clusters<2, 8, 3>(cluster);
+        case 4 * 16 + 4: return max_clusters<4, 4, 5>(cluster);
+        default: return 0;
+    }
+}
 
 cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, int kw, cudaStream_t stream) {
     if (p.num_items == 0) return cudaSuccess;

@@ -35,6 +35,7 @@ struct AttnParams {
     float* part_o;   // [entries][head_dim] fp32, un-normalised, relative to part_ml.x
     float2* part_ml; // [entries] (running max in log2 units, sum)
     int* status;
+    int cluster_size;    // > 1: the launch's CTAs form clusters of this size = the KV splits of one (sequence, KV head), merged in-kernel
     const void* k_new;   // fused append (agx_attn_prefixed_append): the block's K/V rows [total_q][hkv][d], or NULL
     const void* v_new;
     long long num_pages;
@@ -59,6 +60,21 @@ cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+// The same with thread-block clusters of `cluster` CTAs along x (grid.x a multiple of it).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, unsigned cluster,
+                                   cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
@@ -90,6 +106,9 @@ cudaError_t launch_kv_append(int dtype, void* k_pool, void* v_pool, long long nu
 
 // Small-q split-KV kernel (bf16, d = 128, tensor-core mma.sync); mt = m-tiles of 16 rows (1, 2, 4), kw = KV groups
 // (4 or 8 pages per pipeline stage; 8 only with mt <= 2): CTA = 32 * mt * kw threads.
+// Clusters of `cluster` CTAs of the small-q kernel <mt, kw> that can be resident at once on the current device
+// (0 when such a cluster cannot be launched); cached per device.
+int attn_small_max_clusters(int mt, int kw, int cluster);
 cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, int kw, cudaStream_t stream);
 // Scalar fp32-math kernel for AGX_F32 pools (any q, d in {64, 128}).
 cudaError_t launch_attn_simt_f32(const AttnParams& p, cudaStream_t stream);

@@ -134,6 +134,27 @@ def test_small_q_shapes(P, q, hq, hkv):
     run_and_check(w, poison=True)
 
 
+@pytest.mark.parametrize("merge", ["clusters", "combine_kernel"])
+@pytest.mark.parametrize("P,q,hq,hkv,batch", [
+    (4096, 8, 32, 8, 1),      # 17 splits squeezed into clusters of 16 where eight such clusters fit the device
+    (4096, 1, 32, 8, 1), (3000, 5, 32, 8, 1), (700, 8, 32, 8, 1), (300, 2, 32, 8, 1), (1000, 3, 24, 8, 1),
+    (6000, 7, 8, 8, 1), (2500, 12, 4, 1, 1), (4090, 16, 32, 8, 1),
+    (4096, 8, 32, 8, 4),      # four equal sequences: clusters of 4
+    (2000, 4, 32, 8, 2),
+])
+def test_small_q_split_merge_in_clusters_and_by_combine_kernel(P, q, hq, hkv, batch, merge, monkeypatch):
+    """The KV splits of the warp-MMA kernel merged through the clusters' shared memory (one launch) and through
+    partials in global memory plus the combine kernel (two launches): both against the oracle."""
+    monkeypatch.setenv("AGX_CLUSTER_MERGE", "1" if merge == "clusters" else "0")
+    w = W.make_attn_workload(f"cl_{P}_{q}_{batch}", 500 + P + q, "bf16", hq, hkv, 128, [P + 16 * i for i in range(batch)] if batch == 2 else [P] * batch,
+                             [q] * batch, spare_pages=2)
+    b, _ = run_and_check(w, poison=True, sample=(5, 24) if batch > 1 else None)
+    if merge == "clusters" and batch == 1 and 700 <= P <= 1000:     # clusters of 3 or 4 fit any device; one launch, no combine
+        assert b.launches == 1
+    if merge == "combine_kernel" and P >= 700:
+        assert b.launches == 2
+
+
 def test_small_q_ragged_batch_with_shared_prefix():
     P = [2048, 2100, 4000, 2048 + 15, 9000, 2500, 3001, 2048]
     q = [1, 2, 4, 8, 16, 3, 5, 8]
