@@ -117,12 +117,12 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&map_v) : "memory");
     }
     pdl_launch_dependents();
-    pdl_wait();   // from here on global memory written by the launch before this one is read
-    // ---- producer state (warp 0; lane 0 issues the TMA copies).  Page ids are fetched 32 at a time,
-    //      one group ahead, so the page-table latency never sits in front of a copy.
     const int* pt_row = p.page_table + (long long)sp.seq_index * p.pt_stride;
     const int page0 = tok_begin / kPage;
     const int n_pages = (tok_end - tok_begin + kPage - 1) / kPage;
+    pdl_wait();   // from here on global memory written by the launch before this one is read
+    // ---- producer state (warp 0; lane 0 issues the TMA copies).  Page ids are fetched 32 at a time,
+    //      one group ahead, so the page-table latency never sits in front of a copy.
     int ids_cur = 0, ids_next = 0, group_cur = 0;
     auto fetch_ids = [&](int group) {
         const int pi = group * 32 + lane;
