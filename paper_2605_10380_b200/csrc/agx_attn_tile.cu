@@ -70,7 +70,10 @@ constexpr int kPolyPairsOf8 = AGX_POLY_PAIRS;
 
 // barrier slots (8 bytes each)
 enum { BAR_K_FULL = 0, BAR_K_EMPTY = 3, BAR_V_FULL = 6, BAR_V_EMPTY = 9, BAR_S_FULL = 12, BAR_P_READY = 14,
-       BAR_O_FULL = 16, BAR_Q_FULL = 17, BAR_COUNT = 18 };
+       BAR_O_FULL = 16, BAR_Q_FULL = 17, BAR_P_TAIL = 18, BAR_COUNT = 20 };
+// P is handed to the MMA warp in two parts: the first kPvHeadSteps k-steps (16 tokens each) as soon as they are
+// stored, so that their PV MMAs run while the softmax warpgroup still works on the last columns
+constexpr int kPvHeadSteps = 6;
 constexpr int kQLoadThreads = kThreads - 64;  // warps 2..11 bring the Q tiles in
 constexpr int kRegsLow = 96, kRegsHigh = 200; // 128 * 96 + 256 * 200 <= 384 * 168
 
@@ -108,6 +111,10 @@ __device__ __forceinline__ void tmem_ld_x32(uint32_t taddr, uint32_t* r) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st_x16(uint32_t taddr, const uint32_t* r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n"
+                 :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]));
 }
 __device__ __forceinline__ void tmem_st_x32(uint32_t taddr, const uint32_t* r) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n"
@@ -154,9 +161,6 @@ __device__ __forceinline__ void ex2_poly2(uint64_t x, float& p0, float& p1) {
     upk2(t, t0, t1);
     p0 = __int_as_float(__float_as_int(t0) * 8388608 + __float_as_int(q0));
     p1 = __int_as_float(__float_as_int(t1) * 8388608 + __float_as_int(q1));
-}
-__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b, float c) {
-    upk2(fma2p(pk2(a0, a1), pk2(b, b), pk2(c, c)), d0, d1);
 }
 __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
     upk2(add2p(pk2(d0, d1), pk2(a0, a1)), d0, d1);
@@ -369,7 +373,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
     // ---- setup: barriers, TMEM, Q tiles
     if (tid == 0) {
         for (int i = 0; i < BAR_COUNT; ++i)
-            mbar_init(bar(i), (i == BAR_P_READY || i == BAR_P_READY + 1) ? 128u : (i == BAR_Q_FULL) ? (uint32_t)kQLoadThreads : 1u);
+            mbar_init(bar(i), (i == BAR_P_READY || i == BAR_P_READY + 1 || i == BAR_P_TAIL || i == BAR_P_TAIL + 1) ? 128u : (i == BAR_Q_FULL) ? (uint32_t)kQLoadThreads : 1u);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&map_k) : "memory");
@@ -496,14 +500,22 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                     umma_ss(tS[x], q_desc[qt] + off, kd + off, kIdescQK, ks > 0);
                 }
             };
-            auto issue_pv = [&](int x, int stage, int npg, bool first) {  // O_x += P_x V : one k-step per page
+            // O_x += P_x V, one k-step per page: the head part (pages 0 .. kPvHeadSteps-1) once P_READY says those columns
+            // of P are stored, the tail part after P_TAIL
+            auto issue_pv = [&](int x, int stage, int npg, bool first, bool tail) {
                 const uint64_t vd = make_desc(smem_base + v_stage_off(stage), kHalfBytes, 1024);
                 if (npg == 8) {
+                    if (!tail) {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        umma_ts(tO[x], tS[x] + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescPV, !(first && ks == 0));
+                        for (int ks = 0; ks < kPvHeadSteps; ++ks)
+                            umma_ts(tO[x], tS[x] + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescPV, !(first && ks == 0));
+                    } else {
+#pragma unroll
+                        for (int ks = kPvHeadSteps; ks < 8; ++ks)
+                            umma_ts(tO[x], tS[x] + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescPV, true);
+                    }
                 } else {
-                    for (int ks = 0; ks < npg; ++ks)
+                    for (int ks = tail ? kPvHeadSteps : 0; ks < (tail ? npg : min(npg, kPvHeadSteps)); ++ks)
                         umma_ts(tO[x], tS[x] + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescPV, !(first && ks == 0));
                 }
             };
@@ -524,7 +536,11 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                     ok = mbar_wait(bar(BAR_P_READY + x), (t >> 1) & 1, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv(x, vs, npg, t < 2);
+                    issue_pv(x, vs, npg, t < 2, false);
+                    ok = mbar_wait(bar(BAR_P_TAIL + x), (t >> 1) & 1, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(x, vs, npg, t < 2, true);
                     umma_commit(bar(BAR_V_EMPTY + vs));
                     if (t + 2 < n_tiles) {
                         const int nks = (t + 2) % kStagesK, nkph = ((t + 2) / kStagesK) & 1;
@@ -552,7 +568,11 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                 ok = mbar_wait(bar(BAR_P_READY + 0), t & 1, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
-                issue_pv(0, vs, npg, t == 0);
+                issue_pv(0, vs, npg, t == 0, false);
+                ok = mbar_wait(bar(BAR_P_TAIL + 0), t & 1, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                issue_pv(0, vs, npg, t == 0, true);
                 if (more) {
                     ok = mbar_wait(bar(BAR_K_FULL + nks), nkph, abort_flag, p.status);
                     if (!ok) break;
@@ -562,7 +582,11 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                 ok = mbar_wait(bar(BAR_P_READY + 1), t & 1, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
-                issue_pv(1, vs, npg, t == 0);
+                issue_pv(1, vs, npg, t == 0, false);
+                ok = mbar_wait(bar(BAR_P_TAIL + 1), t & 1, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                issue_pv(1, vs, npg, t == 0, true);
                 umma_commit(bar(BAR_V_EMPTY + vs));
                 if (more) {
                     issue_qk(1, nks, 1); umma_commit(bar(BAR_S_FULL + 1));
@@ -603,7 +627,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         if (!warp_has_rows) {   // keep S_FULL / P_READY in step, nothing else
             for (int t = t_first; t < n_tiles && ok; t += kStep) {
                 ok = mbar_wait(bar(BAR_S_FULL + x), ((t - t_first) / kStep) & 1, abort_flag, p.status);
-                if (ok) mbar_arrive(bar(BAR_P_READY + x));
+                if (ok) { mbar_arrive(bar(BAR_P_READY + x)); mbar_arrive(bar(BAR_P_TAIL + x)); }
             }
         } else
         for (int t = t_first; t < n_tiles; t += kStep) {
@@ -617,23 +641,52 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             tmem_wait_ld();
             const int tok0 = kv_begin + t * kBN;
             const bool masked = (tok0 + kBN - 1 > P + tile_i_min) || (tok0 + kBN > kv_end);  // uniform per tile
-            const uint64_t sc2 = pk2(sc, sc);
             float lt0 = 0.f, lt1 = 0.f, lt2 = 0.f, lt3 = 0.f;   // this tile's row sum, four partial sums
-            bool done = false;
-            if (j > 0 && !masked) {
-                // ---- common case, one sweep: exponentials against the running reference m_ref (the
-                //      maximum of earlier tiles, so P may exceed 1) while the tile's own maximum is
-                //      collected on the side; only if that maximum tops m_ref by more than 2^8 is the
-                //      tile redone below with a new reference.
-                const uint64_t nm2 = pk2(-m_ref, -m_ref);
-                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            if (masked) {
+                const int nvis = max(0, min(min(limit + 1, kv_end) - tok0, kBN));        // visible columns: [0, nvis)
 #pragma unroll
-                for (int c = 0; c < 128; c += 4) {   // in place: sreg[c / 2] <- (p[c], p[c + 1])
-                    const float s0 = __uint_as_float(sreg[c]), s1 = __uint_as_float(sreg[c + 1]);
-                    const float s2 = __uint_as_float(sreg[c + 2]), s3 = __uint_as_float(sreg[c + 3]);
-                    mx[(c >> 2) & 3] = max3(mx[(c >> 2) & 3], s0, s1);
-                    mx[((c >> 2) + 2) & 3] = max3(mx[((c >> 2) + 2) & 3], s2, s3);
-                    const uint64_t xa = fma2p(pk2(s0, s1), sc2, nm2), xb = fma2p(pk2(s2, s3), sc2, nm2);
+                for (int c = 0; c < 128; ++c)
+                    if (c >= nvis) sreg[c] = 0xFF800000u;  // -inf: its exponential is exactly 0
+            }
+            // ---- row maximum (four independent chains of 3-input max).  The exponentials below are taken against the
+            //      running reference m_ref (the maximum of earlier tiles, so P may exceed 1); only if this tile's
+            //      maximum tops it by more than 2^8 is the reference moved and O rescaled.
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int c = 0; c < 128; c += 8) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    mx[k] = max3(mx[k], __uint_as_float(sreg[c + 2 * k]), __uint_as_float(sreg[c + 2 * k + 1]));
+            }
+            const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;
+            const bool need = m_tile > m_ref + kRescaleThreshold;
+            if (__any_sync(0xFFFFFFFFu, need)) {
+                const float m_new = need ? m_tile : m_ref;
+                const float factor = need ? ex2(m_ref - m_new) : 1.f;   // m_ref = -inf gives 0
+                if (j > 0) {
+                    uint32_t oreg[32];
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        tmem_ld_x32(tO + c4 * 32, oreg);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * factor);
+                        tmem_st_x32(tO + c4 * 32, oreg);
+                    }
+                    tmem_wait_st();
+                }
+                l_run *= factor;
+                m_ref = m_new;
+            }
+            // ---- P = 2^(S * scale - m_ref) as packed bf16 pairs, in place: sreg[c / 2] <- (p[c], p[c + 1]); the
+            //      first kPvHeadSteps * 16 columns are stored and handed over before the rest is computed
+            const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+            const uint64_t sc2 = pk2(sc, sc), nm2 = pk2(neg_m, neg_m);
+            auto sweep = [&](const int c_lo, const int c_hi) {
+#pragma unroll
+                for (int c = c_lo; c < c_hi; c += 4) {
+                    const uint64_t xa = fma2p(pk2(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])), sc2, nm2);
+                    const uint64_t xb = fma2p(pk2(__uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3])), sc2, nm2);
                     float a0, a1, b0, b1;
                     if (((c >> 1) & 7) < kPolyPairsOf8) ex2_poly2(xa, a0, a1);
                     else { upk2(xa, a0, a1); a0 = ex2(a0); a1 = ex2(a1); }
@@ -644,71 +697,20 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                     sreg[c >> 1] = pack_bf16(a0, a1);
                     sreg[(c >> 1) + 1] = pack_bf16(b0, b1);
                 }
-                const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;
-                if (!__any_sync(0xFFFFFFFFu, m_tile > m_ref + kRescaleThreshold)) {
-                    done = true;
-                } else {   // rare: fetch the scores again (P has not been stored over them yet)
-                    lt0 = lt1 = lt2 = lt3 = 0.f;
-#pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) tmem_ld_x32(tS + c4 * 32, sreg + c4 * 32);
-                    tmem_wait_ld();
-                }
-            }
-            if (!done) {
-                if (masked) {
-                    const int nvis = max(0, min(min(limit + 1, kv_end) - tok0, kBN));        // visible columns: [0, nvis)
-#pragma unroll
-                    for (int c = 0; c < 128; ++c)
-                        if (c >= nvis) sreg[c] = 0xFF800000u;  // -inf: its exponential is exactly 0
-                }
-                // ---- row maximum (four independent chains of 3-input max)
-                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-                for (int c = 0; c < 128; c += 8) {
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        mx[k] = max3(mx[k], __uint_as_float(sreg[c + 2 * k]), __uint_as_float(sreg[c + 2 * k + 1]));
-                }
-                const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sc;
-                const bool need = m_tile > m_ref + kRescaleThreshold;
-                if (__any_sync(0xFFFFFFFFu, need)) {
-                    const float m_new = need ? m_tile : m_ref;
-                    const float factor = need ? ex2(m_ref - m_new) : 1.f;   // m_ref = -inf gives 0
-                    if (j > 0) {
-                        uint32_t oreg[32];
-#pragma unroll
-                        for (int c4 = 0; c4 < 4; ++c4) {
-                            tmem_ld_x32(tO + c4 * 32, oreg);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * factor);
-                            tmem_st_x32(tO + c4 * 32, oreg);
-                        }
-                        tmem_wait_st();
-                    }
-                    l_run *= factor;
-                    m_ref = m_new;
-                }
-                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-                // ---- P = 2^(S * scale - m) as packed bf16 pairs, in place: sreg[c / 2] <- (p[c], p[c + 1])
-#pragma unroll
-                for (int c = 0; c < 128; c += 4) {
-                    float a0, a1, b0, b1;
-                    fma2(a0, a1, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]), sc, neg_m);
-                    fma2(b0, b1, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]), sc, neg_m);
-                    a0 = ex2(a0); a1 = ex2(a1); b0 = ex2(b0); b1 = ex2(b1);
-                    add2(lt0, lt1, a0, a1);
-                    add2(lt2, lt3, b0, b1);
-                    sreg[c >> 1] = pack_bf16(a0, a1);
-                    sreg[(c >> 1) + 1] = pack_bf16(b0, b1);
-                }
-            }
-            l_run += (lt0 + lt1) + (lt2 + lt3);
+            };
+            constexpr int kHeadCols = kPvHeadSteps * 16;   // 96 score columns = 48 packed registers
+            sweep(0, kHeadCols);
             tmem_st_x32(tS, sreg);
-            tmem_st_x32(tS + 32, sreg + 32);
+            tmem_st_x16(tS + 32, sreg + 32);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(BAR_P_READY + x));
+            sweep(kHeadCols, 128);
+            l_run += (lt0 + lt1) + (lt2 + lt3);
+            tmem_st_x16(tS + 48, sreg + 48);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar(BAR_P_TAIL + x));
         }
         if (ok) ok = mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
         if (ok || kStreams) tile_epilogue<kStreams>(smem, tO, m_ref, l_run, ok);
