@@ -11,10 +11,12 @@
 // owns query rows [16 mt, 16 mt + 16) and, in every stage of KW pages, page kg.  K/V pages stream through a
 // 3-stage ring filled by TMA (per page two [16 tokens][64 dims] boxes for K and for V, SWIZZLE_128B so
 // ldmatrix is conflict-free; page ids come from the page table, prefetched 32 at a time) and handed over
-// with full/empty mbarriers, so no thread spends instructions on addresses and warps never meet at a
-// CTA-wide barrier inside the loop; the KV groups keep private online-softmax states that are merged
-// through shared memory at the end.  KW = 8 (16 warps for a 32-row verify block, one CTA per SM) halves the
-// number of dependent page steps per warp, which is what a 4k-token context is bounded by.  Splits write
+// with full/empty mbarriers, so no thread spends instructions on addresses.  Per stage the KV groups of an
+// m-tile meet twice at a named barrier: once to agree on the rows' running maximum (page maxima through
+// shared memory), once to hand round the pages' P (as MMA A fragments, 512 bytes per page).  Each warp
+// then accumulates O over all pages of the stage, but only for the 128 / KW output columns it owns, so
+// the accumulators never have to be merged: at the end only the row sums are added up.  KW = 8 (16 warps
+// for a 32-row verify block, one CTA per SM) halves the number of page steps per warp.  Splits write
 // fp32 (m, l, O) partials; a combine kernel merges them in fixed order, so results are bit-reproducible
 // run to run.
 #include <math.h>
@@ -29,7 +31,6 @@ namespace {
 constexpr int kD = 128;                    // head dim of the bf16 kernels
 constexpr int kRowBytes = kD * 2;          // one (token, head) row
 // KW = KV groups = pages per pipeline stage (4 or 8): stage = KW * 16 tokens, K + V = KW * 8 KB
-constexpr int kMergeStride = 136;          // floats per merged row (conflict-free float2 stores)
 
 
 
@@ -73,14 +74,17 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     constexpr int kThreads = 32 * MT * KW;
     constexpr int kWarps = MT * KW;
     constexpr int kRingBytes = NS * kStageBytes;
-    constexpr int kMergeBytes = MT * kKW * 16 * (kMergeStride * 4 + 8);
-    constexpr int kClusterBytes = MT * 16 * (kD * 4 + 8);   // this CTA's (O, m, l) rows, read by the cluster's other CTAs
-    constexpr int kRegion = kRingBytes > kMergeBytes + kClusterBytes ? kRingBytes : kMergeBytes + kClusterBytes;
+    constexpr int kClusterBytes = MT * 16 * (kD * 4 + 8);   // this CTA's (O, m, l) rows, read by the cluster's other CTAs (in the dead ring)
+    constexpr int kRegion = kRingBytes > kClusterBytes ? kRingBytes : kClusterBytes;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* ring = smem_raw + (smem_base - smem_u32(smem_raw));   // 1024-aligned: TMA swizzle atoms
     unsigned char* q_smem = ring + kRegion;
     const uint32_t bar_base = smem_base + kRegion + MT * 16 * kRowBytes;  // full[NS], empty[NS]
     volatile int* abort_flag = (volatile int*)(q_smem + MT * 16 * kRowBytes + 2 * NS * 8);
+    // exchange area of the KV groups: per-page row maxima, per-group row sums, P fragments of the stage's pages
+    float* x_max = (float*)(q_smem + MT * 16 * kRowBytes + 2 * NS * 8 + 16);   // [MT][16][KW]
+    float* x_l = x_max + MT * 16 * KW;                                          // [MT][16][KW]
+    uint4* x_p = (uint4*)(x_l + MT * 16 * KW);                                  // [MT][KW][32]
     auto full_bar = [&](int i) { return bar_base + 8u * i; };
     auto empty_bar = [&](int i) { return bar_base + 8u * (NS + i); };
 
@@ -203,11 +207,15 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
         }
     }
 
-    float o[16][4];
+    // Warp (mt, kg) scores page kg of every stage against its 16 rows, but accumulates O only for the kCG * 16
+    // output columns it owns, over ALL pages of the stage: the P fragments of the stage's pages travel through shared
+    // memory and the KV groups of an m-tile share one running maximum, so nothing has to be merged at the end.
+    constexpr int kCG = 8 / KW;                    // 16-column groups of O per warp
+    float o[2 * kCG][4];
 #pragma unroll
-    for (int n = 0; n < 16; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
-    float m_run[2] = {-INFINITY, -INFINITY};
-    float l_run[2] = {0.f, 0.f};
+    for (int n = 0; n < 2 * kCG; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+    float m_run[2] = {-INFINITY, -INFINITY};       // the m-tile's running maximum of rows g and g + 8 (log2 units)
+    float l_run[2] = {0.f, 0.f};                   // this lane's share of this KV group's row sums
 
     // row limits (last visible token) for the two rows this thread holds
     int limit[2];
@@ -227,17 +235,29 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
 #pragma unroll
     for (int j = 0; j < 4; ++j) v_off[j] = v_row * 128 + ((v_x ^ (uint32_t)(j << 1)) << 4);
 
+    const int rg = lane >> 2;                      // this lane's rows in the m-tile: rg and rg + 8
+    float* my_max = x_max + (mt * 16 + rg) * KW;   // x_max[mt][row][kg]
+    uint4* my_p = x_p + (mt * KW) * 32 + lane;     // x_p[mt][kg][lane]: page kg's P as the lanes' MMA A fragments
+    auto group_sync = [&]() { asm volatile("bar.sync %0, %1;\n" ::"r"(1 + mt), "n"(32 * KW) : "memory"); };
+
+    bool live = true;   // a warp whose wait gave up keeps meeting the others at the group barriers
     for (int stage = 0; stage < n_stages; ++stage) {
         const int slot = stage % NS;
         if (warp == 0) produce(stage + NS - 1);
-        if (!mbar_wait(full_bar(slot), (stage / NS) & 1, abort_flag, p.status)) break;
+        if (live) live = mbar_wait(full_bar(slot), (stage / NS) & 1, abort_flag, p.status);
 
-        const int tok0 = tok_begin + stage * kStageTokens + kg * kPage;
-        if (tok0 < tok_end) {
-            const uint32_t k_base = smem_base + slot * kStageBytes + kg * 4096;
+        const int stage_tok0 = tok_begin + stage * kStageTokens;
+        const int npg = live ? min(kKW, (tok_end - stage_tok0 + kPage - 1) / kPage) : 0;   // pages of this stage
+        const int tok0 = stage_tok0 + kg * kPage;
+        const bool has_page = kg < npg;
+        const uint32_t stage_base = smem_base + slot * kStageBytes;
+        float s[2][4];
+        float mx[2] = {-INFINITY, -INFINITY};
+        if (has_page) {
+            const uint32_t k_base = stage_base + kg * 4096;
             const uint32_t v_base = k_base + kStageTokens * kRowBytes;
             // slots past the end of the sequence may hold anything: zero those V rows (P is 0 there,
-            // but 0 * NaN is not).  Every warp sharing the page writes the same zeros.
+            // but 0 * NaN is not).  Every warp that scores the page writes the same zeros.
             if (tok0 + kPage > L) {
                 const int valid_rows = L - tok0;
                 for (int idx = lane; idx < (kPage - valid_rows) * 16; idx += 32) {
@@ -246,11 +266,9 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
                 }
                 __syncwarp();
             }
-
-            // S = Q K^T for 16 tokens: two n-tiles of 8 tokens
-            // four accumulation chains of four MMAs each (even and odd k-steps of both n-tiles) instead of two
-            // of eight: a dependent mma.sync is slow to issue, and this chain sits on every page's critical path
-            float s[2][4], s_odd[2][4];
+            // S = Q K^T for 16 tokens: two n-tiles of 8 tokens, as four accumulation chains of four MMAs each
+            // (even and odd k-steps of both n-tiles): a dependent mma.sync is slow to issue
+            float s_odd[2][4];
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt) {
                 s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
@@ -282,117 +300,127 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
                     }
                 }
             }
-            // online softmax for rows A (e = 0,1) and B (e = 2,3); running max kept in log2 units
-            float corr[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                float mx = fmaxf(fmaxf(s[0][2 * h], s[0][2 * h + 1]), fmaxf(s[1][2 * h], s[1][2 * h + 1]));
-                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
-                const float m_new = fmaxf(m_run[h], mx * p.scale_log2);
-                const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
-                corr[h] = ex2(m_run[h] - m_ref);
-                m_run[h] = m_new;
-                float sum = 0.f;
+                float v = fmaxf(fmaxf(s[0][2 * h], s[0][2 * h + 1]), fmaxf(s[1][2 * h], s[1][2 * h + 1]));
+                v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, 1));
+                v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, 2));
+                mx[h] = v * p.scale_log2;
+            }
+        }
+        if ((lane & 3) == 0) { my_max[kg] = mx[0]; my_max[8 * KW + kg] = mx[1]; }
+        group_sync();   // the stage's page maxima of this m-tile are in place
+
+        // one running maximum per row for the whole m-tile; P of this warp's page against it
+        float corr[2];
+        uint32_t pa[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            float m_new = m_run[h];
+#pragma unroll
+            for (int k4 = 0; k4 < KW; k4 += 4) {
+                const float4 v = *(const float4*)(my_max + h * 8 * KW + k4);
+                m_new = fmaxf(fmaxf(m_new, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+            }
+            const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
+            corr[h] = ex2(m_run[h] - m_ref);
+            m_run[h] = m_new;
+            float sum = 0.f;
+            if (has_page) {
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt) {
                     s[nt][2 * h] = ex2(fmaf(s[nt][2 * h], p.scale_log2, -m_ref));
                     s[nt][2 * h + 1] = ex2(fmaf(s[nt][2 * h + 1], p.scale_log2, -m_ref));
                     sum += s[nt][2 * h] + s[nt][2 * h + 1];
                 }
-                l_run[h] = l_run[h] * corr[h] + sum;
             }
-            if (__any_sync(0xFFFFFFFFu, corr[0] != 1.f || corr[1] != 1.f)) {
-#pragma unroll
-                for (int n = 0; n < 16; ++n) {
-                    o[n][0] *= corr[0]; o[n][1] *= corr[0];
-                    o[n][2] *= corr[1]; o[n][3] *= corr[1];
-                }
-            }
-            // O += P V
-            uint32_t pa[4];
+            l_run[h] = l_run[h] * corr[h] + sum;
+        }
+        if (has_page) {
             pa[0] = pack_bf16(s[0][0], s[0][1]);
             pa[1] = pack_bf16(s[0][2], s[0][3]);
             pa[2] = pack_bf16(s[1][0], s[1][1]);
             pa[3] = pack_bf16(s[1][2], s[1][3]);
+        }
+        my_p[kg * 32] = make_uint4(pa[0], pa[1], pa[2], pa[3]);
+        if (__any_sync(0xFFFFFFFFu, corr[0] != 1.f || corr[1] != 1.f)) {
 #pragma unroll
-            for (int cp = 0; cp < 8; ++cp) {
-                uint32_t b0, b1, b2, b3;
-                ldmatrix_x4_trans(b0, b1, b2, b3, v_base + (cp >> 2) * 2048 + v_off[cp & 3]);
-                mma_bf16(o[2 * cp], pa, b0, b1);
-                mma_bf16(o[2 * cp + 1], pa, b2, b3);
+            for (int n = 0; n < 2 * kCG; ++n) {
+                o[n][0] *= corr[0]; o[n][1] *= corr[0];
+                o[n][2] *= corr[1]; o[n][3] *= corr[1];
+            }
+        }
+        group_sync();   // every page's P fragments (and zeroed V rows) are in place
+
+        // O[:, this warp's columns] += P V over the stage's pages
+#pragma unroll
+        for (int k = 0; k < kKW; ++k) {
+            if (k < npg) {
+                const uint4 pk = my_p[k * 32];
+                const uint32_t a[4] = {pk.x, pk.y, pk.z, pk.w};
+                const uint32_t v_base = stage_base + kStageTokens * kRowBytes + k * 4096;
+#pragma unroll
+                for (int c = 0; c < kCG; ++c) {
+                    const int cp = kg * kCG + c;
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4_trans(b0, b1, b2, b3, v_base + (cp >> 2) * 2048 + v_off[cp & 3]);
+                    mma_bf16(o[2 * c], a, b0, b1);
+                    mma_bf16(o[2 * c + 1], a, b2, b3);
+                }
             }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(empty_bar(slot));
+        if (live && lane == 0) mbar_arrive(empty_bar(slot));
     }
-    __syncthreads();  // every armed stage has been consumed: the ring is dead, reuse it for the merge
 
-    // ---- merge the 4 KV groups of each m-tile through shared memory
-    float* merge_o = (float*)ring;                                    // [MT*4][16][kMergeStride]
-    float2* merge_ml = (float2*)(ring + MT * kKW * 16 * kMergeStride * 4);  // [MT*4][16]
-    {
+    // ---- row sums of the m-tile: each KV group's share through shared memory
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 1);
-            l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 2);
-        }
-        float* mo = merge_o + (size_t)(mt * kKW + kg) * 16 * kMergeStride;
-        const int rA = lane >> 2;
-#pragma unroll
-        for (int n = 0; n < 16; ++n) {
-            const int col = n * 8 + 2 * (lane & 3);
-            *(float2*)(mo + rA * kMergeStride + col) = make_float2(o[n][0], o[n][1]);
-            *(float2*)(mo + (rA + 8) * kMergeStride + col) = make_float2(o[n][2], o[n][3]);
-        }
-        if ((lane & 3) == 0) {
-            merge_ml[(mt * kKW + kg) * 16 + rA] = make_float2(m_run[0], l_run[0]);
-            merge_ml[(mt * kKW + kg) * 16 + rA + 8] = make_float2(m_run[1], l_run[1]);
-        }
+    for (int h = 0; h < 2; ++h) {
+        l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 1);
+        l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 2);
     }
-    __syncthreads();
+    if ((lane & 3) == 0) { x_l[(mt * 16 + rg) * KW + kg] = l_run[0]; x_l[(mt * 16 + rg + 8) * KW + kg] = l_run[1]; }
+    __syncthreads();  // all row sums in place; every armed stage has been consumed: the ring is dead
 
     // With clusters, the KV splits of this (sequence, KV head) are the cluster's CTAs (rank = split): the split
     // results stay in shared memory and are merged across the cluster below instead of going through global memory.
     const bool in_cluster = p.cluster_size > 1;
-    float* cl_o = (float*)(ring + kMergeBytes);                       // [MT*16][kD]
-    float2* cl_ml = (float2*)(ring + kMergeBytes + MT * 16 * kD * 4);  // [MT*16]
-    // each thread finishes 4 consecutive columns of one row at a time
-    for (int idx = tid; idx < MT * 16 * (kD / 4); idx += kThreads) {
-        const int r = idx / (kD / 4);
-        const int c4 = (idx - r * (kD / 4)) * 4;
+    float* cl_o = (float*)ring;                              // [MT*16][kD]
+    float2* cl_ml = (float2*)(ring + MT * 16 * kD * 4);      // [MT*16]
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int r = mt * 16 + rg + 8 * h;                  // row of the CTA's chunk
         if (row0 + r >= rows) continue;
-        const int rm = r >> 4, rr = r & 15;
-        float m_all = -INFINITY;
-#pragma unroll
-        for (int k = 0; k < kKW; ++k) m_all = fmaxf(m_all, merge_ml[(rm * kKW + k) * 16 + rr].x);
         float l_all = 0.f;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int k = 0; k < kKW; ++k) {
-            const float2 ml = merge_ml[(rm * kKW + k) * 16 + rr];
-            const float w = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m_all);
-            l_all += ml.y * w;
-            const float4 v = *(const float4*)(merge_o + ((size_t)(rm * kKW + k) * 16 + rr) * kMergeStride + c4);
-            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+        for (int k4 = 0; k4 < KW; k4 += 4) {
+            const float4 v = *(const float4*)(x_l + r * KW + k4);
+            l_all += (v.x + v.y) + (v.z + v.w);
         }
+        const float m_all = m_run[h];
         const int i = (row0 + r) / G, hg = (row0 + r) - i * G;
-        const int h = g * G + hg;
+        const int hd = g * G + hg;
+        const bool first = kg == 0 && (lane & 3) == 0;       // one lane per row writes the row's (m, l)
         if (sp.nsplit == 1) {
             const float inv = 1.f / l_all;
-            const long long off = ((long long)(sp.q_row0 + i) * p.hq + h) * kD + c4;
-            uint2 packed;
-            packed.x = pack_bf16(acc.x * inv, acc.y * inv);
-            packed.y = pack_bf16(acc.z * inv, acc.w * inv);
-            *(uint2*)((__nv_bfloat16*)p.out + off) = packed;
-            if (p.lse && c4 == 0) p.lse[(long long)(sp.q_row0 + i) * p.hq + h] = (m_all + log2f(l_all)) * 0.6931471805599453f;
-        } else if (in_cluster) {
-            *(float4*)(cl_o + r * kD + c4) = acc;
-            if (c4 == 0) cl_ml[r] = make_float2(m_all, l_all);
+            __nv_bfloat16* orow = (__nv_bfloat16*)p.out + ((long long)(sp.q_row0 + i) * p.hq + hd) * kD;
+#pragma unroll
+            for (int n = 0; n < 2 * kCG; ++n)
+                *(uint32_t*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)) = pack_bf16(o[n][2 * h] * inv, o[n][2 * h + 1] * inv);
+            if (p.lse && first) p.lse[(long long)(sp.q_row0 + i) * p.hq + hd] = (m_all + log2f(l_all)) * 0.6931471805599453f;
         } else {
-            const long long e = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit + split;
-            *(float4*)(p.part_o + e * kD + c4) = acc;
-            if (c4 == 0) p.part_ml[e] = make_float2(m_all, l_all);
+            float* orow;
+            if (in_cluster) {
+                orow = cl_o + r * kD;
+                if (first) cl_ml[r] = make_float2(m_all, l_all);
+            } else {
+                const long long e = (long long)sp.part_base + ((long long)i * p.hq + hd) * sp.nsplit + split;
+                orow = p.part_o + e * kD;
+                if (first) p.part_ml[e] = make_float2(m_all, l_all);
+            }
+#pragma unroll
+            for (int n = 0; n < 2 * kCG; ++n)
+                *(float2*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)) = make_float2(o[n][2 * h], o[n][2 * h + 1]);
         }
     }
     if (in_cluster && sp.nsplit > 1) {   // (uniform over the cluster: all its CTAs belong to one sequence)
@@ -633,10 +661,11 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
 namespace {
 template <int MT, int KW, int NS>
 constexpr int small_smem_bytes() {
-    constexpr int kMergeBytes = MT * KW * 16 * (kMergeStride * 4 + 8) + MT * 16 * (kD * 4 + 8);   // + the cluster rows
+    constexpr int kClusterBytes = MT * 16 * (kD * 4 + 8);
     constexpr int kRing = NS * 2 * KW * kPage * kRowBytes;
-    // [ring | merge region][Q tile][2 * NS barriers + abort flag] + slack for the 1024-byte alignment
-    return (kRing > kMergeBytes ? kRing : kMergeBytes) + MT * 16 * kRowBytes + 2 * NS * 8 + 16 + 1024;
+    constexpr int kExchange = 2 * MT * 16 * KW * 4 + MT * KW * 32 * 16;
+    // [ring | cluster rows][Q tile][2 * NS barriers + abort flag][exchange area] + slack for the 1024-byte alignment
+    return (kRing > kClusterBytes ? kRing : kClusterBytes) + MT * 16 * kRowBytes + 2 * NS * 8 + 16 + kExchange + 1024;
 }
 
 template <int MT, int KW, int NS>
