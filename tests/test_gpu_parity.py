@@ -155,6 +155,14 @@ def test_small_q_split_merge_in_clusters_and_by_combine_kernel(P, q, hq, hkv, ba
         assert b.launches == 2
 
 
+@pytest.mark.parametrize("P,q,hq,hkv", [(0, 1, 32, 8), (17, 4, 32, 8), (1000, 3, 24, 8), (2049, 5, 32, 8), (4096, 8, 32, 8), (300, 16, 4, 4)])
+def test_small_q_kernel_with_four_kv_groups(P, q, hq, hkv, monkeypatch):
+    """AGX_SMALL_KW=4: four pages per pipeline stage, each warp owning two 16-column groups of O."""
+    monkeypatch.setenv("AGX_SMALL_KW", "4")
+    w = W.make_attn_workload(f"kw4_{P}_{q}", 900 + P + q, "bf16", hq, hkv, 128, [P], [q], spare_pages=2)
+    run_and_check(w, poison=True)
+
+
 def test_small_q_ragged_batch_with_shared_prefix():
     P = [2048, 2100, 4000, 2048 + 15, 9000, 2500, 3001, 2048]
     q = [1, 2, 4, 8, 16, 3, 5, 8]
