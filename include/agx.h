@@ -136,7 +136,9 @@ AGX_API int64_t agx_attn_workspace_bytes(agx_handle* handle, int32_t B, const in
  * shorter than 12288 tokens run the split-KV warp-MMA kernel (latency-bound); up to 32 rows over a
  * longer context, or 33..128 rows over any context, run the tensor-core kernel with one padded Q tile
  * whose KV tiles alternate between two softmax warpgroups (HBM-bound); longer blocks run the
- * tensor-core kernel with 256-row tiles (tensor-bound).  Sequences of all kinds may share a batch.
+ * tensor-core kernel with 256-row tiles (tensor-bound).  Sequences of all kinds may share a batch; two or
+ * more blocks of at most 32 rows whose contexts add up to 24576 tokens or more (at 8 KV heads) all take the
+ * padded-tile kernel, whatever their single lengths.
  * Errors: AGX_E_INVAL (null/misaligned, q_len < 1, prefix_len < 0, workspace too small),
  * AGX_E_RANGE ((P + q) exceeds 16 * page_table_stride), AGX_E_CUDA.  Page ids outside
  * [0, num_pages) set AGX_DEV_BAD_PAGE and read as zeros.

@@ -21,7 +21,8 @@ struct agx_handle {
     int small_min_split;    // tokens; tuning knob (env AGX_SMALL_MIN_SPLIT)
     int force_mma_sync;     // route large q through the mma.sync kernel (env AGX_FORCE_MMA_SYNC)
     int debug_plan;         // print launch plans to stderr (env AGX_DEBUG_PLAN)
-    int small_kw;           // pages per pipeline stage of the warp-MMA kernel, 4 or 8 (env AGX_SMALL_KW)
+    int small_kw;           // pages per pipeline stage of the warp-MMA kernel: 4, 8, or 0 = chosen per batch (env AGX_SMALL_KW)
+    int batch_stream_tokens; // total tokens of a batch's small blocks from which they all take the stream schedule (env AGX_BATCH_STREAM_TOKENS)
     bool cluster_merge;     // KV splits of the small-q kernel merged inside thread-block clusters where the batch allows (env AGX_CLUSTER_MERGE=0 turns it off)
     int zero_copy;          // host steps: bit 0 = kernels read small pinned inputs, bit 1 = kernels write `out` into a pinned buffer (env AGX_ZERO_COPY, default 3)
     int stream_min_tokens;  // context length from which blocks of <= 32 rows take the tensor-core stream schedule (env AGX_STREAM_MIN_TOKENS)
@@ -57,6 +58,7 @@ struct Launch {
     Kind kind;
     int total_rows;  // sum of q_len over the launch's sequences
     int num_items;
+    int kw;          // small-q kernel: pages per pipeline stage (KV groups), 4 or 8
     int cluster;     // > 1: CTAs per cluster = KV splits of every sequence of the launch, merged in-kernel (no partials)
     std::vector<SeqPlan> seqs;
 };
@@ -80,6 +82,20 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
         if ((long long)row0[s] + Q[s] > (1 << 30)) return fail(h, AGX_E_RANGE, "too many rows");
         row0[s + 1] = row0[s] + Q[s];
     }
+    // Blocks of at most 32 rows: measured on B200 (GQA 32/8, equal sequences), what decides is the batch's total
+    // context, not each sequence's: from ~24k tokens in all (two sequences or more) the tensor-core stream schedule
+    // wins whatever the single lengths; below that the warp-MMA kernel, with 4-page stages and two CTAs per SM from
+    // ~8k tokens in all, with 8-page stages (one 16-warp CTA per SM) for less.  A single sequence keeps its own
+    // cross-over (stream_min_tokens).
+    long long small_tokens = 0;
+    int small_seqs = 0;
+    if (c.dtype != AGX_F32)
+        for (int s = 0; s < B; ++s)
+            if (Q[s] * G <= 32) { small_tokens += P[s] + Q[s]; ++small_seqs; }
+    small_tokens = small_tokens * c.num_kv_heads / 8;   // the thresholds were measured with 8 KV heads: scale to the same bytes
+    const bool batch_streams = small_seqs >= 2 && small_tokens >= h->batch_stream_tokens;
+    long long warp_mma_tokens = 0;
+    int warp_mma_seqs = 0;
     std::vector<int> groups[KIND_COUNT];
     for (int s = 0; s < B; ++s) {
         Kind k;
@@ -90,14 +106,16 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
             // up to 128 rows: one Q tile per CTA, KV tiles alternating between two softmax warpgroups (HBM-bound
             // streaming on the tcgen05 pipe); blocks of at most 32 rows over short contexts stay with the warp-MMA
             // kernel, whose start-up is shorter (measured cross-over: 8k-16k tokens at 32 rows, none above 32 rows)
-            if (tile_ok && rows <= 128 && (rows > 32 || P[s] + Q[s] >= h->stream_min_tokens)) k = KIND_STREAM;
+            if (tile_ok && rows <= 128 && (rows > 32 || batch_streams || P[s] + Q[s] >= h->stream_min_tokens)) k = KIND_STREAM;
             else if (rows <= 16) k = KIND_SMALL1;
             else if (rows <= 32) k = KIND_SMALL2;
             else if (rows <= kSmallRowsMax || h->force_mma_sync || !attn_tile_available()) k = KIND_SMALL4;
             else k = KIND_TILE;
+            if (k == KIND_SMALL1 || k == KIND_SMALL2) { warp_mma_tokens += P[s] + Q[s]; ++warp_mma_seqs; }
         }
         groups[k].push_back(s);
     }
+    const int small_kw = h->small_kw ? h->small_kw : (warp_mma_seqs >= 2 && warp_mma_tokens * c.num_kv_heads / 8 >= 8192) ? 4 : 8;
     for (int k = 0; k < KIND_COUNT; ++k) {
         const std::vector<int>& seqs = groups[k];
         if (seqs.empty()) continue;
@@ -107,7 +125,7 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
         std::vector<long long> per_seq_items(seqs.size());
         if (k == KIND_SIMT) { unit = 64; min_split = 256; target = h->sm_count * 16; }
         else if (k == KIND_TILE || k == KIND_STREAM) { unit = 128; min_split = k == KIND_TILE ? 512 : 256; target = h->sm_count; }
-        else { unit = 64; min_split = h->small_min_split; target = h->sm_count * ((k == KIND_SMALL4 || h->small_kw == 8) ? 1 : 2); }
+        else { unit = 64; min_split = h->small_min_split; target = h->sm_count * ((k == KIND_SMALL4 || small_kw == 8) ? 1 : 2); }
         const int rows_per_chunk = (k == KIND_SMALL1) ? 16 : (k == KIND_SMALL2) ? 32 : (k == KIND_SMALL4) ? 64 : (k == KIND_STREAM) ? 128 : 256;
         long long work = 0;
         for (size_t n = 0; n < seqs.size(); ++n) {
@@ -163,7 +181,7 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
             }
             if (ok && common >= 2 && common <= 16) {
                 const int mt = k == KIND_SMALL1 ? 1 : k == KIND_SMALL2 ? 2 : 4;
-                const int fit = attn_small_max_clusters(mt, mt == 4 ? 4 : h->small_kw, common);
+                const int fit = attn_small_max_clusters(mt, mt == 4 ? 4 : small_kw, common);
                 if (fit >= base_items) cluster = common;
                 if (h->debug_plan) fprintf(stderr, "agx plan: clusters of %d: %d fit the device, %lld needed\n", common, fit, base_items);
             }
@@ -175,6 +193,7 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
             ln.total_rows = 0;
             ln.num_items = 0;
             ln.cluster = cluster;
+            ln.kw = (k == KIND_SMALL4) ? 4 : small_kw;
             for (size_t n = a; n < std::min(seqs.size(), a + kMaxSeqs); ++n) {
                 const int s = seqs[n];
                 const int L = P[s] + Q[s];
@@ -204,8 +223,8 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
                 ln.seqs.push_back(sp);
             }
             if (h->debug_plan && k != KIND_TILE && k != KIND_STREAM)
-                fprintf(stderr, "agx plan: kind %d, %zu sequences, %d CTAs, first sequence %d splits of %d tokens%s\n", k,
-                        ln.seqs.size(), ln.num_items, ln.seqs[0].nsplit, ln.seqs[0].split_tokens,
+                fprintf(stderr, "agx plan: kind %d (stages of %d pages), %zu sequences, %d CTAs, first sequence %d splits of %d tokens%s\n", k,
+                        ln.kw, ln.seqs.size(), ln.num_items, ln.seqs[0].nsplit, ln.seqs[0].split_tokens,
                         cluster ? ", merged in clusters" : "");
             plan.launches.push_back(std::move(ln));
         }
@@ -260,7 +279,9 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     env = getenv("AGX_ZERO_COPY");
     h->zero_copy = env ? atoi(env) : 3;
     env = getenv("AGX_SMALL_KW");
-    h->small_kw = (env && atoi(env) == 4) ? 4 : 8;
+    h->small_kw = (env && (atoi(env) == 4 || atoi(env) == 8)) ? atoi(env) : 0;
+    env = getenv("AGX_BATCH_STREAM_TOKENS");   // (forcing the per-sequence cross-over also switches the batch rule off)
+    h->batch_stream_tokens = env ? atoi(env) : getenv("AGX_STREAM_MIN_TOKENS") ? 0x7FFFFFFF : 24576;
     env = getenv("AGX_DEBUG_PLAN");
     h->debug_plan = env ? atoi(env) : 0;
     cudaError_t e = cudaGetDevice(&h->device);
@@ -377,8 +398,8 @@ static agx_status attn_impl(agx_handle* h, const void* q_block, const void* k_ne
             }
         }
         switch (ln.kind) {
-            case KIND_SMALL1: e = launch_attn_small_bf16(p, 1, h->small_kw, stream); break;
-            case KIND_SMALL2: e = launch_attn_small_bf16(p, 2, h->small_kw, stream); break;
+            case KIND_SMALL1: e = launch_attn_small_bf16(p, 1, ln.kw, stream); break;
+            case KIND_SMALL2: e = launch_attn_small_bf16(p, 2, ln.kw, stream); break;
             case KIND_SMALL4: e = launch_attn_small_bf16(p, 4, 4, stream); break;
             case KIND_SIMT: e = launch_attn_simt_f32(p, stream); break;
             case KIND_TILE: e = launch_attn_tile_bf16(p, false, stream); break;

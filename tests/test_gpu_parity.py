@@ -163,6 +163,17 @@ def test_small_q_kernel_with_four_kv_groups(P, q, hq, hkv, monkeypatch):
     run_and_check(w, poison=True)
 
 
+@pytest.mark.parametrize("P,q", [
+    ([2100, 2048, 2300, 1990], [8, 8, 1, 5]),          # > 8k tokens in all: warp-MMA kernel with 4-page stages
+    ([9000, 8200, 8192, 7000], [4, 8, 8, 1]),          # > 24k tokens in all: every block on the stream schedule
+    ([3000, 100], [8, 8]), ([5000, 4000, 17], [1, 1, 1]),
+])
+def test_batches_dispatched_by_their_total_context(P, q):
+    w = W.make_attn_workload(f"batch_{sum(P)}", 4000 + sum(P), "bf16", 32, 8, 128, P, q, spare_pages=2)
+    run_and_check(w, sample=(9, 20), poison=True)
+    run_and_check(w, sample=(9, 20), fused=True)
+
+
 def test_small_q_ragged_batch_with_shared_prefix():
     P = [2048, 2100, 4000, 2048 + 15, 9000, 2500, 3001, 2048]
     q = [1, 2, 4, 8, 16, 3, 5, 8]
