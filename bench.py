@@ -304,6 +304,20 @@ def extra_workloads(torch, agx, W, peaks, steps, warmup):
         torch.cuda.empty_cache()
     except Exception as e:  # keep the headline line alive
         out["c5_long_context_verify"] = {"error": repr(e)}
+    # batched verify (serving-style; the paper's own setting is batch 1): 16 x (P = 8192, q = 8), 537 MB of KV per call
+    try:
+        lv = LayeredVerify(torch, agx, W, [8192] * 16, [8] * 16, 32, 8, 128, 1, 0, 6)
+        g = capture(torch, lambda: lv.step(attn_only=True))
+        ms = time_graph(torch, g, max(steps // 10, 20), max(warmup, 3))
+        by = lv.bytes_per_layer()
+        out["batched_verify_16x8192"] = {
+            "ms": ms, "query_tok_per_s": 128 / (ms * 1e-3),
+            "roofline": {"bound": "hbm", "achieved": by / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "peak_source": peaks["source"]}}
+        del lv, g
+        torch.cuda.empty_cache()
+    except Exception as e:
+        out["batched_verify_16x8192"] = {"error": repr(e)}
     # accept step alone: one read of the logits; 64 distinct buffers rotated inside one graph so they come from HBM
     try:
         acc = {}
