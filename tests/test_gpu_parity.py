@@ -174,6 +174,26 @@ def test_batches_dispatched_by_their_total_context(P, q):
     run_and_check(w, sample=(9, 20), fused=True)
 
 
+@pytest.mark.parametrize("fused", [False, True])
+def test_more_sequences_than_one_launch_holds(fused):
+    """70 sequences (a launch holds 48): several launches per kernel kind, contexts from empty to a few pages, one long."""
+    rng = np.random.default_rng(123)
+    P = rng.integers(0, 300, 70).tolist(); P[5] = 0; P[17] = 5000; P[40] = 2049
+    q = rng.integers(1, 9, 70).tolist(); q[17] = 3; q[33] = 40       # one block of 160 rows rides along
+    w = W.make_attn_workload("many_seqs", 321, "bf16", 32, 8, 128, P, q, spare_pages=1)
+    run_and_check(w, poison=not fused, fused=fused)
+
+
+@pytest.mark.parametrize("hq,hkv", [(16, 2), (16, 16), (8, 1), (40, 8)])
+def test_other_head_layouts(hq, hkv):
+    G = hq // hkv
+    P = [1000, 37, 4100, 0]
+    q = [max(1, 32 // G), 1, max(1, 16 // G), 2]
+    w = W.make_attn_workload(f"heads_{hq}_{hkv}", 55 + hq, "bf16", hq, hkv, 128, P, q, spare_pages=1)
+    run_and_check(w, poison=True)
+    run_and_check(w, fused=True)
+
+
 def test_small_q_ragged_batch_with_shared_prefix():
     P = [2048, 2100, 4000, 2048 + 15, 9000, 2500, 3001, 2048]
     q = [1, 2, 4, 8, 16, 3, 5, 8]
