@@ -420,7 +420,8 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
             }
 #pragma unroll
             for (int n = 0; n < 2 * kCG; ++n)
-                *(float2*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)) = make_float2(o[n][2 * h], o[n][2 * h + 1]);
+                if (in_cluster) *(float2*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)) = make_float2(o[n][2 * h], o[n][2 * h + 1]);
+                else __stcg((float2*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)), make_float2(o[n][2 * h], o[n][2 * h + 1]));   // read next by other SMs
         }
     }
     if (in_cluster && sp.nsplit > 1) {   // (uniform over the cluster: all its CTAs belong to one sequence)
@@ -572,15 +573,15 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
     if (ns <= 32) {
         // One round trip to memory: lane k fetches (m, l) of split k while every lane already fetches its
         // columns of every split's O row; the weights then travel by shuffle, splits in index order.
-        const float2 ml = (lane < ns) ? p.part_ml[e0 + lane] : make_float2(-INFINITY, 0.f);
+        const float2 ml = (lane < ns) ? __ldcg(p.part_ml + e0 + lane) : make_float2(-INFINITY, 0.f);
         float4 v[16], v2[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j)
-            if (j < ns && c4 < D) v[j] = *(const float4*)(p.part_o + (e0 + j) * D + c4);
+            if (j < ns && c4 < D) v[j] = __ldcg((const float4*)(p.part_o + (e0 + j) * D + c4));   // written by other SMs just before: past the L1
         if (ns > 16) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-                if (16 + j < ns && c4 < D) v2[j] = *(const float4*)(p.part_o + (e0 + 16 + j) * D + c4);
+                if (16 + j < ns && c4 < D) v2[j] = __ldcg((const float4*)(p.part_o + (e0 + 16 + j) * D + c4));
         }
         m_all = ml.x;
 #pragma unroll
