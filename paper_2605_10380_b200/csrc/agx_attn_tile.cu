@@ -195,6 +195,7 @@ struct EpiCtx {
     float* part_o;
     float2* part_ml;
     float* lse;
+    unsigned long long magic;   // (row * magic) >> 32 == row / G exactly for rows < 2^22
 };
 template <bool kStreams>
 __device__ __forceinline__ TileItem locate_item(const AttnParams& p, int block) {
@@ -263,21 +264,39 @@ __device__ __noinline__ void tile_epilogue(unsigned char* smem, uint32_t tO, flo
     if (!warp_has_rows) return;
     unsigned char* stage = smem + kOffK + (warp - 4) * 16384;    // [32 rows][512 B], 16-byte units XOR-swizzled by row
     const int r_warp0 = it.row0 + (warp - 4) * 32;               // first row of this warp
-    const uint64_t magic = (0x100000000ull + it.G - 1) / it.G;   // (row * magic) >> 32 == row / G exactly for rows < 2^22
+    const uint64_t magic = cx.magic;                             // (row * magic) >> 32 == row / G exactly for rows < 2^22
     const bool single = it.nsplit == 1;
     const float inv = (l_run > 0.f) ? 1.f / l_run : 0.f;
+    // per-row scalars, and the row's destination: lane j works them out for row j once, the copy loop below fetches
+    // them by shuffle (a single warp doing the index arithmetic row by row took longer than the copies themselves)
+    unsigned long long row_dst = 0;
+    {
+        const int r = r_warp0 + lane;
+        if (r < it.rows) {
+            const int i = (int)(((uint64_t)(uint32_t)r * magic) >> 32), h = it.g * it.G + (r - i * it.G);
+            if (single) {
+                if (cx.lse) cx.lse[(long long)(it.q_row0 + i) * cx.hq + h] = (m_ref + log2f(l_run)) * 0.6931471805599453f;
+                row_dst = (unsigned long long)((unsigned char*)cx.out + ((long long)(it.q_row0 + i) * cx.hq + h) * 256);
+            } else {
+                const long long e = (long long)cx.part_base + ((long long)i * cx.hq + h) * it.nsplit + it.split;
+                cx.part_ml[e] = make_float2(m_ref, l_run);
+                row_dst = (unsigned long long)(cx.part_o + e * kD);
+            }
+        }
+    }
     tc_fence_after();
     {
-        uint32_t oreg[32];
+        uint32_t oreg[64];   // two 32-column chunks per TMEM round trip
 #pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) {
-            tmem_ld_x32(tO + c4 * 32, oreg);
+        for (int c8 = 0; c8 < 4; c8 += 2) {
+            tmem_ld_x32(tO + c8 * 32, oreg);
+            tmem_ld_x32(tO + c8 * 32 + 32, oreg + 32);
             tmem_wait_ld();
             if (kStreams) {
                 const unsigned char* park = smem + kOffPark + ((((warp & 3) << 5) + lane) * 512);
 #pragma unroll
-                for (int v = 0; v < 8; ++v) {
-                    const float4 o1 = *(const float4*)(park + (((c4 * 8 + v) ^ lane) << 4));
+                for (int v = 0; v < 16; ++v) {
+                    const float4 o1 = *(const float4*)(park + (((c8 * 8 + v) ^ lane) << 4));
                     oreg[4 * v + 0] = __float_as_uint(__uint_as_float(oreg[4 * v + 0]) * w_own + (w_other != 0.f ? o1.x * w_other : 0.f));
                     oreg[4 * v + 1] = __float_as_uint(__uint_as_float(oreg[4 * v + 1]) * w_own + (w_other != 0.f ? o1.y * w_other : 0.f));
                     oreg[4 * v + 2] = __float_as_uint(__uint_as_float(oreg[4 * v + 2]) * w_own + (w_other != 0.f ? o1.z * w_other : 0.f));
@@ -286,24 +305,33 @@ __device__ __noinline__ void tile_epilogue(unsigned char* smem, uint32_t tO, flo
             }
             if (single) {
 #pragma unroll
-                for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * inv);
+                for (int c = 0; c < 64; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * inv);
             }
+            if (kStreams) {
+                // one warp with at most 32 rows: each lane stores its own row straight from registers (16 KB in all;
+                // staging it through shared memory for whole-row stores took a single warp longer than these do)
+                if (row_dst) {
 #pragma unroll
-            for (int v = 0; v < 8; ++v)
-                *(uint4*)(stage + lane * 512 + (((c4 * 8 + v) ^ lane) << 4)) = make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
-        }
-    }
-    {   // per-row scalars
-        const int r = r_warp0 + lane;
-        if (r < it.rows) {
-            const int i = (int)(((uint64_t)(uint32_t)r * magic) >> 32), h = it.g * it.G + (r - i * it.G);
-            if (single) {
-                if (cx.lse) cx.lse[(long long)(it.q_row0 + i) * cx.hq + h] = (m_ref + log2f(l_run)) * 0.6931471805599453f;
+                    for (int v = 0; v < 16; ++v) {
+                        if (single) {
+                            uint2 pk;
+                            pk.x = pack_bf16(__uint_as_float(oreg[4 * v]), __uint_as_float(oreg[4 * v + 1]));
+                            pk.y = pack_bf16(__uint_as_float(oreg[4 * v + 2]), __uint_as_float(oreg[4 * v + 3]));
+                            *(uint2*)((unsigned char*)row_dst + (c8 * 8 + v) * 8) = pk;
+                        } else {
+                            __stcg((uint4*)((unsigned char*)row_dst + (c8 * 8 + v) * 16),
+                                   make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]));
+                        }
+                    }
+                }
             } else {
-                cx.part_ml[(long long)cx.part_base + ((long long)i * cx.hq + h) * it.nsplit + it.split] = make_float2(m_ref, l_run);
+#pragma unroll
+                for (int v = 0; v < 16; ++v)
+                    *(uint4*)(stage + lane * 512 + (((c8 * 8 + v) ^ lane) << 4)) = make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
             }
         }
     }
+    if (kStreams) return;
     __syncwarp();
     // a warp writes one row per instruction: lane j moves 16-byte unit j (fp32) or converts it to 8 bytes of bf16;
     // eight rows' loads are in flight before the first store
@@ -318,17 +346,16 @@ __device__ __noinline__ void tile_epilogue(unsigned char* smem, uint32_t tO, flo
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const int rl = rl0 + u;
-            if (rl >= n_valid) break;
-            const int ro = r_warp0 + rl;
-            const int io = (int)(((uint64_t)(uint32_t)ro * magic) >> 32), ho = it.g * it.G + (ro - io * it.G);
-            if (single) {
-                uint2 pk;
-                pk.x = pack_bf16(__uint_as_float(v[u].x), __uint_as_float(v[u].y));
-                pk.y = pack_bf16(__uint_as_float(v[u].z), __uint_as_float(v[u].w));
-                *(uint2*)((unsigned char*)cx.out + (((long long)(it.q_row0 + io) * cx.hq + ho) * 256 + lane * 8)) = pk;
-            } else {
-                const long long e = (long long)cx.part_base + ((long long)io * cx.hq + ho) * it.nsplit + it.split;
-                *(uint4*)((unsigned char*)(cx.part_o + e * kD) + lane * 16) = v[u];
+            const unsigned long long dst = __shfl_sync(0xFFFFFFFFu, row_dst, rl & 31);
+            if (rl < n_valid) {
+                if (single) {
+                    uint2 pk;
+                    pk.x = pack_bf16(__uint_as_float(v[u].x), __uint_as_float(v[u].y));
+                    pk.y = pack_bf16(__uint_as_float(v[u].z), __uint_as_float(v[u].w));
+                    *(uint2*)((unsigned char*)dst + lane * 8) = pk;
+                } else {
+                    __stcg((uint4*)((unsigned char*)dst + lane * 16), v[u]);   // read next by other SMs
+                }
             }
         }
     }
@@ -603,6 +630,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         cx->it = locate_item<kStreams>(p, blockIdx.x);
         cx->part_base = sp.part_base; cx->hq = p.hq;
         cx->out = p.out; cx->part_o = p.part_o; cx->part_ml = p.part_ml; cx->lse = p.lse;
+        cx->magic = (0x100000000ull + (unsigned)G - 1) / (unsigned)G;   // a 64-bit division: done here, off the epilogue's path
     }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsHigh));
