@@ -133,7 +133,7 @@ AGX_API int64_t agx_attn_workspace_bytes(agx_handle* handle, int32_t B, const in
  *   workspace    : device, >= agx_attn_workspace_bytes(...) bytes, 256-byte aligned (may be NULL
  *                  when that figure is 0)
  * Dispatch (G = num_q_heads / num_kv_heads): up to 32 query rows per KV head (q_len * G) over a context
- * shorter than 12288 tokens run the split-KV warp-MMA kernel (latency-bound); up to 32 rows over a
+ * shorter than about 7k tokens (10k for q_len * G <= 8) run the split-KV warp-MMA kernel (latency-bound); up to 32 rows over a
  * longer context, or 33..128 rows over any context, run the tensor-core kernel with one padded Q tile
  * whose KV tiles alternate between two softmax warpgroups (HBM-bound); longer blocks run the
  * tensor-core kernel with 256-row tiles (tensor-bound).  Sequences of all kinds may share a batch; two or
