@@ -549,7 +549,7 @@ template <bool kBf16Out>
 __global__ void __launch_bounds__(128)
 attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
     pdl_launch_dependents();
-    pdl_wait();
+    // (everything up to the wait depends on the kernel arguments only and runs while the attention kernel drains)
     const int lane = threadIdx.x & 31;
     const int rh = blockIdx.x * 4 + (threadIdx.x >> 5);  // index over (local row, head) of the launch's sequences
     if (rh >= total_rows * p.hq) return;
@@ -570,6 +570,8 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
     const int c4 = lane * 4;               // each lane owns 4 output columns
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float m_all, l_all;
+    const float* o_src = p.part_o + e0 * D + c4;
+    pdl_wait();   // the partials are complete
     if (ns <= 32) {
         // One round trip to memory: lane k fetches (m, l) of split k while every lane already fetches its
         // columns of every split's O row; the weights then travel by shuffle, splits in index order.
@@ -577,11 +579,11 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
         float4 v[16], v2[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j)
-            if (j < ns && c4 < D) v[j] = __ldcg((const float4*)(p.part_o + (e0 + j) * D + c4));   // written by other SMs just before: past the L1
+            if (j < ns && c4 < D) v[j] = __ldcg((const float4*)(o_src + j * D));   // written by other SMs just before: past the L1
         if (ns > 16) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-                if (16 + j < ns && c4 < D) v2[j] = __ldcg((const float4*)(p.part_o + (e0 + 16 + j) * D + c4));
+                if (16 + j < ns && c4 < D) v2[j] = __ldcg((const float4*)(o_src + (16 + j) * D));
         }
         m_all = ml.x;
 #pragma unroll
