@@ -44,6 +44,8 @@ __device__ __forceinline__ void scan_vec(const uint4 v, unsigned int base, unsig
     }
 }
 
+constexpr int kFoldKeys = 2048;              // 16 KB of shared memory for the final fold
+
 template <bool kBf16, bool kVec>
 __global__ void __launch_bounds__(256)
 accept_kernel(const void* __restrict__ logits, long long row_stride, int vocab, int chunk_elems, int chunks,
@@ -125,16 +127,31 @@ accept_kernel(const void* __restrict__ logits, long long row_stride, int vocab, 
     if (!is_last) return;
     __threadfence();
 
-    // final fold: one thread per row
-    for (int r = threadIdx.x; r < total_q; r += 256) {
+    // final fold: one warp per row, the row's chunk keys spread over the lanes.  Up to kFoldKeys keys are first
+    // brought into shared memory by all threads at once (one memory round trip whatever the number of rows).
+    __shared__ unsigned long long keys[kFoldKeys];
+    const int n_keys = total_q * chunks;
+    const bool staged = n_keys <= kFoldKeys;
+    if (staged) {
+        for (int k = threadIdx.x; k < n_keys; k += 256) keys[k] = __ldcg(partials + k);
+        __syncthreads();
+    }
+    for (int r = threadIdx.x >> 5; r < total_q; r += 8) {
         unsigned long long b = 0ull;
-        for (int c = 0; c < chunks; ++c) {
-            const unsigned long long v = __ldcg(partials + (size_t)r * chunks + c);
+        for (int c = threadIdx.x & 31; c < chunks; c += 32) {
+            const unsigned long long v = staged ? keys[r * chunks + c] : __ldcg(partials + (size_t)r * chunks + c);
             b = v > b ? v : b;
         }
-        const int t = (int)(0xFFFFFFFFu - (unsigned int)(b & 0xFFFFFFFFull));
-        tokens[r] = t;
-        if (argmax) argmax[r] = t;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, b, off);
+            b = o > b ? o : b;
+        }
+        if ((threadIdx.x & 31) == 0) {
+            const int t = (int)(0xFFFFFFFFu - (unsigned int)(b & 0xFFFFFFFFull));
+            tokens[r] = t;
+            if (argmax) argmax[r] = t;
+        }
     }
     __syncthreads();
     // draft comparison and commit: one thread per sequence
