@@ -39,7 +39,7 @@ WORKLOAD = ("decode verification (c2): batch 1, cached context 4096, q=8, GQA 32
             "page 16 shuffled, 32 per-layer KV pools + accept on bf16 logits [8,128256]")
 # DRAM bytes of one attention call of this workload (attention kernel 16,957,696 + combine kernel 2,305,280), from the
 # ncu capture summarised under profiles/; set to None whenever one of the two kernels changes until it is re-captured
-NCU_TRAFFIC_BYTES = 16975616 + 2305536
+NCU_TRAFFIC_BYTES = 16975360 + 2436096
 
 
 # --------------------------------------------------------------------------- peaks / clocks
