@@ -154,16 +154,26 @@ accept_kernel(const void* __restrict__ logits, long long row_stride, int vocab, 
         }
     }
     __syncthreads();
-    // draft comparison and commit: one thread per sequence
-    for (int s = threadIdx.x; s < B; s += 256) {
+    // draft comparison and commit: one warp per sequence, 32 drafts compared at a time (the winners are read back
+    // past the L1: other warps of this block wrote them a moment ago)
+    for (int s = threadIdx.x >> 5; s < B; s += 8) {
+        const int lane = threadIdx.x & 31;
         const int r0 = cu_q[s];
         const int k = cu_q[s + 1] - r0 - 1;
         const int* dr = drafts + (r0 - s);
         int a = 0;
-        while (a < k && dr[a] == tokens[r0 + a]) ++a;
-        accept_len[s] = a;
-        next_token[s] = tokens[r0 + a];
-        if (seq_lens) seq_lens[s] = seq_lens[s] + a + 1;
+        while (a < k) {
+            const bool match = (a + lane < k) ? (dr[a + lane] == __ldcg(tokens + r0 + a + lane)) : false;
+            const unsigned int m = __ballot_sync(0xFFFFFFFFu, match);
+            const int run = (m == 0xFFFFFFFFu) ? 32 : __ffs(~m) - 1;   // leading matches of this group of 32
+            a += run;
+            if (run < 32) break;
+        }
+        if (lane == 0) {
+            accept_len[s] = a;
+            next_token[s] = __ldcg(tokens + r0 + a);
+            if (seq_lens) seq_lens[s] = seq_lens[s] + a + 1;
+        }
     }
 }
 
