@@ -545,9 +545,12 @@ attn_simt_f32_kernel(const __grid_constant__ AttnParams p) {
 // --------------------------------------------------------------------------------------------
 // Combine: out[row, h] = sum_k O_k 2^(m_k - m) / sum_k l_k 2^(m_k - m), splits in index order.
 // One warp per (row, head); lanes own 4 consecutive floats of each 128-wide chunk.
-template <bool kBf16Out>
-__global__ void __launch_bounds__(128)
+// kFew: no sequence of the launch has more than 4 splits (the prefill kernels): four O rows per warp instead of 32 keep
+// the register count low enough for 16 CTAs per SM, which is what the 19 MB of partials of a split prefill need.
+template <bool kBf16Out, bool kFew>
+__global__ void __launch_bounds__(128, kFew ? 10 : 3)
 attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
+    constexpr int kInFlight = kFew ? 4 : 16;
     pdl_launch_dependents();
     // (everything up to the wait depends on the kernel arguments only and runs while the attention kernel drains)
     const int lane = threadIdx.x & 31;
@@ -576,11 +579,11 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
         // One round trip to memory: lane k fetches (m, l) of split k while every lane already fetches its
         // columns of every split's O row; the weights then travel by shuffle, splits in index order.
         const float2 ml = (lane < ns) ? __ldcg(p.part_ml + e0 + lane) : make_float2(-INFINITY, 0.f);
-        float4 v[16], v2[16];
+        float4 v[kInFlight], v2[kFew ? 1 : 16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
+        for (int j = 0; j < kInFlight; ++j)
             if (j < ns && c4 < D) v[j] = __ldcg((const float4*)(o_src + j * D));   // written by other SMs just before: past the L1
-        if (ns > 16) {
+        if (!kFew && ns > 16) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
                 if (16 + j < ns && c4 < D) v2[j] = __ldcg((const float4*)(o_src + (16 + j) * D));
@@ -593,13 +596,13 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xFFFFFFFFu, l_all, off);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
+        for (int j = 0; j < kInFlight; ++j) {
             const float w = __shfl_sync(0xFFFFFFFFu, w_mine, j);
             if (j < ns && w != 0.f && c4 < D) {   // a split that saw no token for this row publishes only (m, l) = (-inf, 0)
                 acc.x += v[j].x * w; acc.y += v[j].y * w; acc.z += v[j].z * w; acc.w += v[j].w * w;
             }
         }
-        if (ns > 16) {
+        if (!kFew && ns > 16) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
                 const float w = __shfl_sync(0xFFFFFFFFu, w_mine, 16 + j);
@@ -755,8 +758,14 @@ cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, 
     const long long n = (long long)total_rows * p.hq;
     if (n == 0) return cudaSuccess;
     const int blocks = (int)((n + 3) / 4);
-    if (dtype == AGX_BF16) return launch_chained(attn_combine_kernel<true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
-    return launch_chained(attn_combine_kernel<false>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+    bool few = true;
+    for (int i = 0; i < p.num_seqs; ++i) few &= p.seq[i].nsplit <= 4;
+    if (dtype == AGX_BF16) {
+        if (few) return launch_chained(attn_combine_kernel<true, true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+        return launch_chained(attn_combine_kernel<true, false>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+    }
+    if (few) return launch_chained(attn_combine_kernel<false, true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+    return launch_chained(attn_combine_kernel<false, false>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
 }
 
 }  // namespace agx
