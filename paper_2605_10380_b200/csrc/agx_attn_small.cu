@@ -545,12 +545,13 @@ attn_simt_f32_kernel(const __grid_constant__ AttnParams p) {
 // --------------------------------------------------------------------------------------------
 // Combine: out[row, h] = sum_k O_k 2^(m_k - m) / sum_k l_k 2^(m_k - m), splits in index order.
 // One warp per (row, head); lanes own 4 consecutive floats of each 128-wide chunk.
-// kFew: no sequence of the launch has more than 4 splits (the prefill kernels): four O rows per warp instead of 32 keep
-// the register count low enough for 16 CTAs per SM, which is what the 19 MB of partials of a split prefill need.
-template <bool kBf16Out, bool kFew>
-__global__ void __launch_bounds__(128, kFew ? 10 : 3)
+// kMaxNs: no sequence of the launch has more splits than this (4, 16, or any number).  Four O rows per warp instead of 32
+// keep the register count low enough for ten CTAs per SM, which is what the 19 MB of partials of a split prefill need.
+template <bool kBf16Out, int kMaxNs>
+__global__ void __launch_bounds__(128, kMaxNs <= 4 ? 10 : kMaxNs <= 16 ? 5 : 3)
 attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
-    constexpr int kInFlight = kFew ? 4 : 16;
+    constexpr bool kFew = kMaxNs <= 16;          // no second batch of 16 rows
+    constexpr int kInFlight = kMaxNs <= 4 ? 4 : 16;
     pdl_launch_dependents();
     // (everything up to the wait depends on the kernel arguments only and runs while the attention kernel drains)
     const int lane = threadIdx.x & 31;
@@ -575,7 +576,7 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
     float m_all, l_all;
     const float* o_src = p.part_o + e0 * D + c4;
     pdl_wait();   // the partials are complete
-    if (ns <= 32) {
+    if (kMaxNs <= 32 || ns <= 32) {
         // One round trip to memory: lane k fetches (m, l) of split k while every lane already fetches its
         // columns of every split's O row; the weights then travel by shuffle, splits in index order.
         const float2 ml = (lane < ns) ? __ldcg(p.part_ml + e0 + lane) : make_float2(-INFINITY, 0.f);
@@ -758,14 +759,16 @@ cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, 
     const long long n = (long long)total_rows * p.hq;
     if (n == 0) return cudaSuccess;
     const int blocks = (int)((n + 3) / 4);
-    bool few = true;
-    for (int i = 0; i < p.num_seqs; ++i) few &= p.seq[i].nsplit <= 4;
+    int ns_max = 1;
+    for (int i = 0; i < p.num_seqs; ++i) ns_max = p.seq[i].nsplit > ns_max ? p.seq[i].nsplit : ns_max;
     if (dtype == AGX_BF16) {
-        if (few) return launch_chained(attn_combine_kernel<true, true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
-        return launch_chained(attn_combine_kernel<true, false>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+        if (ns_max <= 4) return launch_chained(attn_combine_kernel<true, 4>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+        if (ns_max <= 16) return launch_chained(attn_combine_kernel<true, 16>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+        return launch_chained(attn_combine_kernel<true, 1 << 30>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
     }
-    if (few) return launch_chained(attn_combine_kernel<false, true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
-    return launch_chained(attn_combine_kernel<false, false>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+    if (ns_max <= 4) return launch_chained(attn_combine_kernel<false, 4>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+    if (ns_max <= 16) return launch_chained(attn_combine_kernel<false, 16>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+    return launch_chained(attn_combine_kernel<false, 1 << 30>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
 }
 
 }  // namespace agx
