@@ -382,6 +382,7 @@ static agx_status attn_impl(agx_handle* h, const void* q_block, const void* k_ne
     p.pt_stride = pt_stride;
     p.hq = h->cfg.num_q_heads; p.hkv = h->cfg.num_kv_heads; p.head_dim = h->cfg.head_dim;
     p.scale_log2 = h->scale * 1.4426950408889634f;
+    p.row_div_magic = (0x100000000ull + (unsigned)(p.hq / p.hkv) - 1) / (unsigned)(p.hq / p.hkv);
     for (const Launch& ln : plan.launches) {
         p.num_seqs = (int)ln.seqs.size();
         p.num_items = ln.num_items;

@@ -70,7 +70,7 @@ constexpr int kPolyPairsOf8 = AGX_POLY_PAIRS;
 
 // barrier slots (8 bytes each)
 enum { BAR_K_FULL = 0, BAR_K_EMPTY = 3, BAR_V_FULL = 6, BAR_V_EMPTY = 9, BAR_S_FULL = 12, BAR_P_READY = 14,
-       BAR_O_FULL = 16, BAR_Q_FULL = 17, BAR_P_TAIL = 18, BAR_COUNT = 20 };
+       BAR_O_FULL = 16, BAR_Q_FULL = 17, BAR_P_TAIL = 18, BAR_CTX = 20, BAR_COUNT = 21 };
 // P is handed to the MMA warp in two parts: the first kPvHeadSteps k-steps (16 tokens each) as soon as they are
 // stored, so that their PV MMAs run while the softmax warpgroup still works on the last columns
 constexpr int kPvHeadSteps = 6;
@@ -229,6 +229,11 @@ __device__ __forceinline__ TileItem locate_item(const AttnParams& p, int block) 
 template <bool kStreams>
 __device__ __noinline__ void tile_epilogue(unsigned char* smem, uint32_t tO, float m_ref, float l_run, bool ok) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    {   // the context is written by another warp at kernel start: wait for its arrival (long complete, normally)
+        const uint32_t ctx_bar = smem_u32(smem) + kOffBar + 8u * BAR_CTX;
+        volatile int* abort_flag = (volatile int*)(smem + kOffBar + BAR_COUNT * 8);
+        if (!mbar_wait(ctx_bar, 0, abort_flag, nullptr)) ok = false;
+    }
     const EpiCtx cx = *(const EpiCtx*)(smem + kOffCtx);
     const TileItem& it = cx.it;
     const bool warp_has_rows = it.row0 + ((warp & 3) << 5) + (kStreams ? 0 : ((warp - 4) >> 2) * 128) < it.rows;
@@ -630,7 +635,8 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         cx->it = locate_item<kStreams>(p, blockIdx.x);
         cx->part_base = sp.part_base; cx->hq = p.hq;
         cx->out = p.out; cx->part_o = p.part_o; cx->part_ml = p.part_ml; cx->lse = p.lse;
-        cx->magic = (0x100000000ull + (unsigned)G - 1) / (unsigned)G;   // a 64-bit division: done here, off the epilogue's path
+        cx->magic = p.row_div_magic;
+        mbar_arrive(bar(BAR_CTX));   // (release) the epilogue waits on this before it reads the context
     }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsHigh));

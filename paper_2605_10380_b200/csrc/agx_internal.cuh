@@ -35,6 +35,7 @@ struct AttnParams {
     float* part_o;   // [entries][head_dim] fp32, un-normalised, relative to part_ml.x
     float2* part_ml; // [entries] (running max in log2 units, sum)
     int* status;
+    unsigned long long row_div_magic;   // ceil(2^32 / G), G = hq / hkv: (row * magic) >> 32 == row / G for rows < 2^22
     int cluster_size;    // > 1: the launch's CTAs form clusters of this size = the KV splits of one (sequence, KV head), merged in-kernel
     const void* k_new;   // fused append (agx_attn_prefixed_append): the block's K/V rows [total_q][hkv][d], or NULL
     const void* v_new;

@@ -45,7 +45,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitLimitCycles) {
                 *abort_flag = 1;
-                atomicOr(status, AGX_DEV_WAIT_TIMEOUT);
+                if (status) atomicOr(status, AGX_DEV_WAIT_TIMEOUT);
                 return false;
             }
         }

@@ -167,6 +167,7 @@ def test_small_q_kernel_with_four_kv_groups(P, q, hq, hkv, monkeypatch):
     ([2100, 2048, 2300, 1990], [8, 8, 1, 5]),          # > 8k tokens in all: warp-MMA kernel with 4-page stages
     ([9000, 8200, 8192, 7000], [4, 8, 8, 1]),          # > 24k tokens in all: every block on the stream schedule
     ([3000, 100], [8, 8]), ([5000, 4000, 17], [1, 1, 1]),
+    ([8192, 8192], [8, 8]),      # stream schedule whose last KV split is one short tile: its CTAs reach the epilogue at once
 ])
 def test_batches_dispatched_by_their_total_context(P, q):
     w = W.make_attn_workload(f"batch_{sum(P)}", 4000 + sum(P), "bf16", 32, 8, 128, P, q, spare_pages=2)
