@@ -195,6 +195,21 @@ def test_other_head_layouts(hq, hkv):
     run_and_check(w, fused=True)
 
 
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_random_batches_against_oracle(seed):
+    """Ten random batches per seed: 1-6 sequences, contexts from empty to ~20k tokens (skewed to short), verify-sized
+    blocks with an occasional long one; sampled rows against the oracle, fused and unfused."""
+    rng = np.random.default_rng(1000 + seed)
+    for case in range(10):
+        B = int(rng.integers(1, 7))
+        P = [int(x) for x in np.minimum(rng.exponential(3000, B).astype(np.int64) * int(rng.integers(1, 4)), 20000)]
+        q = [int(rng.integers(1, 17)) if rng.random() < 0.85 else int(rng.integers(17, 300)) for _ in range(B)]
+        if rng.random() < 0.3:
+            P[0] = int(rng.integers(0, 3)) * 4096      # page- and tile-aligned prefixes, empty ones
+        w = W.make_attn_workload(f"rand_{seed}_{case}", 9000 + 100 * seed + case, "bf16", 32, 8, 128, P, q, spare_pages=1)
+        run_and_check(w, sample=(case, 12), fused=bool(case & 1))
+
+
 def test_small_q_ragged_batch_with_shared_prefix():
     P = [2048, 2100, 4000, 2048 + 15, 9000, 2500, 3001, 2048]
     q = [1, 2, 4, 8, 16, 3, 5, 8]
