@@ -426,7 +426,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             const int r = row0 + rl;
             const bool valid = r < rows;
             const int rr = valid ? r : 0;
-            const int i = rr / G, hg = rr - i * G;
+            const int i = (int)(((uint64_t)(uint32_t)rr * p.row_div_magic) >> 32), hg = rr - i * G;   // rr / G without the division
             const unsigned char* src = (const unsigned char*)p.q + (((long long)(sp.q_row0 + i) * p.hq + g * G + hg) * 256 + ch * 16);
             const int tile = rl >> 7, rt = rl & 127, half = ch >> 3, u = ch & 7;
             cp_async_16(smem_base + kOffQ + tile * kTileBytes + half * kHalfBytes + rt * 128 + ((u ^ (rt & 7)) << 4), src, valid ? 16u : 0u);
