@@ -210,6 +210,33 @@ def test_random_batches_against_oracle(seed):
         run_and_check(w, sample=(case, 12), fused=bool(case & 1))
 
 
+def test_sixty_random_batches_fused_call_bit_identical_and_reproducible():
+    """Random head layouts, 1-8 sequences, contexts to 24k tokens, blocks from 1 to 700 rows, all in one process (kernel
+    kinds follow one another in every order): the fused call leaves the pools and the output bit-identical to append +
+    attention, twice over, with a clean status word."""
+    rng = np.random.default_rng(77)
+    heads = [(32, 8), (32, 8), (24, 8), (16, 2), (8, 8), (40, 8)]
+    for case in range(60):
+        hq, hkv = heads[int(rng.integers(0, len(heads)))]
+        B = int(rng.integers(1, 9))
+        scale = [300, 3000, 9000][int(rng.integers(0, 3))]
+        P = [int(min(x, 24000)) for x in rng.exponential(scale, B)]
+        if rng.random() < 0.3:
+            P[int(rng.integers(0, B))] = int(rng.integers(0, 6)) * 2048
+        q = []
+        for _ in range(B):
+            u = rng.random()
+            q.append(int(rng.integers(1, 17)) if u < 0.8 else int(rng.integers(17, 140)) if u < 0.95 else int(rng.integers(140, 700)))
+        w = W.make_attn_workload(f"rnd_{case}", 50000 + case, "bf16", hq, hkv, 128, P, q, spare_pages=1)
+        two = DeviceBatch(w); two.append(); two.attend()
+        one = DeviceBatch(w); one.attend_append()
+        again = DeviceBatch(w); again.attend_append()
+        assert one.status() == 0 and two.status() == 0 and again.status() == 0, (case, P, q)
+        assert torch.equal(one.k_pool, two.k_pool) and torch.equal(one.v_pool, two.v_pool), (case, P, q)
+        assert torch.equal(one.out, two.out) and torch.equal(one.out, again.out), (case, P, q)
+        assert bool(torch.isfinite(one.out.float()).all()), (case, P, q)
+
+
 def test_small_q_ragged_batch_with_shared_prefix():
     P = [2048, 2100, 4000, 2048 + 15, 9000, 2500, 3001, 2048]
     q = [1, 2, 4, 8, 16, 3, 5, 8]
