@@ -505,6 +505,30 @@ def test_verify_step_host_matches_oracle(enqueue_only, memory, monkeypatch):
     assert np.array_equal(h_acc.numpy(), al) and np.array_equal(h_nxt.numpy(), nt) and np.array_equal(h_sl.numpy(), sl)
 
 
+def test_verify_step_host_with_more_sequences_than_one_launch_holds():
+    """60 sequences through the host-buffer step: lengths travel by copy instead of kernel arguments, attention takes
+    several launches."""
+    rng = np.random.default_rng(5)
+    P = rng.integers(0, 400, 60).tolist(); q = rng.integers(1, 6, 60).tolist()
+    w = W.make_attn_workload("host_step_60", 79, "bf16", 32, 8, 128, P, q, spare_pages=1)
+    aw = W.make_planted_accept("host_step_60_accept", 80, "bf16", 4099, w.q_len, w.prefix_len)
+    b = DeviceBatch(w)
+    pin = lambda a, bf=False: (torch.from_numpy(np.ascontiguousarray(a)).view(torch.bfloat16) if bf else torch.from_numpy(np.ascontiguousarray(a))).pin_memory()
+    hq, hk, hv, hl, hd = pin(w.q_block, True), pin(w.k_new, True), pin(w.v_new, True), pin(aw.logits, True), pin(aw.drafts)
+    h_out = torch.zeros((w.total_q, 32, 128), dtype=torch.bfloat16).pin_memory()
+    h_acc, h_nxt, h_sl = (torch.full((60,), -7, dtype=torch.int32).pin_memory() for _ in range(3))
+    ws = torch.empty(b.h.verify_step_host_workspace_bytes(w.prefix_len, w.q_len, "bf16", aw.logits.shape[1], aw.vocab), dtype=torch.uint8, device="cuda")
+    b.h.verify_step_host(b.k_pool, b.v_pool, b.page_table, w.prefix_len, w.q_len, hq, hk, hv, hl, "bf16", aw.logits.shape[1], aw.vocab,
+                         hd, h_out, h_acc, h_nxt, h_sl, ws)
+    assert b.status() == 0
+    kp, vp = oracle_pools_after_append(w)
+    assert np.array_equal(host_storage(b.k_pool, "bf16"), kp) and np.array_equal(host_storage(b.v_pool, "bf16"), vp)
+    ref, _ = oracle.attn_paged_batch(w.q_block, kp, vp, w.page_table, "bf16", w.prefix_len, w.q_len, w.cu_q)
+    check_attention(h_out.to(torch.float64).numpy(), ref, "host step, 60 sequences")
+    am, al, nt, sl = oracle.accept_greedy(aw.logits, "bf16", aw.vocab, aw.drafts, aw.cu_q, aw.prefix_len)
+    assert np.array_equal(h_acc.numpy(), al) and np.array_equal(h_nxt.numpy(), nt) and np.array_equal(h_sl.numpy(), sl)
+
+
 # ------------------------------------------------------------------ n-gram draft table (Sec. 4.3)
 def _ngram_case(h, stream, n, contexts, k, fill):
     from oracle.toy_lm import build_ngram_table, ngram_drafts
