@@ -374,6 +374,50 @@ def extra_workloads(torch, agx, W, peaks, steps, warmup):
         out["multi_token_tax"] = tax
     except Exception as e:
         out["multi_token_tax"] = {"error": repr(e)}
+    # the steps around the hot path: n-gram draft table (Sec. 4.3) and prefix-reuse page traffic (Sec. 4.2)
+    try:
+        h = agx.Handle(32, 8, 128, "bf16")
+        rng = np.random.default_rng(17)
+        n_tok = 4096                                                   # a prompt-sized token stream over a 2k-token alphabet
+        toks = torch.from_numpy(rng.integers(0, 2048, n_tok).astype(np.int32)).cuda()
+        lut = torch.empty(agx.ngram_lut_bytes(n_tok), dtype=torch.uint8, device="cuda")
+        nws = torch.empty(agx.ngram_workspace_bytes(n_tok), dtype=torch.uint8, device="cuda")
+        g = capture(torch, lambda: h.ngram_build(toks, 3, lut, nws))
+        t_build = time_graph(torch, g, 200, 5)
+        ctx = toks[100:102].reshape(1, 2).contiguous()
+        fill = torch.zeros((1, 4), dtype=torch.int32, device="cuda")
+        dr = torch.zeros((1, 4), dtype=torch.int32, device="cuda"); hd = torch.zeros(1, dtype=torch.int32, device="cuda")
+        g2 = capture(torch, lambda: h.ngram_draft(lut, ctx, fill, 4, dr, hd))
+        t_draft = time_graph(torch, g2, 200, 5)
+        out["ngram_trigram_4096_tokens"] = {"build_us": t_build * 1e3, "draft_4_tokens_us": t_draft * 1e3,
+                                            "paper_build_ms_on_its_cpu": 83.0}
+        # copy of one cut page per sequence (16 sequences), and import of a 3072-token stored prefix from pinned host memory
+        pages, hkv, d = 4096, 8, 128
+        kp = torch.zeros((pages, hkv, 16, d), dtype=torch.bfloat16, device="cuda"); vp = torch.zeros_like(kp)
+        src = torch.arange(0, 16, dtype=torch.int32, device="cuda"); dst = torch.arange(100, 116, dtype=torch.int32, device="cuda")
+        g3 = capture(torch, lambda: h.kv_copy_pages(kp, vp, src, dst))
+        t_copy = time_graph(torch, g3, 200, 5)
+        n_imp = 3072 // 16
+        hk = torch.zeros((n_imp, hkv, 16, d), dtype=torch.bfloat16).pin_memory(); hv = torch.zeros_like(hk).pin_memory()
+        dst_imp = torch.arange(200, 200 + n_imp, dtype=torch.int32, device="cuda")
+        stg = torch.empty(h.kv_import_staging_bytes(n_imp), dtype=torch.uint8, device="cuda")
+        for _ in range(3):
+            h.kv_import_pages(kp, vp, hk, hv, dst_imp, stg)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            h.kv_import_pages(kp, vp, hk, hv, dst_imp, stg)
+        e1.record(); torch.cuda.synchronize()
+        t_imp = e0.elapsed_time(e1) / 20
+        imp_bytes = 2 * n_imp * hkv * 16 * d * 2
+        out["prefix_reuse_pages"] = {"copy_16_pages_us": t_copy * 1e3, "import_3072_tokens_us": t_imp * 1e3,
+                                     "import_GB/s": imp_bytes / (t_imp * 1e-3) / 1e9, "import_bytes": imp_bytes}
+        del kp, vp, g, g2, g3
+        torch.cuda.empty_cache()
+    except Exception as e:
+        out["ngram_trigram_4096_tokens"] = out.get("ngram_trigram_4096_tokens", {"error": repr(e)})
+        out["prefix_reuse_pages"] = out.get("prefix_reuse_pages", {"error": repr(e)})
     # prefix-cached prefill: P = 3072, q = 512, 24/8; tensor-bound.  4 layer pools are rotated.
     for name, P, q, hq in (("c3_prefix_prefill", 3072, 512, 24), ("c5_long_context_prefill", 30720, 2048, 32)):
         try:

@@ -386,9 +386,11 @@ AGX_API agx_status agx_kv_copy_pages(agx_handle* handle, void* k_pool, void* v_p
  * agx_kv_import_pages - bring precomputed KV pages from host memory into the pool.
  * Sec. 4.2 / Sec. 5.1: the KV caches of the static prefix and of the selected cluster combinations are computed
  * once, kept in storage and loaded when a request reuses them (the paper loads from SSD into unified
- * memory; here the stored pages sit in host memory and cross to the GPU).  Two host-to-device copies into
- * a staging area and one scatter kernel, all on `stream`: issued on a stream of its own, an import
- * overlaps attention that runs on other streams over pages already resident.
+ * memory; here the stored pages sit in host memory and cross to the GPU).  When h_k and h_v are pinned and
+ * mapped into the device's address space (cudaHostAlloc / cudaHostRegister), the scatter kernel reads the pages
+ * across the bus itself, one pass at bus speed; otherwise two host-to-device copies fill the staging area first.
+ * Everything runs on `stream`: issued on a stream of its own, an import overlaps attention that runs on other
+ * streams over pages already resident.
  *   h_k_pages, h_v_pages : HOST, [count][num_kv_heads][16][head_dim] of the handle's element type (pinned
  *                          memory makes the copies asynchronous)
  *   dst_pages            : device int32 [count]: pool page that receives imported page i; ids outside

@@ -760,11 +760,21 @@ agx_status agx_kv_import_pages(agx_handle* h, void* k_pool, void* v_pool, int64_
     if (staging_bytes < 2 * half) return fail(h, AGX_E_INVAL, "staging too small: %zu < %zu", staging_bytes, 2 * half);
     cudaStream_t stream = (cudaStream_t)stream_v;
     char* st = (char*)staging;
-    cudaError_t e = cudaMemcpyAsync(st, h_k, half, cudaMemcpyHostToDevice, stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(st + half, h_v, half, cudaMemcpyHostToDevice, stream);
-    if (e == cudaSuccess)
-        e = launch_scatter_pages(h->cfg.dtype, k_pool, v_pool, num_pages, st, st + half, dst_pages, count, h->cfg.num_kv_heads,
+    // Stored pages in pinned, device-mapped host memory are read across the bus by the scatter kernel itself (one pass,
+    // no staging); anything else is copied into the staging area first.
+    const void* mk = (h->zero_copy & 1) ? mapped_alias(h_k) : nullptr;
+    const void* mv = mk ? mapped_alias(h_v) : nullptr;
+    cudaError_t e = cudaSuccess;
+    if (mv) {
+        e = launch_scatter_pages(h->cfg.dtype, k_pool, v_pool, num_pages, mk, mv, dst_pages, count, h->cfg.num_kv_heads,
                                  h->cfg.head_dim, h->d_status, stream);
+    } else {
+        e = cudaMemcpyAsync(st, h_k, half, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(st + half, h_v, half, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess)
+            e = launch_scatter_pages(h->cfg.dtype, k_pool, v_pool, num_pages, st, st + half, dst_pages, count, h->cfg.num_kv_heads,
+                                     h->cfg.head_dim, h->d_status, stream);
+    }
     if (e != cudaSuccess) return cuda_fail(h, e, "page import");
     h->last_launches = 1;
     return AGX_OK;
