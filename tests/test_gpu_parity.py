@@ -433,10 +433,12 @@ def test_prefix_reuse_with_tail_cut_shares_full_pages_and_copies_the_cut_page():
     assert h.get_status() & agx.AGX_DEV_BAD_PAGE
 
 
-def test_import_of_stored_pages_from_host_memory_overlapping_attention_on_another_stream():
+@pytest.mark.parametrize("zero_copy", ["3", "0"], ids=["read_by_kernel", "staged_copies"])
+def test_import_of_stored_pages_from_host_memory_overlapping_attention_on_another_stream(zero_copy, monkeypatch):
     """Stored KV pages (Sec. 4.2) come from pinned host memory into scattered pool pages, bit for bit, on a stream
     of their own while attention over resident pages runs on another; a sequence then attends over the imported
     prefix."""
+    monkeypatch.setenv("AGX_ZERO_COPY", zero_copy)
     w = W.make_attn_workload("import", 91, "bf16", 32, 8, 128, [3072], [64], spare_pages=4)
     h = agx.Handle(32, 8, 128, "bf16")
     n_imp = 3072 // 16
