@@ -183,10 +183,10 @@ class LayeredVerify:
                                             self.page_table, self.P, self.Q, self.out[l], None, self.ws)
                 n += self.h.last_launch_count()
         if not attn_only and self.vocab:
-            self.seq_lens.copy_(self.prefix_dev)
+            # (the committed lengths simply keep advancing from replay to replay: their values feed nothing here)
             self.h.accept_greedy(self.logits, "bf16", self.vocab, self.drafts, self.cu_dev, self.acc, self.nxt, None,
                                  self.seq_lens, self.acc_ws)
-            n += self.h.last_launch_count() + 1  # + the device-to-device length reset (a torch copy kernel)
+            n += self.h.last_launch_count()
         return n
 
     def bytes_per_layer(self):
