@@ -10,6 +10,8 @@
 
 #include "agx_internal.cuh"
 
+namespace { struct Plan; }
+
 struct agx_handle {
     agx_config cfg;
     float scale;
@@ -27,6 +29,9 @@ struct agx_handle {
     int zero_copy;          // host steps: bit 0 = kernels read small pinned inputs, bit 1 = kernels write `out` into a pinned buffer (env AGX_ZERO_COPY, default 3)
     int stream_min_tokens;  // context length from which blocks of <= 32 rows take the tensor-core stream schedule (env AGX_STREAM_MIN_TOKENS; -1 = by block height)
     std::vector<int32_t> cu_host;  // staging for agx_verify_step_host (lives until its final sync)
+    // the launch plan of the last batch seen: the layers of a model step all ask for the same one
+    Plan* plan_cache;
+    std::vector<int32_t> plan_P, plan_Q;
     char err[512];
 };
 
@@ -70,7 +75,7 @@ struct Plan {
 };
 
 // Decide kernel kind, KV splits and partial slots for every sequence (host lengths only).
-agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, int pt_stride, Plan& plan) {
+agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, int pt_stride, Plan& plan) {
     const agx_config& c = h->cfg;
     const int G = c.num_q_heads / c.num_kv_heads;
     std::vector<int> row0(B + 1, 0);
@@ -239,6 +244,29 @@ agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, i
     return AGX_OK;
 }
 
+// The plan for this batch: the cached one when the lengths are those of the last call on the handle.
+agx_status make_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, int pt_stride, const Plan*& out) {
+    if (h->plan_cache && (int)h->plan_P.size() == B && memcmp(h->plan_P.data(), P, sizeof(int32_t) * B) == 0 &&
+        memcmp(h->plan_Q.data(), Q, sizeof(int32_t) * B) == 0) {
+        if (pt_stride >= 0)
+            for (int s = 0; s < B; ++s)
+                if ((long long)P[s] + Q[s] > (long long)pt_stride * kPage)
+                    return fail(h, AGX_E_RANGE, "sequence %d: %d + %d tokens exceed the page table (%d pages)", s, P[s], Q[s], pt_stride);
+        out = h->plan_cache;
+        return AGX_OK;
+    }
+    if (!h->plan_cache) h->plan_cache = new (std::nothrow) Plan;
+    if (!h->plan_cache) return fail(h, AGX_E_NOMEM, "out of host memory");
+    h->plan_P.clear();   // (invalid while it is rebuilt)
+    *h->plan_cache = Plan();
+    agx_status st = build_plan(h, B, P, Q, pt_stride, *h->plan_cache);
+    if (st != AGX_OK) return st;
+    h->plan_P.assign(P, P + B);
+    h->plan_Q.assign(Q, Q + B);
+    out = h->plan_cache;
+    return AGX_OK;
+}
+
 inline size_t part_ml_bytes(long long entries) { return (size_t)((entries * sizeof(float2) + 255) / 256 * 256); }
 
 }  // namespace
@@ -308,6 +336,7 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
 agx_status agx_destroy(agx_handle* h) {
     if (!h) return AGX_E_INVAL;
     cudaFree(h->d_status);
+    delete h->plan_cache;
     delete h;
     return AGX_OK;
 }
@@ -337,9 +366,10 @@ int64_t agx_attn_workspace_bytes(agx_handle* h, int32_t B, const int32_t* P, con
     if (B < 0) return fail(h, AGX_E_INVAL, "negative B");
     if (B == 0) return 0;
     if (!P || !Q) return fail(h, AGX_E_INVAL, "null pointer");
-    Plan plan;
-    agx_status st = make_plan(h, B, P, Q, -1, plan);
+    const Plan* plan_ptr = nullptr;
+    agx_status st = make_plan(h, B, P, Q, -1, plan_ptr);
     if (st != AGX_OK) return st;
+    const Plan& plan = *plan_ptr;
     if (plan.part_entries == 0) return 0;
     return (int64_t)(part_ml_bytes(plan.part_entries) + (size_t)plan.part_entries * h->cfg.head_dim * sizeof(float));
 }
@@ -361,9 +391,10 @@ static agx_status attn_impl(agx_handle* h, const void* q_block, const void* k_ne
     if (!aligned(q_block, 16) || !aligned(out, 16) || !aligned(k_pool, 256) || !aligned(v_pool, 256))
         return fail(h, AGX_E_INVAL, "q_block/out must be 16-byte and pools 256-byte aligned");
     if (num_pages < 1 || pt_stride < 1) return fail(h, AGX_E_INVAL, "num_pages and page_table_stride must be >= 1");
-    Plan plan;
-    agx_status st = make_plan(h, B, P, Q, pt_stride, plan);
+    const Plan* plan_ptr = nullptr;
+    agx_status st = make_plan(h, B, P, Q, pt_stride, plan_ptr);
     if (st != AGX_OK) return st;
+    const Plan& plan = *plan_ptr;
     const size_t need = plan.part_entries == 0 ? 0
         : part_ml_bytes(plan.part_entries) + (size_t)plan.part_entries * h->cfg.head_dim * sizeof(float);
     if (need > 0) {
