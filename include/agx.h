@@ -404,6 +404,29 @@ AGX_API agx_status agx_kv_import_pages(agx_handle* handle, void* k_pool, void* v
                                        const void* h_k_pages, const void* h_v_pages, const int32_t* dst_pages,
                                        int32_t count, void* staging, size_t staging_bytes, void* stream);
 
+/*
+ * agx_set_option - per-handle switches.  No paper counterpart (plumbing).
+ *   AGX_OPT_EARLY_PREFIX_LOADS (value 0 / 1, default 0; environment AGX_EARLY_PREFIX sets the default)
+ *       The attention kernels are chained to the launch in front of them by programmatic dependent launch: their CTAs
+ *       take their seats while that launch drains and wait for it before touching memory it may have written.  With
+ *       this option on, the CTAs fetch page-table entries and K/V pages that lie wholly below the cached-prefix length
+ *       (tokens < 16 * floor(prefix_len / 16)) BEFORE that wait, so the first loads of one attention call overlap the
+ *       tail of the previous kernel.  The caller thereby vouches that no work still in flight on the stream when the
+ *       call is enqueued writes the page table or those pages: true for a cache written by earlier steps or by other
+ *       layers' calls on other pools; NOT true directly behind agx_kv_import_pages, agx_kv_copy_pages or a
+ *       chunked prefill's previous chunk on the same pool (leave the option off there, or put an event or any launch
+ *       that is not part of this library in between).  The block's own rows and Q are always read after the wait.
+ *   AGX_OPT_WAIT_LIMIT_CYCLES (value >= 1000, default 4e9 ~ 2 s)
+ *       Clock ticks after which an in-kernel wait gives up, sets AGX_DEV_WAIT_TIMEOUT and winds the CTA down.
+ *   AGX_OPT_TEST_DROP_STAGE (value = stage index, -1 = off, default -1)
+ *       Test hook for the give-up path: the copy-issuing warp of every attention CTA leaves that K/V pipeline stage out
+ *       (nothing is armed, nothing is copied), so the waits for it run out after the wait limit and the launch ends
+ *       with AGX_DEV_WAIT_TIMEOUT.  Meant to be used with a short wait limit; results of such a launch are invalid.
+ * Errors: AGX_E_INVAL (unknown option), AGX_E_RANGE.
+ */
+enum { AGX_OPT_EARLY_PREFIX_LOADS = 1, AGX_OPT_WAIT_LIMIT_CYCLES = 2, AGX_OPT_TEST_DROP_STAGE = 3 };
+AGX_API agx_status agx_set_option(agx_handle* handle, int32_t option, int64_t value);
+
 /* Number of kernels the last agx_attn_prefixed / agx_accept_greedy / agx_kv_append call on this
  * handle launched (for launch accounting in benchmarks). */
 AGX_API int32_t agx_last_launch_count(const agx_handle* handle);

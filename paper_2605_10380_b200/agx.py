@@ -16,6 +16,7 @@ import numpy as np
 AGX_OK = 0
 AGX_BF16, AGX_F32 = 0, 1
 AGX_DEV_BAD_PAGE, AGX_DEV_WAIT_TIMEOUT, AGX_DEV_BAD_TOKEN = 1, 2, 4
+AGX_OPT_EARLY_PREFIX_LOADS, AGX_OPT_WAIT_LIMIT_CYCLES, AGX_OPT_TEST_DROP_STAGE = 1, 2, 3
 DTYPES = {"bf16": AGX_BF16, "f32": AGX_F32}
 
 _LIB_PATH = Path(__file__).resolve().parent / "lib" / "libagx.so"
@@ -28,7 +29,7 @@ EXPORTS = (
     "agx_verify_step_host_workspace_bytes", "agx_verify_step_host", "agx_verify_step_host_enqueue",
     "agx_accept_greedy_static", "agx_ngram_lut_bytes", "agx_ngram_workspace_bytes", "agx_ngram_build", "agx_ngram_draft",
     "agx_pw_select_combinations", "agx_pw_longest_prefix", "agx_kv_copy_pages",
-    "agx_kv_import_staging_bytes", "agx_kv_import_pages",
+    "agx_kv_import_staging_bytes", "agx_kv_import_pages", "agx_set_option",
 )
 
 
@@ -153,6 +154,8 @@ def load() -> ctypes.CDLL:
     lib.agx_kv_import_staging_bytes.restype = i64
     lib.agx_kv_import_pages.argtypes = [vp, vp, vp, i64, vp, vp, vp, i32, vp, ctypes.c_size_t, vp]
     lib.agx_kv_import_pages.restype = i32
+    lib.agx_set_option.argtypes = [vp, i32, i64]
+    lib.agx_set_option.restype = i32
     _lib = lib
     return lib
 
@@ -218,6 +221,10 @@ class Handle:
     def _check(self, st: int, where: str):
         if st != AGX_OK:
             raise AgxError(st, where, self._lib.agx_last_error(self._h).decode())
+
+    # -- agx_set_option
+    def set_option(self, option: int, value: int) -> None:
+        self._check(self._lib.agx_set_option(self._h, int(option), int(value)), "agx_set_option")
 
     def last_launch_count(self) -> int:
         return int(self._lib.agx_last_launch_count(self._h))

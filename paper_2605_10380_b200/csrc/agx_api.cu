@@ -6,11 +6,20 @@
 
 #include <algorithm>
 #include <new>
+#include <unordered_map>
 #include <vector>
 
 #include "agx_internal.cuh"
 
-namespace { struct Plan; }
+namespace {
+struct Plan;
+// TMA view of one KV pool, kept per pool address: encoding a tensor map costs about as much host time as a launch.
+struct PoolMap {
+    alignas(64) CUtensorMap map;
+    long long num_pages;
+    int hkv;
+};
+}  // namespace
 
 struct agx_handle {
     agx_config cfg;
@@ -28,6 +37,10 @@ struct agx_handle {
     bool cluster_merge;     // KV splits of the small-q kernel merged inside thread-block clusters where the batch allows (env AGX_CLUSTER_MERGE=0 turns it off)
     int zero_copy;          // host steps: bit 0 = kernels read small pinned inputs, bit 1 = kernels write `out` into a pinned buffer (env AGX_ZERO_COPY, default 3)
     int stream_min_tokens;  // context length from which blocks of <= 32 rows take the tensor-core stream schedule (env AGX_STREAM_MIN_TOKENS; -1 = by block height)
+    long long wait_limit_cycles;   // AGX_OPT_WAIT_LIMIT_CYCLES
+    int early_prefix;       // AGX_OPT_EARLY_PREFIX_LOADS
+    int drop_stage;         // AGX_OPT_TEST_DROP_STAGE (-1 = none)
+    std::unordered_map<const void*, PoolMap> pool_maps;
     std::vector<int32_t> cu_host;  // staging for agx_verify_step_host (lives until its final sync)
     // the launch plan of the last batch seen: the layers of a model step all ask for the same one
     Plan* plan_cache;
@@ -54,6 +67,19 @@ agx_status cuda_fail(agx_handle* h, cudaError_t e, const char* what) {
 }
 
 inline bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+// The handle's tensor map of a pool (encoded on first use of that address with that geometry).
+const CUtensorMap* pool_map(agx_handle* h, const void* pool, long long num_pages, int hkv) {
+    auto it = h->pool_maps.find(pool);
+    if (it != h->pool_maps.end() && it->second.num_pages == num_pages && it->second.hkv == hkv) return &it->second.map;
+    if (h->pool_maps.size() >= 4096) h->pool_maps.clear();
+    PoolMap& pm = h->pool_maps[pool];
+    pm.num_pages = -1;
+    if (!make_pool_map(&pm.map, pool, num_pages, hkv)) { h->pool_maps.erase(pool); return nullptr; }
+    pm.num_pages = num_pages;
+    pm.hkv = hkv;
+    return &pm.map;
+}
 inline int round_up(long long v, int m) { return (int)((v + m - 1) / m * m); }
 inline int elem_size(int dtype) { return dtype == AGX_BF16 ? 2 : 4; }
 
@@ -107,7 +133,7 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
         if (c.dtype == AGX_F32) k = KIND_SIMT;
         else {
             const int rows = Q[s] * G;
-            const bool tile_ok = !h->force_mma_sync && attn_tile_available();
+            const bool tile_ok = !h->force_mma_sync;
             // up to 128 rows: one Q tile per CTA, KV tiles alternating between two softmax warpgroups (HBM-bound
             // streaming on the tcgen05 pipe); blocks of at most 32 rows over short contexts stay with the warp-MMA
             // kernel, whose fixed costs are lower (none above 32 rows)
@@ -116,7 +142,7 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
             if (tile_ok && rows <= 128 && (rows > 32 || batch_streams || P[s] + Q[s] >= cross)) k = KIND_STREAM;
             else if (rows <= 16) k = KIND_SMALL1;
             else if (rows <= 32) k = KIND_SMALL2;
-            else if (rows <= kSmallRowsMax || h->force_mma_sync || !attn_tile_available()) k = KIND_SMALL4;
+            else if (rows <= kSmallRowsMax || h->force_mma_sync) k = KIND_SMALL4;
             else k = KIND_TILE;
             if (k == KIND_SMALL1 || k == KIND_SMALL2) { warp_mma_tokens += P[s] + Q[s]; ++warp_mma_seqs; }
         }
@@ -319,6 +345,10 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     h->batch_stream_tokens = env ? atoi(env) : getenv("AGX_STREAM_MIN_TOKENS") ? 0x7FFFFFFF : 24576;
     env = getenv("AGX_DEBUG_PLAN");
     h->debug_plan = env ? atoi(env) : 0;
+    h->wait_limit_cycles = kWaitLimitCycles;
+    env = getenv("AGX_EARLY_PREFIX");
+    h->early_prefix = env ? atoi(env) : 0;
+    h->drop_stage = -1;
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
     int major = 0;
@@ -414,6 +444,16 @@ static agx_status attn_impl(agx_handle* h, const void* q_block, const void* k_ne
     p.hq = h->cfg.num_q_heads; p.hkv = h->cfg.num_kv_heads; p.head_dim = h->cfg.head_dim;
     p.scale_log2 = h->scale * 1.4426950408889634f;
     p.row_div_magic = (0x100000000ull + (unsigned)(p.hq / p.hkv) - 1) / (unsigned)(p.hq / p.hkv);
+    p.wait_limit_cycles = h->wait_limit_cycles;
+    p.early_prefix = h->early_prefix;
+    p.drop_stage = h->drop_stage;
+    const CUtensorMap *map_k = nullptr, *map_v = nullptr;
+    if (h->cfg.dtype == AGX_BF16) {
+        if ((long long)num_pages * p.hkv * kPage > 0x7FFFFFFFll) return fail(h, AGX_E_RANGE, "pool too large for one tensor map");
+        map_k = pool_map(h, k_pool, num_pages, p.hkv);
+        map_v = pool_map(h, v_pool, num_pages, p.hkv);
+        if (!map_k || !map_v) return fail(h, AGX_E_CUDA, "cuTensorMapEncodeTiled failed");
+    }
     for (const Launch& ln : plan.launches) {
         p.num_seqs = (int)ln.seqs.size();
         p.num_items = ln.num_items;
@@ -426,6 +466,7 @@ static agx_status attn_impl(agx_handle* h, const void* q_block, const void* k_ne
         }
         cudaError_t e;
         p.cluster_size = ln.cluster;
+        p.part_half = ln.kind == KIND_TILE;
         p.k_new = p.v_new = nullptr;
         if (k_new) {
             p.k_new = k_new; p.v_new = v_new;
@@ -437,12 +478,12 @@ static agx_status attn_impl(agx_handle* h, const void* q_block, const void* k_ne
             }
         }
         switch (ln.kind) {
-            case KIND_SMALL1: e = launch_attn_small_bf16(p, 1, ln.kw, stream); break;
-            case KIND_SMALL2: e = launch_attn_small_bf16(p, 2, ln.kw, stream); break;
-            case KIND_SMALL4: e = launch_attn_small_bf16(p, 4, 4, stream); break;
+            case KIND_SMALL1: e = launch_attn_small_bf16(p, 1, ln.kw, *map_k, *map_v, stream); break;
+            case KIND_SMALL2: e = launch_attn_small_bf16(p, 2, ln.kw, *map_k, *map_v, stream); break;
+            case KIND_SMALL4: e = launch_attn_small_bf16(p, 4, 4, *map_k, *map_v, stream); break;
             case KIND_SIMT: e = launch_attn_simt_f32(p, stream); break;
-            case KIND_TILE: e = launch_attn_tile_bf16(p, false, stream); break;
-            case KIND_STREAM: e = launch_attn_tile_bf16(p, true, stream); break;
+            case KIND_TILE: e = launch_attn_tile_bf16(p, false, *map_k, *map_v, stream); break;
+            case KIND_STREAM: e = launch_attn_tile_bf16(p, true, *map_k, *map_v, stream); break;
             default: return fail(h, AGX_E_UNSUPPORTED, "unknown kernel kind");
         }
         if (e != cudaSuccess) return cuda_fail(h, e, "attention launch");
@@ -535,6 +576,25 @@ agx_status agx_get_status(agx_handle* h, void* stream, int32_t* device_status) {
 }
 
 int32_t agx_last_launch_count(const agx_handle* h) { return h ? h->last_launches : 0; }
+
+agx_status agx_set_option(agx_handle* h, int32_t option, int64_t value) {
+    if (!h) return AGX_E_INVAL;
+    switch (option) {
+        case AGX_OPT_EARLY_PREFIX_LOADS:
+            h->early_prefix = value != 0;
+            return AGX_OK;
+        case AGX_OPT_WAIT_LIMIT_CYCLES:
+            if (value < 1000) return fail(h, AGX_E_RANGE, "wait limit below 1000 cycles");
+            h->wait_limit_cycles = value;
+            return AGX_OK;
+        case AGX_OPT_TEST_DROP_STAGE:
+            if (value < -1 || value > 0x7FFFFFFF) return fail(h, AGX_E_RANGE, "stage index");
+            h->drop_stage = (int)value;
+            return AGX_OK;
+        default:
+            return fail(h, AGX_E_INVAL, "unknown option %d", option);
+    }
+}
 
 }  // extern "C"
 

@@ -19,6 +19,7 @@
 // for a 32-row verify block, one CTA per SM) halves the number of page steps per warp.  Splits write
 // fp32 (m, l, O) partials; a combine kernel merges them in fixed order, so results are bit-reproducible
 // run to run.
+#include <cuda_fp16.h>
 #include <math.h>
 
 #include "agx_internal.cuh"
@@ -124,7 +125,13 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     const int* pt_row = p.page_table + (long long)sp.seq_index * p.pt_stride;
     const int page0 = tok_begin / kPage;
     const int n_pages = (tok_end - tok_begin + kPage - 1) / kPage;
-    pdl_wait();   // from here on global memory written by the launch before this one is read
+    // A CTA whose KV split holds block rows stores them itself first (fused append) and keeps its copies back until
+    // they are in place.  Any other CTA may, with p.early_prefix (the caller vouches that the page table and the pages
+    // below the cached-prefix length are not written by a launch still in flight), fetch page ids and K/V stages that
+    // lie wholly inside the cached prefix before the dependency wait, i.e. while the launch in front drains.
+    const bool own_rows = p.k_new && tok_begin < L && tok_begin + sp.split_tokens > P;
+    const bool pre = p.early_prefix && !own_rows;
+    if (!(warp == 0 && pre)) pdl_wait();   // from here on global memory written by the launch before this one is read
     // ---- producer state (warp 0; lane 0 issues the TMA copies).  Page ids are fetched 32 at a time,
     //      one group ahead, so the page-table latency never sits in front of a copy.
     int ids_cur = 0, ids_next = 0, group_cur = 0;
@@ -138,10 +145,11 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
         return (int)id;
     };
     bool alive = true;
+    int last_armed = -1;              // last stage whose copies were armed (lane 0 of warp 0)
     auto produce = [&](int stage) {   // called by all lanes of warp 0
         if (stage >= n_stages || !alive) return;
         const int slot = stage % NS;
-        alive = mbar_wait(empty_bar(slot), ((stage / NS) & 1) ^ 1, abort_flag, p.status);
+        alive = mbar_wait(empty_bar(slot), ((stage / NS) & 1) ^ 1, abort_flag, p.status, p.wait_limit_cycles);
         if (!alive) return;
         const int pi0 = stage * kKW;
         if ((pi0 >> 5) != group_cur) { ids_cur = ids_next; group_cur = pi0 >> 5; ids_next = fetch_ids(group_cur + 1); }
@@ -149,8 +157,10 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
         int id[kKW];
 #pragma unroll
         for (int pg = 0; pg < kKW; ++pg) id[pg] = __shfl_sync(0xFFFFFFFFu, ids_cur, (pi0 + pg) & 31);
+        if (stage == p.drop_stage) return;   // test hook: this stage never arrives, its consumers' waits run out
         if (lane == 0) {
             mbar_arrive_expect_tx(full_bar(slot), npg * 8192u);
+            last_armed = stage;
             const uint32_t dst0 = smem_base + slot * kStageBytes;
 #pragma unroll
             for (int pg = 0; pg < kKW; ++pg) {
@@ -166,19 +176,23 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
         }
     };
     // The producer lane set the barriers up itself, so it needs nothing from the other warps: it fetches the page
-    // ids and issues the first copies at once, while the others bring the Q tile in.  Only a CTA that first writes
-    // rows of its own (fused append) holds its copies back until those rows are in place.
-    const bool early = !(p.k_new && tok_begin < L && tok_begin + sp.split_tokens > P);
+    // ids and issues the first copies at once, while the others bring the Q tile in.
     if (warp == 0) {
         __syncwarp();   // lane 0's barrier initialisation, before the other lanes poll those barriers
         ids_cur = fetch_ids(0);
         ids_next = fetch_ids(1);
-        if (early) {
+        bool waited = !pre;
+        if (!own_rows) {
+            const int stable_end = P & ~(kPage - 1);   // tokens below this sit in pages no append of this block touches
 #pragma unroll
-            for (int s = 0; s < NS - 1; ++s) produce(s);
+            for (int s = 0; s < NS - 1; ++s) {
+                if (!waited && tok_begin + (s + 1) * kStageTokens > stable_end) { pdl_wait(); waited = true; }
+                produce(s);
+            }
         }
+        if (!waited) pdl_wait();
     }
-    if (p.k_new) append_rows_bf16(p, sp, g, tok_begin, tok_begin + sp.split_tokens, tid, kThreads);   // fused append (row_chunks == 1)
+    if (own_rows) append_rows_bf16(p, sp, g, tok_begin, tok_begin + sp.split_tokens, tid, kThreads);   // fused append (row_chunks == 1)
     // ---- Q tile -> shared (rows beyond q*G are zero), by the warps other than the producer's
     for (int c = tid - 32; c >= 0 && c < MT * 16 * 16; c += kThreads - 32) {
         const int r = c >> 4, ch = c & 15;
@@ -191,7 +205,7 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
         *(uint4*)(q_smem + swz(r, ch)) = v;
     }
     __syncthreads();  // barriers initialised, Q tile visible
-    if (warp == 0 && !early) {
+    if (warp == 0 && own_rows) {
 #pragma unroll
         for (int s = 0; s < NS - 1; ++s) produce(s);
     }
@@ -244,7 +258,7 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     for (int stage = 0; stage < n_stages; ++stage) {
         const int slot = stage % NS;
         if (warp == 0) produce(stage + NS - 1);
-        if (live) live = mbar_wait(full_bar(slot), (stage / NS) & 1, abort_flag, p.status);
+        if (live) live = mbar_wait(full_bar(slot), (stage / NS) & 1, abort_flag, p.status, p.wait_limit_cycles);
 
         const int stage_tok0 = tok_begin + stage * kStageTokens;
         const int npg = live ? min(kKW, (tok_end - stage_tok0 + kPage - 1) / kPage) : 0;   // pages of this stage
@@ -380,6 +394,12 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
         l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 2);
     }
     if ((lane & 3) == 0) { x_l[(mt * 16 + rg) * KW + kg] = l_run[0]; x_l[(mt * 16 + rg + 8) * KW + kg] = l_run[1]; }
+    // After a wait gave up, copies armed by the producer lane may still be on their way into the ring: it waits for
+    // them (bounded by the clock alone) before the CTA reuses or releases that shared memory.
+    if (tid == 0 && *abort_flag) {
+        for (int s = max(0, last_armed - NS + 1); s <= last_armed; ++s)
+            if (s != p.drop_stage) mbar_drain(full_bar(s % NS), (s / NS) & 1, p.wait_limit_cycles);
+    }
     __syncthreads();  // all row sums in place; every armed stage has been consumed: the ring is dead
 
     // With clusters, the KV splits of this (sequence, KV head) are the cluster's CTAs (rank = split): the split
@@ -546,8 +566,20 @@ attn_simt_f32_kernel(const __grid_constant__ AttnParams p) {
 // Combine: out[row, h] = sum_k O_k 2^(m_k - m) / sum_k l_k 2^(m_k - m), splits in index order.
 // One warp per (row, head); lanes own 4 consecutive floats of each 128-wide chunk.
 // kMaxNs: no sequence of the launch has more splits than this (4, 16, or any number).  Four O rows per warp instead of 32
-// keep the register count low enough for ten CTAs per SM, which is what the 19 MB of partials of a split prefill need.
-template <bool kBf16Out, int kMaxNs>
+// keep the register count low enough for ten CTAs per SM, which is what the partials of a split prefill need.
+// kHalfPart: the partial rows are fp16 and already divided by their own sums l_k (the 256-row tensor-core schedule), so
+// split k weighs l_k 2^(m_k - m) instead of 2^(m_k - m).
+template <bool kHalfPart>
+__device__ __forceinline__ float4 load_part4(const AttnParams& p, long long entry, int c4) {
+    if (kHalfPart) {
+        const uint2 raw = __ldcg((const uint2*)((const unsigned char*)p.part_o + entry * 512 + c4 * 2));   // written by other SMs just before: past the L1
+        const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+        const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+        return make_float4(a.x, a.y, b.x, b.y);
+    }
+    return __ldcg((const float4*)(p.part_o + entry * p.head_dim + c4));
+}
+template <bool kBf16Out, int kMaxNs, bool kHalfPart>
 __global__ void __launch_bounds__(128, kMaxNs <= 4 ? 10 : kMaxNs <= 16 ? 5 : 3)
 attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
     constexpr bool kFew = kMaxNs <= 16;          // no second batch of 16 rows
@@ -574,7 +606,6 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
     const int c4 = lane * 4;               // each lane owns 4 output columns
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float m_all, l_all;
-    const float* o_src = p.part_o + e0 * D + c4;
     pdl_wait();   // the partials are complete
     if (kMaxNs <= 32 || ns <= 32) {
         // One round trip to memory: lane k fetches (m, l) of split k while every lane already fetches its
@@ -583,17 +614,18 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
         float4 v[kInFlight], v2[kFew ? 1 : 16];
 #pragma unroll
         for (int j = 0; j < kInFlight; ++j)
-            if (j < ns && c4 < D) v[j] = __ldcg((const float4*)(o_src + j * D));   // written by other SMs just before: past the L1
+            if (j < ns && c4 < D) v[j] = load_part4<kHalfPart>(p, e0 + j, c4);
         if (!kFew && ns > 16) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-                if (16 + j < ns && c4 < D) v2[j] = __ldcg((const float4*)(o_src + (16 + j) * D));
+                if (16 + j < ns && c4 < D) v2[j] = load_part4<kHalfPart>(p, e0 + 16 + j, c4);
         }
         m_all = ml.x;
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, off));
-        const float w_mine = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m_all);
-        l_all = ml.y * w_mine;
+        const float e_mine = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m_all);
+        l_all = ml.y * e_mine;
+        const float w_mine = kHalfPart ? l_all : e_mine;   // weight of this lane's split's O row
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xFFFFFFFFu, l_all, off);
 #pragma unroll
@@ -632,9 +664,9 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
                 float4 v[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const float mk = p.part_ml[e0 + k + j].x;
-                    w[j] = (mk == -INFINITY) ? 0.f : exp2f(mk - m_all);
-                    v[j] = *(const float4*)(p.part_o + (e0 + k + j) * D + c4);
+                    const float2 mlk = p.part_ml[e0 + k + j];
+                    w[j] = (mlk.x == -INFINITY) ? 0.f : exp2f(mlk.x - m_all) * (kHalfPart ? mlk.y : 1.f);
+                    v[j] = load_part4<kHalfPart>(p, e0 + k + j, c4);
                 }
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -642,9 +674,9 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
                 }
             }
             for (; k < ns; ++k) {
-                const float mk = p.part_ml[e0 + k].x;
-                const float w = (mk == -INFINITY) ? 0.f : exp2f(mk - m_all);
-                const float4 v = *(const float4*)(p.part_o + (e0 + k) * D + c4);
+                const float2 mlk = p.part_ml[e0 + k];
+                const float w = (mlk.x == -INFINITY) ? 0.f : exp2f(mlk.x - m_all) * (kHalfPart ? mlk.y : 1.f);
+                const float4 v = load_part4<kHalfPart>(p, e0 + k, c4);
                 if (w != 0.f) { acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w; }
             }
         }
@@ -732,12 +764,9 @@ int attn_small_max_clusters(int mt, int kw, int cluster) {
     }
 }
 
-cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, int kw, cudaStream_t stream) {
+cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, int kw, const CUtensorMap& map_k, const CUtensorMap& map_v,
+                                   cudaStream_t stream) {
     if (p.num_items == 0) return cudaSuccess;
-    if ((long long)p.num_pages * p.hkv * kPage > 0x7FFFFFFFll) return cudaErrorInvalidValue;
-    alignas(64) CUtensorMap map_k, map_v;
-    if (!make_pool_map(&map_k, p.k_pool, p.num_pages, p.hkv) || !make_pool_map(&map_v, p.v_pool, p.num_pages, p.hkv))
-        return cudaErrorNotSupported;
     switch (mt * 16 + kw) {
         case 1 * 16 + 4: return launch_small<1, 4, 3>(p, map_k, map_v, stream);
         case 2 * 16 + 4: return launch_small<2, 4, 3>(p, map_k, map_v, stream);
@@ -761,14 +790,19 @@ cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, 
     const int blocks = (int)((n + 3) / 4);
     int ns_max = 1;
     for (int i = 0; i < p.num_seqs; ++i) ns_max = p.seq[i].nsplit > ns_max ? p.seq[i].nsplit : ns_max;
-    if (dtype == AGX_BF16) {
-        if (ns_max <= 4) return launch_chained(attn_combine_kernel<true, 4>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
-        if (ns_max <= 16) return launch_chained(attn_combine_kernel<true, 16>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
-        return launch_chained(attn_combine_kernel<true, 1 << 30>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+    if (dtype == AGX_BF16 && p.part_half) {
+        if (ns_max <= 4) return launch_chained(attn_combine_kernel<true, 4, true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+        if (ns_max <= 16) return launch_chained(attn_combine_kernel<true, 16, true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+        return launch_chained(attn_combine_kernel<true, 1 << 30, true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
     }
-    if (ns_max <= 4) return launch_chained(attn_combine_kernel<false, 4>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
-    if (ns_max <= 16) return launch_chained(attn_combine_kernel<false, 16>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
-    return launch_chained(attn_combine_kernel<false, 1 << 30>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+    if (dtype == AGX_BF16) {
+        if (ns_max <= 4) return launch_chained(attn_combine_kernel<true, 4, false>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+        if (ns_max <= 16) return launch_chained(attn_combine_kernel<true, 16, false>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+        return launch_chained(attn_combine_kernel<true, 1 << 30, false>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+    }
+    if (ns_max <= 4) return launch_chained(attn_combine_kernel<false, 4, false>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+    if (ns_max <= 16) return launch_chained(attn_combine_kernel<false, 16, false>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+    return launch_chained(attn_combine_kernel<false, 1 << 30, false>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
 }
 
 }  // namespace agx

@@ -170,6 +170,11 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;\n" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
@@ -232,7 +237,7 @@ __device__ __noinline__ void tile_epilogue(unsigned char* smem, uint32_t tO, flo
     {   // the context is written by another warp at kernel start: wait for its arrival (long complete, normally)
         const uint32_t ctx_bar = smem_u32(smem) + kOffBar + 8u * BAR_CTX;
         volatile int* abort_flag = (volatile int*)(smem + kOffBar + BAR_COUNT * 8);
-        if (!mbar_wait(ctx_bar, 0, abort_flag, nullptr)) ok = false;
+        if (!mbar_wait(ctx_bar, 0, abort_flag, nullptr, *(const long long*)(smem + kOffBar + BAR_COUNT * 8 + 16))) ok = false;
     }
     const EpiCtx cx = *(const EpiCtx*)(smem + kOffCtx);
     const TileItem& it = cx.it;
@@ -308,7 +313,7 @@ __device__ __noinline__ void tile_epilogue(unsigned char* smem, uint32_t tO, flo
                     oreg[4 * v + 3] = __float_as_uint(__uint_as_float(oreg[4 * v + 3]) * w_own + (w_other != 0.f ? o1.w * w_other : 0.f));
                 }
             }
-            if (single) {
+            if (single || !kStreams) {   // (the 256-row schedule normalises its split partials too: they leave as fp16)
 #pragma unroll
                 for (int c = 0; c < 64; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * inv);
             }
@@ -330,37 +335,46 @@ __device__ __noinline__ void tile_epilogue(unsigned char* smem, uint32_t tO, flo
                     }
                 }
             } else {
+                // pack to the 16-bit output format first (bf16 results, fp16 split partials): 256 bytes per row go through
+                // the staging area, 16-byte units XOR-swizzled by row
 #pragma unroll
-                for (int v = 0; v < 16; ++v)
-                    *(uint4*)(stage + lane * 512 + (((c8 * 8 + v) ^ lane) << 4)) = make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]);
+                for (int v = 0; v < 8; ++v) {
+                    uint4 pk;
+                    if (single) {
+                        pk.x = pack_bf16(__uint_as_float(oreg[8 * v + 0]), __uint_as_float(oreg[8 * v + 1]));
+                        pk.y = pack_bf16(__uint_as_float(oreg[8 * v + 2]), __uint_as_float(oreg[8 * v + 3]));
+                        pk.z = pack_bf16(__uint_as_float(oreg[8 * v + 4]), __uint_as_float(oreg[8 * v + 5]));
+                        pk.w = pack_bf16(__uint_as_float(oreg[8 * v + 6]), __uint_as_float(oreg[8 * v + 7]));
+                    } else {
+                        pk.x = pack_f16(__uint_as_float(oreg[8 * v + 0]), __uint_as_float(oreg[8 * v + 1]));
+                        pk.y = pack_f16(__uint_as_float(oreg[8 * v + 2]), __uint_as_float(oreg[8 * v + 3]));
+                        pk.z = pack_f16(__uint_as_float(oreg[8 * v + 4]), __uint_as_float(oreg[8 * v + 5]));
+                        pk.w = pack_f16(__uint_as_float(oreg[8 * v + 6]), __uint_as_float(oreg[8 * v + 7]));
+                    }
+                    *(uint4*)(stage + lane * 256 + ((((c8 >> 1) * 8 + v) ^ (lane & 15)) << 4)) = pk;
+                }
             }
         }
     }
     if (kStreams) return;
     __syncwarp();
-    // a warp writes one row per instruction: lane j moves 16-byte unit j (fp32) or converts it to 8 bytes of bf16;
-    // eight rows' loads are in flight before the first store
+    // a half-warp writes one 256-byte row per instruction (lane j moves 16-byte unit j % 16 of row 2 u + j / 16); eight
+    // row pairs' loads are in flight before the first store
     const int n_valid = min(32, it.rows - r_warp0);
-    for (int rl0 = 0; rl0 < n_valid; rl0 += 8) {
+    for (int rl0 = 0; rl0 < n_valid; rl0 += 16) {
         uint4 v[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            const int rl = rl0 + u;
-            v[u] = *(const uint4*)(stage + (rl & 31) * 512 + ((lane ^ (rl & 31)) << 4));
+            const int rl = rl0 + 2 * u + (lane >> 4);
+            v[u] = *(const uint4*)(stage + rl * 256 + (((lane & 15) ^ (rl & 15)) << 4));
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            const int rl = rl0 + u;
+            const int rl = rl0 + 2 * u + (lane >> 4);
             const unsigned long long dst = __shfl_sync(0xFFFFFFFFu, row_dst, rl & 31);
             if (rl < n_valid) {
-                if (single) {
-                    uint2 pk;
-                    pk.x = pack_bf16(__uint_as_float(v[u].x), __uint_as_float(v[u].y));
-                    pk.y = pack_bf16(__uint_as_float(v[u].z), __uint_as_float(v[u].w));
-                    *(uint2*)((unsigned char*)dst + lane * 8) = pk;
-                } else {
-                    __stcg((uint4*)((unsigned char*)dst + lane * 16), v[u]);   // read next by other SMs
-                }
+                if (single) *(uint4*)((unsigned char*)dst + (lane & 15) * 16) = v[u];
+                else __stcg((uint4*)((unsigned char*)dst + (lane & 15) * 16), v[u]);   // split partial: read next by other SMs
             }
         }
     }
@@ -407,6 +421,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         for (int i = 0; i < BAR_COUNT; ++i)
             mbar_init(bar(i), (i == BAR_P_READY || i == BAR_P_READY + 1 || i == BAR_P_TAIL || i == BAR_P_TAIL + 1) ? 128u : (i == BAR_Q_FULL) ? (uint32_t)kQLoadThreads : 1u);
         *abort_flag = 0;
+        *(long long*)(smem + kOffBar + BAR_COUNT * 8 + 16) = p.wait_limit_cycles;   // for the out-of-line epilogue
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&map_k) : "memory");
         asm volatile("prefetch.tensormap [%0];\n" ::"l"(&map_v) : "memory");
@@ -415,9 +430,14 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
-    pdl_wait();   // from here on global memory written by the launch before this one is read (Q, page table, K/V)
+    // Early loads: with p.early_prefix the caller vouches that the page table and the K/V pages below the cached-prefix
+    // length are not written by any launch still in flight, so the producer warp may fetch them while the launch in
+    // front of this one drains.  A CTA that first stores block rows of its own (fused append) keeps to the usual order.
+    const bool own_rows = p.k_new && kv_begin < L && kv_begin + sp.split_tokens > P;
+    const bool early_cta = p.early_prefix && !own_rows;
+    if (!(warp == 0 && early_cta)) pdl_wait();   // from here on global memory written by the launch before this one is read (Q, page table, K/V)
     // fused append (one row chunk per sequence): the block's own K/V rows of this split go into the pages first
-    if (p.k_new && warp >= 2) append_rows_bf16(p, sp, g, kv_begin, kv_begin + sp.split_tokens, tid - 64, kQLoadThreads);
+    if (own_rows && warp >= 2) append_rows_bf16(p, sp, g, kv_begin, kv_begin + sp.split_tokens, tid - 64, kQLoadThreads);
     // Q: 256 rows x 256 B by 16-byte cp.async (all of a thread's copies in flight at once), written in
     // the 128-byte-swizzled K-major operand layout; rows past q * G are zero-filled.
     if (warp >= 2) {
@@ -435,7 +455,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
     // Barriers initialised, TMEM address published.  Warp 0 (which set the barriers up and needs nothing
     // from the others) only signals and goes straight to the page table and its first K/V copies.
     tc_fence_before();
-    if (warp == 0 && !p.k_new) { __syncwarp(); asm volatile("bar.arrive 2, %0;\n" ::"n"(kThreads) : "memory"); }   // (a fused append must land first)
+    if (warp == 0 && !own_rows) { __syncwarp(); asm volatile("bar.arrive 2, %0;\n" ::"n"(kThreads) : "memory"); }   // (a fused append must land first)
     else asm volatile("bar.sync 2, %0;\n" ::"n"(kThreads) : "memory");
     tc_fence_after();
     const uint32_t tmem_base = (warp == 0) ? 0u : *tmem_slot;
@@ -456,7 +476,14 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         const int n_pages_total = (kv_end - kv_begin + kPage - 1) / kPage;
         int ids = 0;  // page ids of the current group of 4 tiles: lane l holds page (group * 32 + l)
         bool ok = true;
+        bool waited = !early_cta;       // has this warp passed the dependency wait?
+        const int stable_end = P & ~(kPage - 1);   // tokens below this sit in pages no append of this block touches
+        int last_k = -1, last_v = -1;   // last tiles whose copies were armed (for the drain below)
         for (int t = 0; t < n_tiles && ok; ++t) {
+            const int tok0 = kv_begin + t * kBN;
+            const bool stable = tok0 + kBN <= stable_end;
+            // K/V tiles wholly inside the cached prefix, as far as free stages go, may be requested before the wait
+            if (!waited && !(stable && t < kStagesK)) { pdl_wait(); waited = true; }
             if ((t & 3) == 0) {
                 const int pi = t * 8 + lane;
                 long long id = 0;
@@ -466,18 +493,19 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                 }
                 ids = (int)id;
             }
+            if (t == p.drop_stage) continue;   // test hook: this tile never arrives, its consumers' waits run out
             const int ks = t % kStagesK, kph = (t / kStagesK) & 1;
             const int vs = t % kStagesV, vph = (t / kStagesV) & 1;
             const int npg = pages_in_tile(t);
-            const int tok0 = kv_begin + t * kBN;
             const int pg = lane - (t & 3) * 8;              // this lane's page of the tile
             const bool mine = pg >= 0 && pg < npg;
             const int y = (ids * p.hkv + g) * kPage;
             // ---- K
-            ok = mbar_wait(bar(BAR_K_EMPTY + ks), kph ^ 1, abort_flag, p.status);
+            ok = mbar_wait(bar(BAR_K_EMPTY + ks), kph ^ 1, abort_flag, p.status, p.wait_limit_cycles);
             if (!ok) break;
             if (lane == 0) mbar_arrive_expect_tx(bar(BAR_K_FULL + ks), npg * 4096u);
             __syncwarp();
+            last_k = t;
             if (mine) {
                 const uint32_t dst = smem_base + kOffK + ks * kTileBytes + pg * 2048;
                 tma_load_2d(dst, &map_k, 0, y, bar(BAR_K_FULL + ks));
@@ -485,7 +513,8 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             }
             // ---- V (the page that holds token L, if L is not page-aligned, is copied by hand so that
             //      slots past the end of the sequence are zeros whatever the pool holds there)
-            ok = mbar_wait(bar(BAR_V_EMPTY + vs), vph ^ 1, abort_flag, p.status);
+            if (!waited && !(stable && t < kStagesV)) { pdl_wait(); waited = true; }
+            ok = mbar_wait(bar(BAR_V_EMPTY + vs), vph ^ 1, abort_flag, p.status, p.wait_limit_cycles);
             if (!ok) break;
             const int ragged_pg = ((L & 15) != 0 && (L >> 4) >= (tok0 >> 4) && (L >> 4) < (tok0 >> 4) + npg) ? (L >> 4) - (tok0 >> 4) : -1;
             if (ragged_pg >= 0) {
@@ -495,7 +524,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                 for (int idx = lane; idx < 256; idx += 32) {
                     const int r = idx >> 4, ch = idx & 15, half = ch >> 3, u = ch & 7;
                     uint4 v = make_uint4(0, 0, 0, 0);
-                    if (r < valid_rows) v = __ldg((const uint4*)(src + r * 256 + ch * 16));
+                    if (r < valid_rows) v = __ldcg((const uint4*)(src + r * 256 + ch * 16));   // (rows a fused append may just have written)
                     *(uint4*)(smem + v_stage_off(vs) + half * kHalfBytes + ragged_pg * 2048 + r * 128 + ((u ^ (r & 7)) << 4)) = v;
                 }
                 asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
@@ -503,18 +532,20 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             }
             if (lane == 0) mbar_arrive_expect_tx(bar(BAR_V_FULL + vs), (npg - (ragged_pg >= 0 ? 1 : 0)) * 4096u);
             __syncwarp();
+            last_v = t;
             if (mine && pg != ragged_pg) {
                 const uint32_t dst = smem_base + v_stage_off(vs) + pg * 2048;
                 tma_load_2d(dst, &map_v, 0, y, bar(BAR_V_FULL + vs));
                 tma_load_2d(dst + kHalfBytes, &map_v, 64, y, bar(BAR_V_FULL + vs));
             }
         }
-        // drain: the copies this warp started must land before the CTA's shared memory goes away
+        // drain: the copies this warp started must land before the CTA's shared memory goes away.  Bounded by the
+        // clock alone: after a time-out elsewhere in the CTA the abort flag is up, and the copies still have to land.
         if (lane == 0) {
-            for (int t = max(0, n_tiles - kStagesK); t < n_tiles; ++t)
-                mbar_wait(bar(BAR_K_FULL + t % kStagesK), (t / kStagesK) & 1, abort_flag, p.status);
-            for (int t = max(0, n_tiles - kStagesV); t < n_tiles; ++t)
-                mbar_wait(bar(BAR_V_FULL + t % kStagesV), (t / kStagesV) & 1, abort_flag, p.status);
+            for (int t = max(0, last_k - kStagesK + 1); t <= last_k; ++t)
+                if (t != p.drop_stage) mbar_drain(bar(BAR_K_FULL + t % kStagesK), (t / kStagesK) & 1, p.wait_limit_cycles);
+            for (int t = max(0, last_v - kStagesV + 1); t <= last_v; ++t)
+                if (t != p.drop_stage) mbar_drain(bar(BAR_V_FULL + t % kStagesV), (t / kStagesV) & 1, p.wait_limit_cycles);
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
@@ -551,11 +582,11 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                         umma_ts(tO[x], tS[x] + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescPV, !(first && ks == 0));
                 }
             };
-            bool ok = mbar_wait(bar(BAR_Q_FULL), 0, abort_flag, p.status);
+            bool ok = mbar_wait(bar(BAR_Q_FULL), 0, abort_flag, p.status, p.wait_limit_cycles);
             if (kStreams) {
                 // stream x = t & 1 owns KV tile t:  S_0(0) S_1(1) | O_x += P_x V(t), S_x(t + 2) | ...
                 for (int t = 0; t < 2 && t < n_tiles && ok; ++t) {
-                    ok = mbar_wait(bar(BAR_K_FULL + t), 0, abort_flag, p.status);
+                    ok = mbar_wait(bar(BAR_K_FULL + t), 0, abort_flag, p.status, p.wait_limit_cycles);
                     if (!ok) break;
                     tc_fence_after();
                     issue_qk(0, t, t); umma_commit(bar(BAR_S_FULL + t));
@@ -563,20 +594,20 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                 }
                 for (int t = 0; t < n_tiles && ok; ++t) {
                     const int x = t & 1, vs = t % kStagesV, vph = (t / kStagesV) & 1, npg = pages_in_tile(t);
-                    ok = mbar_wait(bar(BAR_V_FULL + vs), vph, abort_flag, p.status);
+                    ok = mbar_wait(bar(BAR_V_FULL + vs), vph, abort_flag, p.status, p.wait_limit_cycles);
                     if (!ok) break;
-                    ok = mbar_wait(bar(BAR_P_READY + x), (t >> 1) & 1, abort_flag, p.status);
+                    ok = mbar_wait(bar(BAR_P_READY + x), (t >> 1) & 1, abort_flag, p.status, p.wait_limit_cycles);
                     if (!ok) break;
                     tc_fence_after();
                     issue_pv(x, vs, npg, t < 2, false);
-                    ok = mbar_wait(bar(BAR_P_TAIL + x), (t >> 1) & 1, abort_flag, p.status);
+                    ok = mbar_wait(bar(BAR_P_TAIL + x), (t >> 1) & 1, abort_flag, p.status, p.wait_limit_cycles);
                     if (!ok) break;
                     tc_fence_after();
                     issue_pv(x, vs, npg, t < 2, true);
                     umma_commit(bar(BAR_V_EMPTY + vs));
                     if (t + 2 < n_tiles) {
                         const int nks = (t + 2) % kStagesK, nkph = ((t + 2) / kStagesK) & 1;
-                        ok = mbar_wait(bar(BAR_K_FULL + nks), nkph, abort_flag, p.status);
+                        ok = mbar_wait(bar(BAR_K_FULL + nks), nkph, abort_flag, p.status, p.wait_limit_cycles);
                         if (!ok) break;
                         tc_fence_after();
                         issue_qk(0, nks, x); umma_commit(bar(BAR_S_FULL + x));
@@ -584,7 +615,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                     }
                 }
             } else {
-            if (ok) ok = mbar_wait(bar(BAR_K_FULL + 0), 0, abort_flag, p.status);
+            if (ok) ok = mbar_wait(bar(BAR_K_FULL + 0), 0, abort_flag, p.status, p.wait_limit_cycles);
             if (ok) {
                 tc_fence_after();
                 issue_qk(0, 0, 0); umma_commit(bar(BAR_S_FULL + 0));
@@ -595,27 +626,27 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
                 const int vs = t % kStagesV, vph = (t / kStagesV) & 1, npg = pages_in_tile(t);
                 const bool more = t + 1 < n_tiles;
                 const int nks = (t + 1) % kStagesK, nkph = ((t + 1) / kStagesK) & 1;
-                ok = mbar_wait(bar(BAR_V_FULL + vs), vph, abort_flag, p.status);
+                ok = mbar_wait(bar(BAR_V_FULL + vs), vph, abort_flag, p.status, p.wait_limit_cycles);
                 if (!ok) break;
-                ok = mbar_wait(bar(BAR_P_READY + 0), t & 1, abort_flag, p.status);
+                ok = mbar_wait(bar(BAR_P_READY + 0), t & 1, abort_flag, p.status, p.wait_limit_cycles);
                 if (!ok) break;
                 tc_fence_after();
                 issue_pv(0, vs, npg, t == 0, false);
-                ok = mbar_wait(bar(BAR_P_TAIL + 0), t & 1, abort_flag, p.status);
+                ok = mbar_wait(bar(BAR_P_TAIL + 0), t & 1, abort_flag, p.status, p.wait_limit_cycles);
                 if (!ok) break;
                 tc_fence_after();
                 issue_pv(0, vs, npg, t == 0, true);
                 if (more) {
-                    ok = mbar_wait(bar(BAR_K_FULL + nks), nkph, abort_flag, p.status);
+                    ok = mbar_wait(bar(BAR_K_FULL + nks), nkph, abort_flag, p.status, p.wait_limit_cycles);
                     if (!ok) break;
                     tc_fence_after();
                     issue_qk(0, nks, 0); umma_commit(bar(BAR_S_FULL + 0));
                 }
-                ok = mbar_wait(bar(BAR_P_READY + 1), t & 1, abort_flag, p.status);
+                ok = mbar_wait(bar(BAR_P_READY + 1), t & 1, abort_flag, p.status, p.wait_limit_cycles);
                 if (!ok) break;
                 tc_fence_after();
                 issue_pv(1, vs, npg, t == 0, false);
-                ok = mbar_wait(bar(BAR_P_TAIL + 1), t & 1, abort_flag, p.status);
+                ok = mbar_wait(bar(BAR_P_TAIL + 1), t & 1, abort_flag, p.status, p.wait_limit_cycles);
                 if (!ok) break;
                 tc_fence_after();
                 issue_pv(1, vs, npg, t == 0, true);
@@ -627,7 +658,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             }
             }
             umma_commit(bar(BAR_O_FULL));  // arrives when every MMA issued above has completed
-            mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
+            mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status, p.wait_limit_cycles);
         }
         __syncwarp();
     } else if (tid == 32 * 3) {   // an otherwise idle warp parks the epilogue's context
@@ -660,13 +691,13 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         const int t_first = kStreams ? x : 0;
         if (!warp_has_rows) {   // keep S_FULL / P_READY in step, nothing else
             for (int t = t_first; t < n_tiles && ok; t += kStep) {
-                ok = mbar_wait(bar(BAR_S_FULL + x), ((t - t_first) / kStep) & 1, abort_flag, p.status);
+                ok = mbar_wait(bar(BAR_S_FULL + x), ((t - t_first) / kStep) & 1, abort_flag, p.status, p.wait_limit_cycles);
                 if (ok) { mbar_arrive(bar(BAR_P_READY + x)); mbar_arrive(bar(BAR_P_TAIL + x)); }
             }
         } else
         for (int t = t_first; t < n_tiles; t += kStep) {
             const int j = (t - t_first) / kStep;             // this warpgroup's j-th tile
-            ok = mbar_wait(bar(BAR_S_FULL + x), j & 1, abort_flag, p.status);
+            ok = mbar_wait(bar(BAR_S_FULL + x), j & 1, abort_flag, p.status, p.wait_limit_cycles);
             if (!ok) break;
             tc_fence_after();
             uint32_t sreg[128];
@@ -746,7 +777,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
             tc_fence_before();
             mbar_arrive(bar(BAR_P_TAIL + x));
         }
-        if (ok) ok = mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status);
+        if (ok) ok = mbar_wait(bar(BAR_O_FULL), 0, abort_flag, p.status, p.wait_limit_cycles);
         if (ok || kStreams) tile_epilogue<kStreams>(smem, tO, m_ref, l_run, ok);
     }
     // ---- teardown
@@ -759,8 +790,6 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
 }
 
 // --------------------------------------------------------------------------------------------
-bool attn_tile_available() { return true; }
-
 namespace {
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -811,12 +840,9 @@ cudaError_t launch_tile(const AttnParams& p, const CUtensorMap& map_k, const CUt
 }
 }  // namespace
 
-cudaError_t launch_attn_tile_bf16(const AttnParams& p, bool streams, cudaStream_t stream) {
+cudaError_t launch_attn_tile_bf16(const AttnParams& p, bool streams, const CUtensorMap& map_k, const CUtensorMap& map_v,
+                                  cudaStream_t stream) {
     if (p.num_items == 0) return cudaSuccess;
-    if ((long long)p.num_pages * p.hkv * kPage > 0x7FFFFFFFll) return cudaErrorInvalidValue;
-    alignas(64) CUtensorMap map_k, map_v;
-    if (!make_pool_map(&map_k, p.k_pool, p.num_pages, p.hkv) || !make_pool_map(&map_v, p.v_pool, p.num_pages, p.hkv))
-        return cudaErrorNotSupported;
     return streams ? launch_tile<true>(p, map_k, map_v, stream) : launch_tile<false>(p, map_k, map_v, stream);
 }
 

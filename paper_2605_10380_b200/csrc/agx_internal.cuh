@@ -1,5 +1,6 @@
 // Internal declarations shared by the agx CUDA sources (not part of the C ABI).
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -11,6 +12,10 @@ namespace agx {
 constexpr int kPage = 16;          // tokens per KV page
 constexpr int kMaxSeqs = 48;       // sequences per attention launch (plans travel as kernel arguments)
 constexpr int kSmallRowsMax = 64;  // q_len * G above this goes to the tile kernel
+constexpr long long kWaitLimitCycles = 4000000000ll;  // ~2 s at 1.9 GHz: default limit of every in-kernel wait
+
+// 2-D TMA view of a KV pool: [num_pages * Hkv * 16 rows][128 dims] bf16, box = 16 rows x 64 dims, SWIZZLE_128B.
+bool make_pool_map(CUtensorMap* map, const void* pool, long long num_pages, int hkv);
 
 // Per-sequence launch plan, built on the host from the host lengths.
 struct SeqPlan {
@@ -32,10 +37,12 @@ struct AttnParams {
     const int* page_table;
     void* out;
     float* lse;
-    float* part_o;   // [entries][head_dim] fp32, un-normalised, relative to part_ml.x
+    float* part_o;   // [entries][head_dim] fp32, un-normalised, relative to part_ml.x; or, with part_half, rows NORMALISED by their
+                     // own sum and stored as fp16 in the first 256 bytes of the same 512-byte slots
     float2* part_ml; // [entries] (running max in log2 units, sum)
     int* status;
     unsigned long long row_div_magic;   // ceil(2^32 / G), G = hq / hkv: (row * magic) >> 32 == row / G for rows < 2^22
+    int part_half;       // != 0: split partials of this launch are normalised fp16 rows (256-row tensor-core schedule)
     int cluster_size;    // > 1: the launch's CTAs form clusters of this size = the KV splits of one (sequence, KV head), merged in-kernel
     const void* k_new;   // fused append (agx_attn_prefixed_append): the block's K/V rows [total_q][hkv][d], or NULL
     const void* v_new;
@@ -45,6 +52,10 @@ struct AttnParams {
     int num_seqs;
     int num_items;
     float scale_log2;  // scale * log2(e)
+    long long wait_limit_cycles;   // every in-kernel wait gives up after this many clock64 ticks (agx_set_option)
+    int early_prefix;    // != 0: page ids and K/V tiles that lie wholly inside the cached prefix may be fetched before the
+                         // dependency wait (the caller vouches that no launch still in flight writes them)
+    int drop_stage;      // test hook: the producer leaves this K/V stage (tile) out, so its consumers' waits run out; -1 = none
     SeqPlan seq[kMaxSeqs];
 };
 
@@ -110,17 +121,18 @@ cudaError_t launch_kv_append(int dtype, void* k_pool, void* v_pool, long long nu
 // Clusters of `cluster` CTAs of the small-q kernel <mt, kw> that can be resident at once on the current device
 // (0 when such a cluster cannot be launched); cached per device.
 int attn_small_max_clusters(int mt, int kw, int cluster);
-cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, int kw, cudaStream_t stream);
+cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, int kw, const CUtensorMap& map_k, const CUtensorMap& map_v,
+                                   cudaStream_t stream);
 // Scalar fp32-math kernel for AGX_F32 pools (any q, d in {64, 128}).
 cudaError_t launch_attn_simt_f32(const AttnParams& p, cudaStream_t stream);
 // Merge of split partials into out / lse.
-cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, cudaStream_t stream);
+cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, cudaStream_t stream);   // honours p.part_half
 
-bool attn_tile_available();
 // Tensor-core tile kernel (bf16, d = 128, tcgen05 + TMEM + TMA).  streams = false: 256 query rows per CTA
 // (two Q tiles); streams = true: 128 rows per CTA whose KV tiles alternate between two softmax warpgroups
 // (verify blocks and short suffixes over long contexts).
-cudaError_t launch_attn_tile_bf16(const AttnParams& p, bool streams, cudaStream_t stream);
+cudaError_t launch_attn_tile_bf16(const AttnParams& p, bool streams, const CUtensorMap& map_k, const CUtensorMap& map_v,
+                                  cudaStream_t stream);
 
 cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_stride, int vocab, const int* drafts,
                           const int* cu_q, int B, int total_q, int* accept_len, int* next_token, int* argmax,

@@ -9,11 +9,6 @@
 
 namespace agx {
 
-constexpr long long kWaitLimitCycles = 4000000000ll;  // ~2 s at 1.9 GHz: every in-kernel wait gives up after this
-
-// 2-D TMA view of a KV pool: [num_pages * Hkv * 16 rows][128 dims] bf16, box = 16 rows x 64 dims, SWIZZLE_128B.
-bool make_pool_map(CUtensorMap* map, const void* pool, long long num_pages, int hkv);
-
 namespace {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -35,7 +30,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false (and raises the CTA's abort flag) when the limit is hit or another
 // role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          long long limit_cycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     int spins = 0;
@@ -43,13 +39,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit_cycles) {
                 *abort_flag = 1;
                 if (status) atomicOr(status, AGX_DEV_WAIT_TIMEOUT);
                 return false;
             }
         }
     }
+}
+
+// Wait of the copy-issuing lane for copies it has armed itself, when the CTA winds down: bounded by the clock only.
+// The abort flag is ignored on purpose, since the shared memory the copies land in must stay allocated until they have.
+__device__ __forceinline__ bool mbar_drain(uint32_t bar, uint32_t parity, long long limit_cycles) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > limit_cycles) return false;
+    return true;
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
