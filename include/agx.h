@@ -215,12 +215,13 @@ AGX_API agx_status agx_accept_greedy(agx_handle* handle, const void* logits, int
  * it uses a fixed scratch array inside the library (about 73 KB of device memory on every GPU that
  * loads the library, held until the process exits).
  *
- * Limits: total_q <= 2048 logits rows per call, and rows x vocabulary chunks <= 8192 (the call
- * uses fewer, larger chunks to stay inside that); larger requests return AGX_E_RANGE and should
- * use agx_accept_greedy with a workspace.
+ * Limit: total_q <= 2048 logits rows per call; more rows return AGX_E_RANGE and should use
+ * agx_accept_greedy with a workspace.  (Each row is scanned in as many vocabulary chunks as fit the
+ * array's 8192 key slots, at most 8 CTAs per SM.)
  *
  * The first call on each device looks up the device address of the scratch array (that device
- * must be current); make that first call outside any stream capture.  Every call uses the same
+ * must be current); make that first call outside any stream capture.  The look-up is guarded, so
+ * several host threads may make their first calls at the same time.  Every call uses the same
  * array: the call clears the part that has to start at zero, but two calls that overlap on the GPU
  * (different streams, no ordering between them) race on it and give undefined results.  Calls on
  * one stream, or ordered by events, are safe.

@@ -213,6 +213,9 @@ cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_st
 // per-chunk argmax keys, the per-row winners and the ticket counter) lives in a fixed array that
 // is part of the loaded module, so every GPU that loads the library carries these 73 KB until the
 // process exits.
+#include <atomic>
+#include <mutex>
+
 namespace agx {
 namespace {
 constexpr int kStaticMaxRows = 2048;    // logits rows per call
@@ -223,10 +226,13 @@ constexpr size_t kStaticBytes = 256 + (size_t)kStaticMaxSlots * 8 + (size_t)kSta
 static __device__ __align__(256) unsigned char g_accept_scratch[kStaticBytes];
 
 struct StaticDeviceState {
-    void* scratch;  // device address of g_accept_scratch on that device (NULL until resolved)
-    int sm_count;
+    std::atomic<void*> scratch{nullptr};  // device address of g_accept_scratch on that device (NULL until resolved)
+    int sm_count = 0;                     // written before `scratch` is published
 };
 StaticDeviceState g_static_state[kStaticDevices];
+std::mutex g_static_init;                 // serialises the one-time set-up (several host threads may make the first call)
+
+inline bool aligned_to(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 }  // namespace
 }  // namespace agx
 
@@ -242,34 +248,44 @@ extern "C" AGX_API agx_status agx_accept_greedy_static(const void* logits, int32
     if (logits_dtype != AGX_BF16 && logits_dtype != AGX_F32) return AGX_E_UNSUPPORTED;
     if (vocab < 1 || row_stride < vocab) return AGX_E_RANGE;
     if (!logits || !cu_q || !accept_len || !next_token || (!drafts && total_q > B)) return AGX_E_INVAL;
+    // the same alignment rules as the workspace variant: a misaligned pointer is an argument error, not a device fault
+    if (!aligned_to(logits, logits_dtype == AGX_BF16 ? 2 : 4) || !aligned_to(drafts, 4) || !aligned_to(cu_q, 4) ||
+        !aligned_to(accept_len, 4) || !aligned_to(next_token, 4) || !aligned_to(argmax, 4) || !aligned_to(seq_lens, 4))
+        return AGX_E_INVAL;
     if (total_q > kStaticMaxRows) return AGX_E_RANGE;  // beyond the fixed scratch: use agx_accept_greedy
 
     int device = -1;
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kStaticDevices) return AGX_E_CUDA;
     StaticDeviceState& st = g_static_state[device];
-    if (!st.scratch) {
+    void* scratch = st.scratch.load(std::memory_order_acquire);
+    if (!scratch) {
         // One-time set-up for this device, with it current.  In host code the array's name is only a
         // stand-in for the symbol; the address kernels can use has to be asked for.
-        void* ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_accept_scratch) != cudaSuccess || !ptr) return AGX_E_CUDA;
-        int sms = 0;
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1) return AGX_E_CUDA;
-        st.sm_count = sms;
-        st.scratch = ptr;
+        std::lock_guard<std::mutex> lock(g_static_init);
+        scratch = st.scratch.load(std::memory_order_relaxed);
+        if (!scratch) {
+            void* ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_accept_scratch) != cudaSuccess || !ptr) return AGX_E_CUDA;
+            int sms = 0;
+            if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1) return AGX_E_CUDA;
+            st.sm_count = sms;
+            st.scratch.store(ptr, std::memory_order_release);
+            scratch = ptr;
+        }
     }
-    // same chunking rule as the workspace variant, then shrunk to the fixed number of slots
+    // Chunks per row: enough CTAs that every thread needs a single trip of two 16-byte loads (8 per SM, as the workspace
+    // variant aims for), as far as the fixed number of key slots goes: rows * chunks <= target + rows <= kStaticMaxSlots.
     const int vec = logits_dtype == AGX_BF16 ? 8 : 4;
-    int want = (2 * st.sm_count + total_q - 1) / total_q;
-    const int max_chunks = (vocab + 256 * vec * 2 - 1) / (256 * vec * 2);
+    const int target = 8 * st.sm_count < kStaticMaxSlots - kStaticMaxRows ? 8 * st.sm_count : kStaticMaxSlots - kStaticMaxRows;
+    int want = (target + total_q - 1) / total_q;
+    const int max_chunks = (vocab + 256 * vec * 2 - 1) / (256 * vec * 2);   // >= 2 vectors per thread
     if (want > max_chunks) want = max_chunks;
-    if (want > kStaticMaxSlots / total_q) want = kStaticMaxSlots / total_q;
     if (want < 1) want = 1;
     int chunk_elems = (vocab + want - 1) / want;
     chunk_elems = (chunk_elems + vec - 1) / vec * vec;
-    const int chunks = (vocab + chunk_elems - 1) / chunk_elems;
-    if ((long long)chunks * total_q > kStaticMaxSlots) return AGX_E_RANGE;
+    const int chunks = (vocab + chunk_elems - 1) / chunk_elems;   // <= want
 
-    unsigned char* base = (unsigned char*)st.scratch;
+    unsigned char* base = (unsigned char*)scratch;
     // the array keeps whatever the previous call left: the ticket counter must start at zero
     if (cudaMemsetAsync(base, 0, 256, (cudaStream_t)stream) != cudaSuccess) return AGX_E_CUDA;
     // launch_accept places the per-row winners right behind total_q * chunks keys

@@ -325,6 +325,3 @@ def c5_long_context(seed: int = 5, verify_only: bool = False, prefill_only: bool
         P, q = P[4:], q[4:]
     return make_attn_workload("c5_long_context", seed, "bf16", 32, 8, 128, P, q)
 
-
-def accept_for(name: str, seed: int, dtype: str, vocab: int, q_len, prefix_len) -> AcceptWorkload:
-    return make_planted_accept(name, seed, dtype, vocab, q_len, prefix_len)

@@ -84,10 +84,10 @@ def check_attention(gpu: np.ndarray, ref: np.ndarray, what: str = "", strict: bo
     ||gpu - ref||_inf / ||ref||_inf <= 2e-2.
 
     The 1e-2 absolute bound is stated for unit-variance inputs whose outputs are averages, i.e. of
-    magnitude below 1.  A row whose reference exceeds 1 in magnitude (very short contexts, where one
-    value row dominates) gets the bound scaled by that magnitude: bfloat16 output spacing is 2^-7
-    relative, so at |o| >= 4 even the correctly rounded result can miss 1e-2.  ``strict=True`` (the
-    named configurations) applies the unscaled 1e-2 to every row."""
+    magnitude below 1.  A row whose reference is larger (contexts of a handful of tokens, where one
+    value row dominates) is allowed what the arithmetic adds on top: outputs are rounded to bfloat16,
+    whose half-ulp is at most 2^-8 relative, so the bound is 1e-2 + 2^-8 * ||ref||_inf.
+    ``strict=True`` (the named configurations) applies the plain 1e-2 to every row."""
     assert gpu.shape == ref.shape
     assert np.all(np.isfinite(gpu)), f"{what}: non-finite output"
     err = np.abs(gpu - ref)
@@ -97,9 +97,9 @@ def check_attention(gpu: np.ndarray, ref: np.ndarray, what: str = "", strict: bo
     row_ref = np.abs(ref).max(axis=-1)
     max_abs = float(row_err.max())
     rel = float((row_err / np.maximum(row_ref, 1e-30)).max())
-    bound = ATOL * (1.0 if strict else np.maximum(1.0, row_ref))
+    bound = ATOL + (0.0 if strict else 2.0 ** -8 * row_ref)
     worst = float((row_err / bound).max())
-    assert worst <= 1.0, f"{what}: max-abs {max_abs:.3e} exceeds {ATOL} (scaled ratio {worst:.2f})"
+    assert worst <= 1.0, f"{what}: max-abs {max_abs:.3e} exceeds its bound (ratio {worst:.2f})"
     assert rel <= RTOL, f"{what}: normwise relative {rel:.3e} > {RTOL}"
     return max_abs, rel
 

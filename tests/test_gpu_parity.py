@@ -16,8 +16,12 @@ from tests.gpu_util import (DeviceBatch, check_attention, dev, host_storage, ora
 pytestmark = pytest.mark.gpu
 
 
-def run_and_check(w, sample=None, poison=False, strict=False, fused=False):
+def run_and_check(w, sample=None, poison=False, strict=False, fused=False, select=None, options=()):
+    """sample=(seed, n): n random (row, head) pairs per sequence plus the corners; select={s: (rows, heads)}: those
+    pairs for sequence s and EVERY output row of the other sequences; neither: every output row of the batch."""
     b = DeviceBatch(w)
+    for opt, val in options:
+        b.h.set_option(opt, val)
     if poison:  # slots past P + q in every sequence's last page hold NaN: they must never be read
         nanbits = 0x7FC0 if w.dtype == "bf16" else np.float32(np.nan)
         for s in range(w.batch):
@@ -38,10 +42,25 @@ def run_and_check(w, sample=None, poison=False, strict=False, fused=False):
     gk = host_storage(b.k_pool, w.dtype); gv = host_storage(b.v_pool, w.dtype)
     if not poison:
         assert np.array_equal(gk, kp) and np.array_equal(gv, vp)
-    if sample is None:
+    if sample is None and select is None:
         ref, ref_lse = oracle.attn_paged_batch(w.q_block, kp, vp, w.page_table, w.dtype, w.prefix_len, w.q_len, w.cu_q)
         stats = check_attention(out, ref, w.name, strict)
         assert np.max(np.abs(lse - ref_lse)) <= 2e-3, "lse"
+    elif select is not None:
+        stats = (0.0, 0.0)
+        for s in range(w.batch):
+            q = int(w.q_len[s]); r0 = int(w.cu_q[s])
+            if s in select:
+                si, sh = (np.asarray(a, dtype=np.int32) for a in select[s])
+                ref, ref_lse, _ = oracle.attn_paged(w.q_block[r0:r0 + q], kp, vp, w.page_table[s], w.dtype,
+                                                    int(w.prefix_len[s]), select=(si, sh))
+                got, got_lse = out[r0 + si, sh], lse[r0 + si, sh]
+            else:
+                ref, ref_lse, _ = oracle.attn_paged(w.q_block[r0:r0 + q], kp, vp, w.page_table[s], w.dtype, int(w.prefix_len[s]))
+                got, got_lse = out[r0:r0 + q], lse[r0:r0 + q]
+            st = check_attention(got, ref, f"{w.name} seq {s}", strict)
+            stats = (max(stats[0], st[0]), max(stats[1], st[1]))
+            assert np.max(np.abs(got_lse - ref_lse)) <= 2e-3
     else:
         rng = np.random.default_rng(sample[0])
         stats = (0.0, 0.0)
@@ -102,18 +121,35 @@ def test_c1_accept_fp32_first_two_of_three_match():
 
 def test_c4_ragged_mixed_batch_shared_prefix():
     """16 sequences, lognormal prefixes, verify blocks and suffix prefills in one call, first 2048
-    tokens' pages shared by all: every sequence's first and last block row plus seeded samples."""
+    tokens' pages shared by all: EVERY output row of every sequence against the oracle."""
     w = W.c4_ragged_mixed()
     assert np.all(w.page_table[:, :128] == w.page_table[0, :128])
-    b, _ = run_and_check(w, sample=(4, 24), strict=True)
+    b, _ = run_and_check(w, strict=True)
     assert b.launches >= 3  # split-KV kernel(s), tile kernel, combine
 
 
+def tile_edge_rows(q, G, hq, seed, extra):
+    """(row, head) pairs that look into every CTA of the 256-row schedule: for every KV head the rows at
+    positions 0, 127, 128 and 255 of every 256-row chunk (first and last row of both Q tiles), plus `extra`
+    seeded random pairs."""
+    hkv = hq // G
+    si, sh = [], []
+    for g in range(hkv):
+        for r in range(0, q * G):
+            if r % 256 in (0, 127, 128, 255) or r == q * G - 1:
+                si.append(r // G); sh.append(g * G + r % G)
+    rng = np.random.default_rng(seed)
+    si += rng.integers(0, q, extra).tolist(); sh += rng.integers(0, hq, extra).tolist()
+    return np.asarray(si, np.int32), np.asarray(sh, np.int32)
+
+
 def test_c5_long_context_verify_and_prefill():
-    """4 x (P = 32768, q = 8) plus 1 x (P = 30720, q = 2048) in one call, sampled rows against the
-    oracle; then the accept step on bf16 logits [4 x 8, 128256]."""
+    """4 x (P = 32768, q = 8) plus 1 x (P = 30720, q = 2048) in one call.  Every output row of the four verify
+    blocks is compared with the oracle; of the 2048-row prefill, the first and last row of every 128-row Q tile
+    of every KV head (so every (row chunk, KV head, KV split) CTA is looked at) plus 200 random (row, head)
+    pairs.  Then the accept step on bf16 logits [4 x 8, 128256]."""
     w = W.c5_long_context()
-    b, _ = run_and_check(w, sample=(6, 24), strict=True)
+    b, _ = run_and_check(w, strict=True, select={4: tile_edge_rows(2048, 4, 32, 6, 200)})
     h = agx.Handle(32, 8, 128, "bf16")
     aw = W.make_planted_accept("c5_accept", 55, "bf16", 128256, [8] * 4, [32768] * 4)
     ref = oracle.accept_greedy(aw.logits, "bf16", aw.vocab, aw.drafts, aw.cu_q, aw.prefix_len)
@@ -726,14 +762,14 @@ def test_fused_append_reports_a_bad_page_and_skips_the_row():
 ])
 def test_tile_kernel_shapes(P, q, hq, hkv):
     w = W.make_attn_workload(f"tile_{P}_{q}", 2000 + P + q, "bf16", hq, hkv, 128, [P], [q], spare_pages=2)
-    run_and_check(w, sample=(11, 150), poison=True)
+    run_and_check(w, poison=True)   # every output row
 
 
 def test_c3_prefix_cached_prefill_and_full_prefill_rows():
     """Prefix-cached prefill (P = 3072, q = 512, 24/8 heads) against the oracle, and the oracle's own
     check that these rows equal rows 3072.. of a full 3584-token uncached prefill."""
     w = W.c3_prefix_prefill()
-    b, stats = run_and_check(w, sample=(5, 300), strict=True)
+    b, stats = run_and_check(w, strict=True)   # every output row
     out = b.out.to(torch.float64).cpu().numpy()
     kp, vp = oracle_pools_after_append(w)
     P, q = 3072, 512
@@ -749,7 +785,7 @@ def test_tile_and_small_kernels_in_one_ragged_batch():
     P = [2048, 2300, 2048 + 7, 4000, 2600, 3000]
     q = [8, 200, 1, 130, 16, 513]
     w = W.make_attn_workload("mixed", 91, "bf16", 32, 8, 128, P, q, shared_prefix_tokens=2048)
-    b, _ = run_and_check(w, sample=(2, 60))
+    b, _ = run_and_check(w)   # every output row
     assert b.launches >= 3
 
 
@@ -759,3 +795,87 @@ def test_tile_kernel_matches_mma_sync_baseline(monkeypatch):
     monkeypatch.setenv("AGX_FORCE_MMA_SYNC", "1")
     b2 = DeviceBatch(w); b2.append(); c, _ = b2.attend()
     assert np.max(np.abs(a - c)) < 2e-2
+
+
+# ------------------------------------------------------------------ handle options
+@pytest.mark.parametrize("name,hq,hkv,P,q,env", [
+    ("warp-mma", 32, 8, [4096], [8], {}),
+    ("warp-mma batch", 32, 8, [700, 45, 2000, 16], [8, 3, 1, 16], {}),
+    ("stream", 32, 8, [9000, 8200], [8, 16], {}),
+    ("tile", 24, 8, [3072], [512], {}),
+    ("tile, prefix not page-aligned", 32, 8, [1003, 130], [200, 77], {}),
+])
+def test_early_prefix_loads_change_nothing(name, hq, hkv, P, q, env, monkeypatch):
+    """AGX_OPT_EARLY_PREFIX_LOADS only moves loads of cached-prefix pages in front of the dependency wait: with the
+    option on, a chain of (append, attention) pairs whose block rows change every round must give, bit for bit,
+    what the same chain gives with the option off - in the two-call form, where the rows read were written by
+    the launch directly in front, and in the fused form."""
+    w = W.make_attn_workload("early_" + name, 77, "bf16", hq, hkv, 128, P, q)
+    outs = {}
+    for early in (0, 1):
+        b = DeviceBatch(w)
+        b.h.set_option(agx.AGX_OPT_EARLY_PREFIX_LOADS, early)
+        g = torch.Generator(device="cuda"); g.manual_seed(5)
+        got = []
+        for it in range(6):
+            b.k_new.copy_(torch.randn(b.k_new.shape, generator=g, device="cuda").to(torch.bfloat16))
+            b.v_new.copy_(torch.randn(b.v_new.shape, generator=g, device="cuda").to(torch.bfloat16))
+            if it % 2 == 0:
+                b.append()
+                b.h.attn_prefixed(b.q_block, b.k_pool, b.v_pool, b.page_table, w.prefix_len, w.q_len, b.out, b.lse, b.ws)
+            else:
+                b.h.attn_prefixed_append(b.q_block, b.k_new, b.v_new, b.k_pool, b.v_pool, b.page_table, w.prefix_len,
+                                         w.q_len, b.out, b.lse, b.ws)
+            got.append(b.out.clone())
+        torch.cuda.synchronize()
+        assert b.status() == 0
+        outs[early] = got
+    for a, c in zip(outs[0], outs[1]):
+        assert torch.equal(a, c)
+    # and the last round against the oracle
+    w.k_new[:] = host_storage(b.k_new, "bf16"); w.v_new[:] = host_storage(b.v_new, "bf16")
+    kp, vp = oracle_pools_after_append(w)
+    ref, _ = oracle.attn_paged_batch(w.q_block, kp, vp, w.page_table, w.dtype, w.prefix_len, w.q_len, w.cu_q)
+    check_attention(outs[1][-1].to(torch.float64).cpu().numpy(), ref, name)
+
+
+@pytest.mark.parametrize("name,hq,hkv,P,q,stage,env", [
+    ("warp-mma kernel", 4, 1, [300], [8], 0, {}),
+    ("warp-mma kernel, later stage", 4, 1, [900], [4], 2, {"AGX_SMALL_MIN_SPLIT": "1024"}),      # one CTA per KV head, 8 stages
+    ("stream schedule", 4, 1, [500], [20], 0, {}),
+    ("stream schedule, later tile", 4, 1, [900], [20], 3, {"AGX_TILE_SPLIT_TOKENS": "1024"}),   # one split of 8 tiles
+    ("256-row schedule", 4, 1, [300], [100], 0, {}),
+    ("256-row schedule, later tile", 4, 1, [700], [100], 2, {"AGX_TILE_SPLIT_TOKENS": "1024"}),
+])
+def test_a_wait_that_runs_out_sets_the_status_and_leaves_the_handle_usable(name, hq, hkv, P, q, stage, env, monkeypatch):
+    """The give-up path of the bounded in-kernel waits.  With the wait limit cut to 2e5 clock ticks and the test
+    hook that makes the copy-issuing warp leave one K/V stage out (nothing is armed, nothing is copied - a flag that
+    nothing sets), the consumers' waits for that stage run out: the call returns, the device status carries
+    AGX_DEV_WAIT_TIMEOUT, and the next ordinary call on the same handle gives bit for bit what a fresh handle gives."""
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    w = W.make_attn_workload("timeout_" + name, 88, "bf16", hq, hkv, 128, P, q)
+    fresh = DeviceBatch(w); fresh.append(); fresh.attend()
+    assert fresh.status() == 0
+    b = DeviceBatch(w); b.append()
+    b.h.set_option(agx.AGX_OPT_WAIT_LIMIT_CYCLES, 200000)
+    b.h.set_option(agx.AGX_OPT_TEST_DROP_STAGE, stage)
+    b.attend()                                   # returns (synchronises) although a stage never arrived
+    assert b.status() & agx.AGX_DEV_WAIT_TIMEOUT
+    assert b.status() == 0                       # reading the status cleared it
+    b.h.set_option(agx.AGX_OPT_TEST_DROP_STAGE, -1)
+    b.h.set_option(agx.AGX_OPT_WAIT_LIMIT_CYCLES, 4000000000)
+    b.out.zero_()
+    b.attend()
+    assert b.status() == 0
+    assert torch.equal(b.out, fresh.out) and torch.equal(b.lse, fresh.lse)
+
+
+def test_set_option_rejects_what_it_does_not_know():
+    h = agx.Handle(32, 8, 128, "bf16")
+    with pytest.raises(agx.AgxError) as e:
+        h.set_option(99, 1)
+    assert e.value.status == -1
+    with pytest.raises(agx.AgxError) as e:
+        h.set_option(agx.AGX_OPT_WAIT_LIMIT_CYCLES, 10)
+    assert e.value.status == -2
