@@ -419,13 +419,19 @@ AGX_API agx_status agx_kv_import_pages(agx_handle* handle, void* k_pool, void* v
  *       that is not part of this library in between).  The block's own rows and Q are always read after the wait.
  *   AGX_OPT_WAIT_LIMIT_CYCLES (value >= 1000, default 4e9 ~ 2 s)
  *       Clock ticks after which an in-kernel wait gives up, sets AGX_DEV_WAIT_TIMEOUT and winds the CTA down.
+ *   AGX_OPT_ZERO_COPY (value = bits 0..3, default 3; environment AGX_ZERO_COPY sets the default)
+ *       Bit 0: kernels read small pinned, device-mapped host inputs (agx_verify_step_host*) and stored pages
+ *       (agx_kv_import_pages) across the bus themselves; cleared, every host buffer goes through copy-engine
+ *       transfers into device staging first.  Bit 1: the attention kernels write `out` straight into a pinned, mapped
+ *       host buffer.  Reading across the bus is the faster way for a call on an idle GPU; the copy engine is the
+ *       better one for an import that should run beside attention on another stream, since it needs no SM.
  *   AGX_OPT_TEST_DROP_STAGE (value = stage index, -1 = off, default -1)
  *       Test hook for the give-up path: the copy-issuing warp of every attention CTA leaves that K/V pipeline stage out
  *       (nothing is armed, nothing is copied), so the waits for it run out after the wait limit and the launch ends
  *       with AGX_DEV_WAIT_TIMEOUT.  Meant to be used with a short wait limit; results of such a launch are invalid.
  * Errors: AGX_E_INVAL (unknown option), AGX_E_RANGE.
  */
-enum { AGX_OPT_EARLY_PREFIX_LOADS = 1, AGX_OPT_WAIT_LIMIT_CYCLES = 2, AGX_OPT_TEST_DROP_STAGE = 3 };
+enum { AGX_OPT_EARLY_PREFIX_LOADS = 1, AGX_OPT_WAIT_LIMIT_CYCLES = 2, AGX_OPT_TEST_DROP_STAGE = 3, AGX_OPT_ZERO_COPY = 4 };
 AGX_API agx_status agx_set_option(agx_handle* handle, int32_t option, int64_t value);
 
 /* Number of kernels the last agx_attn_prefixed / agx_accept_greedy / agx_kv_append call on this

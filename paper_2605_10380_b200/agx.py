@@ -16,7 +16,7 @@ import numpy as np
 AGX_OK = 0
 AGX_BF16, AGX_F32 = 0, 1
 AGX_DEV_BAD_PAGE, AGX_DEV_WAIT_TIMEOUT, AGX_DEV_BAD_TOKEN = 1, 2, 4
-AGX_OPT_EARLY_PREFIX_LOADS, AGX_OPT_WAIT_LIMIT_CYCLES, AGX_OPT_TEST_DROP_STAGE = 1, 2, 3
+AGX_OPT_EARLY_PREFIX_LOADS, AGX_OPT_WAIT_LIMIT_CYCLES, AGX_OPT_TEST_DROP_STAGE, AGX_OPT_ZERO_COPY = 1, 2, 3, 4
 DTYPES = {"bf16": AGX_BF16, "f32": AGX_F32}
 
 _LIB_PATH = Path(__file__).resolve().parent / "lib" / "libagx.so"
@@ -332,6 +332,32 @@ class Handle:
         if n < 0:
             self._check(n, "agx_verify_step_host_workspace_bytes")
         return n
+
+    # -- agx_verify_step_host_enqueue with the arguments marshalled once
+    def verify_step_host_bind(self, k_pool, v_pool, page_table, h_prefix_len, h_q_len, h_q_block, h_k_new, h_v_new,
+                              h_logits, logits_dtype: str, row_stride: int, vocab: int, h_drafts, h_out, h_accept_len,
+                              h_next_token, h_seq_lens, workspace, stream=None):
+        """Marshal the arguments of ``agx_verify_step_host_enqueue`` once and return a function that makes the
+        call (a model that runs the same step over and over pays the conversion of two dozen arguments only
+        once).  The returned function keeps every buffer alive; it raises on a non-zero status."""
+        P, Q = _h_i32(h_prefix_len), _h_i32(h_q_len)
+        keep = (k_pool, v_pool, page_table, P, Q, h_q_block, h_k_new, h_v_new, h_logits, h_drafts, h_out, h_accept_len,
+                h_next_token, h_seq_lens, workspace)
+        vp = ctypes.c_void_p
+        args = (self._h, vp(_ptr(k_pool)), vp(_ptr(v_pool)), ctypes.c_int64(int(k_pool.shape[0])),
+                vp(_ptr(page_table)), ctypes.c_int32(int(page_table.shape[1])), vp(_ptr(P)), vp(_ptr(Q)),
+                ctypes.c_int32(int(P.shape[0])), vp(_ptr(h_q_block)), vp(_ptr(h_k_new)), vp(_ptr(h_v_new)),
+                vp(_ptr(h_logits)), ctypes.c_int32(DTYPES[logits_dtype]), ctypes.c_int64(int(row_stride)), ctypes.c_int32(int(vocab)),
+                vp(_ptr(h_drafts)), vp(_ptr(h_out)), vp(_ptr(h_accept_len)), vp(_ptr(h_next_token)),
+                vp(_ptr(h_seq_lens)), vp(_ptr(workspace)), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
+                vp(_stream_ptr(stream)))
+        fn = self._lib.agx_verify_step_host_enqueue
+
+        def call(_keep=keep):
+            st = fn(*args)
+            if st != AGX_OK:
+                self._check(st, "agx_verify_step_host_enqueue")
+        return call
 
     # -- agx_verify_step_host (host tensors: pinned torch tensors or numpy arrays)
     def verify_step_host(self, k_pool, v_pool, page_table, h_prefix_len, h_q_len, h_q_block, h_k_new, h_v_new,

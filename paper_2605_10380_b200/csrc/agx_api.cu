@@ -587,6 +587,10 @@ agx_status agx_set_option(agx_handle* h, int32_t option, int64_t value) {
             if (value < 1000) return fail(h, AGX_E_RANGE, "wait limit below 1000 cycles");
             h->wait_limit_cycles = value;
             return AGX_OK;
+        case AGX_OPT_ZERO_COPY:
+            if (value < 0 || value > 3) return fail(h, AGX_E_RANGE, "zero-copy bits");
+            h->zero_copy = (int)value;
+            return AGX_OK;
         case AGX_OPT_TEST_DROP_STAGE:
             if (value < -1 || value > 0x7FFFFFFF) return fail(h, AGX_E_RANGE, "stage index");
             h->drop_stage = (int)value;
