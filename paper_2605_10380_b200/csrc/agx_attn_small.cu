@@ -696,6 +696,82 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
     if (p.lse && lane == 0) p.lse[(long long)(sp.q_row0 + i) * p.hq + h] = (m_all + log2f(l_all)) * 0.6931471805599453f;
 }
 
+// The same merge for the partials of the 256-row tensor-core schedule (fp16 rows divided by their own sums, at most 4
+// splits): one wave of CTAs, each warp taking up to three (row, head) pairs with all their loads in flight at once, so
+// that the merge of a split prefill (12288 pairs, 9 MB of partials) is one memory round trip per warp instead of
+// several waves of short-lived CTAs.
+constexpr int kCombineRows = 3;
+__global__ void __launch_bounds__(128, 8)
+attn_combine_half4_kernel(const __grid_constant__ AttnParams p, int total_rows) {
+    pdl_launch_dependents();
+    const int lane = threadIdx.x & 31;
+    const int n_pairs = total_rows * p.hq;
+    const int stride = gridDim.x * 4;
+    const int rh0 = blockIdx.x * 4 + (threadIdx.x >> 5);
+    long long e0[kCombineRows], out_off[kCombineRows];
+    int ns[kCombineRows];
+#pragma unroll
+    for (int j = 0; j < kCombineRows; ++j) {
+        const int rh = rh0 + j * stride;
+        ns[j] = 0; e0[j] = 0; out_off[j] = 0;
+        if (rh < n_pairs) {
+            const int lrow = rh / p.hq, h = rh - lrow * p.hq;
+            int si = 0, acc_rows = 0;
+#pragma unroll 1
+            for (int s = 0; s < p.num_seqs; ++s) {
+                if (lrow >= acc_rows && lrow < acc_rows + p.seq[s].q_len) { si = s; break; }
+                acc_rows += p.seq[s].q_len;
+            }
+            const SeqPlan& sp = p.seq[si];
+            if (sp.nsplit > 1) {   // (a single split was written directly by the attention kernel)
+                const int i = lrow - acc_rows;
+                ns[j] = sp.nsplit;
+                e0[j] = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit;
+                out_off[j] = (long long)(sp.q_row0 + i) * p.hq + h;
+            }
+        }
+    }
+    pdl_wait();   // the partials are complete
+    float2 ml[kCombineRows];
+    uint2 v[kCombineRows][4];
+#pragma unroll
+    for (int j = 0; j < kCombineRows; ++j) {
+        ml[j] = (lane < ns[j]) ? __ldcg(p.part_ml + e0[j] + lane) : make_float2(-INFINITY, 0.f);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (k < ns[j]) v[j][k] = __ldcg((const uint2*)((const unsigned char*)p.part_o + (e0[j] + k) * 512 + lane * 8));
+    }
+#pragma unroll
+    for (int j = 0; j < kCombineRows; ++j) {
+        if (ns[j] == 0) continue;   // (uniform over the warp)
+        float m_all = ml[j].x;
+#pragma unroll
+        for (int off = 2; off > 0; off >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, off));   // splits sit in lanes 0..3
+        const float w_mine = (ml[j].x == -INFINITY) ? 0.f : exp2f(ml[j].x - m_all) * ml[j].y;
+        float l_all = w_mine;
+#pragma unroll
+        for (int off = 2; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xFFFFFFFFu, l_all, off);
+        m_all = __shfl_sync(0xFFFFFFFFu, m_all, 0);
+        l_all = __shfl_sync(0xFFFFFFFFu, l_all, 0);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float w = __shfl_sync(0xFFFFFFFFu, w_mine, k);
+            if (k < ns[j] && w != 0.f) {   // a split that saw no token for this row publishes only (m, l) = (-inf, 0)
+                const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&v[j][k].x));
+                const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&v[j][k].y));
+                acc.x += a.x * w; acc.y += a.y * w; acc.z += b.x * w; acc.w += b.y * w;
+            }
+        }
+        const float inv = 1.f / l_all;
+        uint2 packed;
+        packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+        packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+        *(uint2*)((__nv_bfloat16*)p.out + out_off[j] * kD + lane * 4) = packed;
+        if (p.lse && lane == 0) p.lse[out_off[j]] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+    }
+}
+
 // --------------------------------------------------------------------------------------------
 namespace {
 template <int MT, int KW, int NS>
@@ -791,7 +867,14 @@ cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, 
     int ns_max = 1;
     for (int i = 0; i < p.num_seqs; ++i) ns_max = p.seq[i].nsplit > ns_max ? p.seq[i].nsplit : ns_max;
     if (dtype == AGX_BF16 && p.part_half) {
-        if (ns_max <= 4) return launch_chained(attn_combine_kernel<true, 4, true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+        if (ns_max <= 4) {
+            int device = 0, sms = 0;
+            if (cudaGetDevice(&device) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+                return cudaErrorInvalidDevice;
+            const int one_wave = sms * 8;
+            const int want = (int)((n + 4 * kCombineRows - 1) / (4 * kCombineRows));   // CTAs whose warps take kCombineRows pairs each
+            return launch_chained(attn_combine_half4_kernel, dim3(want > one_wave ? blocks : (want > 0 ? want : 1)), dim3(128), 0, stream, p, total_rows);
+        }
         if (ns_max <= 16) return launch_chained(attn_combine_kernel<true, 16, true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
         return launch_chained(attn_combine_kernel<true, 1 << 30, true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
     }
