@@ -36,6 +36,7 @@ struct agx_handle {
     int batch_stream_tokens; // total tokens of a batch's small blocks from which they all take the stream schedule (env AGX_BATCH_STREAM_TOKENS)
     bool cluster_merge;     // KV splits of the small-q kernel merged inside thread-block clusters where the batch allows (env AGX_CLUSTER_MERGE=0 turns it off)
     int zero_copy;          // host steps: bit 0 = kernels read small pinned inputs, bit 1 = kernels write `out` into a pinned buffer (env AGX_ZERO_COPY, default 3)
+    int stream_max_rows;    // blocks of up to this many rows per KV head may take the one-Q-tile schedule in 128-row chunks (env AGX_STREAM_MAX_ROWS)
     int stream_min_tokens;  // context length from which blocks of <= 32 rows take the tensor-core stream schedule (env AGX_STREAM_MIN_TOKENS; -1 = by block height)
     long long wait_limit_cycles;   // AGX_OPT_WAIT_LIMIT_CYCLES
     int early_prefix;       // AGX_OPT_EARLY_PREFIX_LOADS
@@ -139,7 +140,7 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
             // kernel, whose fixed costs are lower (none above 32 rows)
             // cross-over of a single sequence (GQA 32/8): q = 8 near 7k tokens, q = 1 near 10k
             const int cross = h->stream_min_tokens >= 0 ? h->stream_min_tokens : (rows > 8 ? 7168 : 10240);
-            if (tile_ok && rows <= 128 && (rows > 32 || batch_streams || P[s] + Q[s] >= cross)) k = KIND_STREAM;
+            if (tile_ok && rows <= h->stream_max_rows && (rows > 32 || batch_streams || P[s] + Q[s] >= cross)) k = KIND_STREAM;
             else if (rows <= 16) k = KIND_SMALL1;
             else if (rows <= 32) k = KIND_SMALL2;
             else if (rows <= kSmallRowsMax || h->force_mma_sync) k = KIND_SMALL4;
@@ -335,6 +336,8 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     h->force_mma_sync = env ? atoi(env) : 0;
     env = getenv("AGX_STREAM_MIN_TOKENS");
     h->stream_min_tokens = env ? atoi(env) : -1;   // -1: the measured cross-over, by block height
+    env = getenv("AGX_STREAM_MAX_ROWS");
+    h->stream_max_rows = env ? atoi(env) : 384;
     env = getenv("AGX_CLUSTER_MERGE");
     h->cluster_merge = !(env && atoi(env) == 0);
     env = getenv("AGX_ZERO_COPY");

@@ -684,6 +684,21 @@ def test_stream_schedule_shapes(P, q, hq, hkv, monkeypatch):
     run_and_check(w, sample=(13, 64) if P > 6000 else None, poison=True)
 
 
+@pytest.mark.parametrize("P,q,hq,hkv", [
+    (700, 80, 32, 8),      # 320 rows per KV head: three 128-row chunks, the last half empty
+    (100, 90, 6, 2),       # G = 3, 270 rows, prefix not page-aligned
+    (1500, 33, 32, 8),     # 132 rows: a second chunk of 4 rows
+    (0, 96, 16, 4),        # pure causal block of 384 rows: chunks that see nothing of the later KV splits
+])
+def test_stream_schedule_with_several_row_chunks(P, q, hq, hkv):
+    """Blocks of 129..384 rows per KV head take the one-Q-tile schedule in 128-row chunks (short suffixes over short
+    prefixes, where its lower fixed costs beat the 256-row schedule): every output row against the oracle, in the
+    two-call and in the fused form."""
+    w = W.make_attn_workload(f"chunks_{P}_{q}", 3000 + P + q, "bf16", hq, hkv, 128, [P], [q], spare_pages=2)
+    run_and_check(w, poison=True)
+    run_and_check(w, poison=True, fused=True)
+
+
 def test_stream_schedule_ragged_batch_matches_warp_mma_kernel(monkeypatch):
     P = [2048, 2100, 4000, 2048 + 15, 9000, 2500, 3001, 2048]
     q = [1, 2, 4, 8, 16, 3, 5, 30]
