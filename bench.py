@@ -914,22 +914,85 @@ def oracle_c1(W):
 
 ONLY = {  # name: (P list, q list, Hq, layers)
     "c2": ([4096], [8], 32, 4),
+    "c2q1": ([4096], [1], 32, 4),
     "c3": ([3072], [512], 24, 1),
+    "c4v": None, "c4p": None,   # the verify / prefill half of the ragged mixed batch (filled in at run time)
     "c5v": ([32768] * 4, [8] * 4, 32, 1),
     "c5p": ([30720], [2048], 32, 1),
     "c5p_small": ([7680], [1024], 32, 1),
-    "m128": ([1000], [128], 32, 2),
+    "b4": ([4096] * 4, [8] * 4, 32, 2),     # four verify blocks: KV splits merged inside thread-block clusters
+    "m80": ([700], [80], 32, 2), "m128": ([1000], [128], 32, 2), "m200": ([1500], [200], 32, 2),
+    "accept8": None, "append512": None, "ngram": None,   # the other kernels of the library
+    "step": None,                                         # the headline step itself, eagerly: the launch list of one step
 }
 
 
 def run_only(args):
-    """Profiling aid: eager (no graph) attention calls of ONE workload, a few launches, one line out."""
+    """Profiling aid: eager (no graph) calls of ONE workload, a few launches, one line out."""
     import torch
     torch.cuda.set_device(0)
     from paper_2605_10380_b200 import agx
     from paper_2605_10380_b200 import workloads as W
-    P, q, hq, layers = ONLY[args.only]
-    lv = LayeredVerify(torch, agx, W, P, q, hq, HKV, D, layers, 0, 7)
+    name = args.only
+    if name == "step":
+        cfg = configs(W)[HEADLINE]
+        lv = LayeredVerify(torch, agx, W, cfg["P"], cfg["q"], cfg["hq"], HKV, D, cfg["layers"], VOCAB, cfg["seed"],
+                           verify=cfg["verify"], shared=cfg["shared"])
+        for _ in range(args.warmup):
+            n = lv.step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            n = lv.step()
+        e1.record()
+        torch.cuda.synchronize()
+        assert lv.h.get_status() == 0
+        print(json.dumps({"only": name, "ms_per_step_eager": e0.elapsed_time(e1) / args.steps, "launches_per_step": n}))
+        return
+    if name in ("accept8", "append512", "ngram"):
+        h = agx.Handle(32, 8, 128, "bf16")
+        if name == "accept8":
+            aw = W.make_planted_accept("only_accept", 9, "bf16", VOCAB, [8], [4096])
+            logits = [torch.from_numpy(aw.logits).cuda().view(torch.bfloat16).clone() for _ in range(3)]
+            drafts = torch.from_numpy(aw.drafts).cuda(); cu = torch.from_numpy(aw.cu_q).cuda()
+            al = torch.zeros(1, dtype=torch.int32, device="cuda"); nt = torch.zeros(1, dtype=torch.int32, device="cuda")
+            ws = torch.empty(h.accept_workspace_bytes(8, VOCAB), dtype=torch.uint8, device="cuda")
+            fn = lambda i: h.accept_greedy(logits[i % 3], "bf16", VOCAB, drafts, cu, al, nt, None, None, ws)
+        elif name == "append512":
+            lv = LayeredVerify(torch, agx, W, [3072], [512], 24, HKV, D, 3, 0, 13)
+            fn = lambda i: lv.h.kv_append(lv.k_pools[i % 3], lv.v_pools[i % 3], lv.k_new[i % 3], lv.v_new[i % 3], lv.page_table,
+                                          lv.prefix_dev, lv.cu_dev)
+        else:
+            rng = np.random.default_rng(17)
+            toks = torch.from_numpy(rng.integers(0, 2048, 4096).astype(np.int32)).cuda()
+            lut = torch.empty(agx.ngram_lut_bytes(4096), dtype=torch.uint8, device="cuda")
+            nws = torch.empty(agx.ngram_workspace_bytes(4096), dtype=torch.uint8, device="cuda")
+            ctx = toks[100:102].reshape(1, 2).contiguous(); fill = torch.zeros((1, 4), dtype=torch.int32, device="cuda")
+            dr = torch.zeros((1, 4), dtype=torch.int32, device="cuda"); hd = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+            def fn(i):
+                h.ngram_build(toks, 3, lut, nws)
+                h.ngram_draft(lut, ctx, fill, 4, dr, hd)
+        for i in range(args.warmup):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.steps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        assert h.get_status() == 0
+        print(json.dumps({"only": name, "ms_per_call_eager": e0.elapsed_time(e1) / args.steps}))
+        return
+    if name in ("c4v", "c4p"):
+        P4, q4 = W.c4_lengths()
+        idx = range(8) if name == "c4v" else range(8, 16)
+        P, q, hq, layers, shared = [int(P4[s]) for s in idx], [int(q4[s]) for s in idx], 32, 1, 2048
+    else:
+        (P, q, hq, layers), shared = ONLY[name], 0
+    lv = LayeredVerify(torch, agx, W, P, q, hq, HKV, D, layers, 0, 7, shared=shared)
     for _ in range(args.warmup):
         for l in range(layers):
             lv.attn_layer(l)
@@ -943,7 +1006,7 @@ def run_only(args):
     torch.cuda.synchronize()
     assert lv.h.get_status() == 0
     ms = e0.elapsed_time(e1) / (args.steps * layers)
-    print(json.dumps({"only": args.only, "ms_per_call_eager": ms, "bytes": lv.bytes_per_layer(),
+    print(json.dumps({"only": name, "ms_per_call_eager": ms, "bytes": lv.bytes_per_layer(),
                       "flops": lv.flops_per_layer(), "GBps": lv.bytes_per_layer() / ms / 1e6,
                       "TFLOPs": lv.flops_per_layer() / ms / 1e9}))
 

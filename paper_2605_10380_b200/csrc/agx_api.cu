@@ -9,9 +9,17 @@
 #include <unordered_map>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "agx_internal.cuh"
 
 namespace {
+// An NVTX range around every call that enqueues work: a timeline tool shows the library's calls by name; with no tool
+// attached a range costs a few nanoseconds.
+struct CallRange {
+    explicit CallRange(const char* name) { nvtxRangePushA(name); }
+    ~CallRange() { nvtxRangePop(); }
+};
 struct Plan;
 // TMA view of one KV pool, kept per pool address: encoding a tensor map costs about as much host time as a launch.
 struct PoolMap {
@@ -377,6 +385,7 @@ agx_status agx_destroy(agx_handle* h) {
 agx_status agx_kv_append(agx_handle* h, void* k_pool, void* v_pool, int64_t num_pages, const void* k_new,
                          const void* v_new, const int32_t* page_table, int32_t pt_stride, const int32_t* prefix_len,
                          const int32_t* cu_q, int32_t B, int32_t total_q, void* stream) {
+    CallRange range_("agx_kv_append");
     if (!h) return AGX_E_INVAL;
     h->last_launches = 0;
     if (B < 0 || total_q < 0) return fail(h, AGX_E_INVAL, "negative B or total_q");
@@ -414,6 +423,7 @@ static agx_status attn_impl(agx_handle* h, const void* q_block, const void* k_ne
                             const void* v_pool, int64_t num_pages, const int32_t* page_table, int32_t pt_stride,
                             const int32_t* P, const int32_t* Q, int32_t B, void* out, float* lse, void* workspace,
                             size_t workspace_bytes, void* stream_v) {
+    CallRange range_("agx_attn_prefixed");
     if (!h) return AGX_E_INVAL;
     h->last_launches = 0;
     if (B < 0) return fail(h, AGX_E_INVAL, "negative B");
@@ -541,6 +551,7 @@ agx_status agx_accept_greedy(agx_handle* h, const void* logits, int32_t logits_d
                              int32_t vocab, const int32_t* drafts, const int32_t* cu_q, int32_t B, int32_t total_q,
                              int32_t* accept_len, int32_t* next_token, int32_t* argmax, int32_t* seq_lens,
                              void* workspace, size_t workspace_bytes, void* stream) {
+    CallRange range_("agx_accept_greedy");
     if (!h) return AGX_E_INVAL;
     h->last_launches = 0;
     if (B < 0 || total_q < 0) return fail(h, AGX_E_INVAL, "negative B or total_q");
@@ -677,6 +688,7 @@ static agx_status verify_step_host_impl(agx_handle* h, void* k_pool, void* v_poo
                                 int32_t logits_dtype, int64_t row_stride, int32_t vocab, const int32_t* h_drafts,
                                 void* h_out, int32_t* h_accept, int32_t* h_next, int32_t* h_seq_lens, void* workspace,
                                 size_t workspace_bytes, void* stream_v, bool sync) {
+    CallRange range_("agx_verify_step_host");
     if (!h) return AGX_E_INVAL;
     HostStepLayout L;
     agx_status st = host_step_layout(h, B, P, Q, logits_dtype, row_stride, vocab, L);
@@ -797,6 +809,7 @@ int64_t agx_ngram_workspace_bytes(int32_t stream_tokens) {
 
 agx_status agx_ngram_build(agx_handle* h, const int32_t* stream_tokens, int32_t num_tokens, int32_t n, void* lut,
                            size_t lut_bytes, void* workspace, size_t workspace_bytes, void* stream) {
+    CallRange range_("agx_ngram_build");
     if (!h) return AGX_E_INVAL;
     h->last_launches = 0;
     if (n != 2 && n != 3) return fail(h, AGX_E_UNSUPPORTED, "n-gram order %d (2 and 3 are built)", n);
@@ -815,6 +828,7 @@ agx_status agx_ngram_build(agx_handle* h, const int32_t* stream_tokens, int32_t 
 
 agx_status agx_ngram_draft(agx_handle* h, const void* lut, const int32_t* context, const int32_t* fill, int32_t B, int32_t k,
                            int32_t* drafts, int32_t* has_draft, void* stream) {
+    CallRange range_("agx_ngram_draft");
     if (!h) return AGX_E_INVAL;
     h->last_launches = 0;
     if (B < 0 || k < 0) return fail(h, AGX_E_INVAL, "negative B or k");
@@ -828,6 +842,7 @@ agx_status agx_ngram_draft(agx_handle* h, const void* lut, const int32_t* contex
 
 agx_status agx_kv_copy_pages(agx_handle* h, void* k_pool, void* v_pool, int64_t num_pages, const int32_t* src,
                              const int32_t* dst, int32_t count, void* stream) {
+    CallRange range_("agx_kv_copy_pages");
     if (!h) return AGX_E_INVAL;
     h->last_launches = 0;
     if (count < 0) return fail(h, AGX_E_INVAL, "negative count");
@@ -848,6 +863,7 @@ int64_t agx_kv_import_staging_bytes(const agx_handle* h, int32_t count) {
 
 agx_status agx_kv_import_pages(agx_handle* h, void* k_pool, void* v_pool, int64_t num_pages, const void* h_k, const void* h_v,
                                const int32_t* dst_pages, int32_t count, void* staging, size_t staging_bytes, void* stream_v) {
+    CallRange range_("agx_kv_import_pages");
     if (!h) return AGX_E_INVAL;
     h->last_launches = 0;
     if (count < 0) return fail(h, AGX_E_INVAL, "negative count");
