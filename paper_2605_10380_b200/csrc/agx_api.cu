@@ -194,14 +194,23 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
             return items;
         };
         if (k == KIND_TILE || k == KIND_STREAM) {
-            // several waves are fine here: pick the split length with the smallest estimated makespan,
-            // waves * (tiles per item + fixed per-CTA cost of ~3 tiles)
+            // several waves are fine here: pick the split length with the smallest estimated makespan, in units of one KV
+            // tile's time (~1.6 us): waves * (tiles per item + fixed per-CTA cost of ~3 tiles), plus what the split costs
+            // afterwards: the merge launch (~2 units) and the partial rows written and read back (~0.3 units per MB;
+            // measured on a ragged batch of eight suffix prefills: 95 MB of partials cost 60 us more than 22 MB)
             int max_len = 0;
             for (int s : seqs) max_len = std::max(max_len, P[s] + Q[s]);
+            const long long row_bytes = k == KIND_TILE ? 256 : 520;   // fp16 row | fp32 row + (m, l)
             long long best_cost = -1;
             for (int c_tokens = min_split; c_tokens < max_len + unit; c_tokens += unit) {
                 const long long waves = (count_items(c_tokens) + h->sm_count - 1) / h->sm_count;
-                const long long cost = waves * (std::min(c_tokens, round_up(max_len, unit)) / unit + 3);
+                long long part_bytes = 0;
+                for (int s : seqs) {
+                    const long long ns = (P[s] + Q[s] + c_tokens - 1) / c_tokens;
+                    if (ns > 1) part_bytes += (long long)Q[s] * c.num_q_heads * ns * row_bytes;
+                }
+                const long long cost = 16 * waves * (std::min(c_tokens, round_up(max_len, unit)) / unit + 3) +
+                                       (part_bytes ? 32 + 5 * (part_bytes >> 20) : 0);
                 if (best_cost < 0 || cost < best_cost) { best_cost = cost; C = c_tokens; }
             }
             if (const char* force = getenv("AGX_TILE_SPLIT_TOKENS")) { if (atoi(force) >= unit) C = atoi(force) / unit * unit; }
