@@ -74,7 +74,7 @@ enum {
 typedef struct agx_config {
     int32_t num_q_heads;  /* Hq */
     int32_t num_kv_heads; /* Hkv, divides Hq */
-    int32_t head_dim;     /* d: 64 or 128 for AGX_F32, 128 for AGX_BF16 */
+    int32_t head_dim;     /* d: 64 or 128 (AGX_BF16 with 64 and AGX_F32 run a scalar fp32 kernel: a correctness path) */
     int32_t page_size;    /* must be 16 */
     int32_t dtype;        /* AGX_BF16 or AGX_F32 */
     float scale;          /* softmax scale; 0 selects 1/sqrt(head_dim) */
@@ -132,7 +132,7 @@ AGX_API int64_t agx_attn_workspace_bytes(agx_handle* handle, int32_t B, const in
  *                  scaled scores
  *   workspace    : device, >= agx_attn_workspace_bytes(...) bytes, 256-byte aligned (may be NULL
  *                  when that figure is 0)
- * Dispatch (G = num_q_heads / num_kv_heads): up to 32 query rows per KV head (q_len * G) over a context
+ * Dispatch (G = num_q_heads / num_kv_heads; bf16 handles with head_dim 128 - other handles run the scalar kernel): up to 32 query rows per KV head (q_len * G) over a context
  * shorter than about 7k tokens (10k for q_len * G <= 8) run the split-KV warp-MMA kernel (latency-bound); up to 32 rows over a
  * longer context, or 33..128 rows over any context, run the tensor-core kernel with one padded Q tile
  * whose KV tiles alternate between two softmax warpgroups (HBM-bound); longer blocks run the

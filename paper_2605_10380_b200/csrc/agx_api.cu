@@ -129,7 +129,8 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
     // cross-over (stream_min_tokens).
     long long small_tokens = 0;
     int small_seqs = 0;
-    if (c.dtype != AGX_F32)
+    const bool scalar_path = c.dtype == AGX_F32 || c.head_dim != 128;   // fp32 pools, and bf16 with head_dim 64
+    if (!scalar_path)
         for (int s = 0; s < B; ++s)
             if (Q[s] * G <= 32) { small_tokens += P[s] + Q[s]; ++small_seqs; }
     small_tokens = small_tokens * c.num_kv_heads / 8;   // the thresholds were measured with 8 KV heads: scale to the same bytes
@@ -139,7 +140,7 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
     std::vector<int> groups[KIND_COUNT];
     for (int s = 0; s < B; ++s) {
         Kind k;
-        if (c.dtype == AGX_F32) k = KIND_SIMT;
+        if (scalar_path) k = KIND_SIMT;
         else {
             const int rows = Q[s] * G;
             const bool tile_ok = !h->force_mma_sync;
@@ -338,7 +339,7 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     if (cfg->num_q_heads < 1 || cfg->num_kv_heads < 1 || cfg->num_q_heads % cfg->num_kv_heads != 0) return AGX_E_INVAL;
     if (cfg->page_size != kPage) return AGX_E_UNSUPPORTED;
     if (cfg->dtype != AGX_BF16 && cfg->dtype != AGX_F32) return AGX_E_UNSUPPORTED;
-    if (cfg->dtype == AGX_BF16 && cfg->head_dim != 128) return AGX_E_UNSUPPORTED;
+    if (cfg->dtype == AGX_BF16 && cfg->head_dim != 128 && cfg->head_dim != 64) return AGX_E_UNSUPPORTED;
     if (cfg->dtype == AGX_F32 && cfg->head_dim != 64 && cfg->head_dim != 128) return AGX_E_UNSUPPORTED;
     if (!(cfg->scale >= 0.f)) return AGX_E_INVAL;
     agx_handle* h = new (std::nothrow) agx_handle();
@@ -470,7 +471,7 @@ static agx_status attn_impl(agx_handle* h, const void* q_block, const void* k_ne
     p.early_prefix = h->early_prefix;
     p.drop_stage = h->drop_stage;
     const CUtensorMap *map_k = nullptr, *map_v = nullptr;
-    if (h->cfg.dtype == AGX_BF16) {
+    if (h->cfg.dtype == AGX_BF16 && h->cfg.head_dim == 128) {
         if ((long long)num_pages * p.hkv * kPage > 0x7FFFFFFFll) return fail(h, AGX_E_RANGE, "pool too large for one tensor map");
         map_k = pool_map(h, k_pool, num_pages, p.hkv);
         map_v = pool_map(h, v_pool, num_pages, p.hkv);
@@ -503,7 +504,7 @@ static agx_status attn_impl(agx_handle* h, const void* q_block, const void* k_ne
             case KIND_SMALL1: e = launch_attn_small_bf16(p, 1, ln.kw, *map_k, *map_v, stream); break;
             case KIND_SMALL2: e = launch_attn_small_bf16(p, 2, ln.kw, *map_k, *map_v, stream); break;
             case KIND_SMALL4: e = launch_attn_small_bf16(p, 4, 4, *map_k, *map_v, stream); break;
-            case KIND_SIMT: e = launch_attn_simt_f32(p, stream); break;
+            case KIND_SIMT: e = launch_attn_simt(p, h->cfg.dtype, stream); break;
             case KIND_TILE: e = launch_attn_tile_bf16(p, false, *map_k, *map_v, stream); break;
             case KIND_STREAM: e = launch_attn_tile_bf16(p, true, *map_k, *map_v, stream); break;
             default: return fail(h, AGX_E_UNSUPPORTED, "unknown kernel kind");

@@ -485,11 +485,17 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
 }
 
 // --------------------------------------------------------------------------------------------
-// Scalar kernel for fp32 pools (any q; d = 64 or 128).  CTA = 4 warps on one (sequence, row, head,
-// split); a warp takes every 4th token, lanes split the head dim, dot products reduce by shuffle.
-template <int D>
+// Scalar kernel for fp32 pools (any q; d = 64 or 128) and for bf16 pools with d = 64 (a correctness path: fp32 arithmetic
+// on the FMA pipes).  CTA = 4 warps on one (sequence, row, head, split); a warp takes every 4th token, lanes split the head
+// dim, dot products reduce by shuffle.
+template <bool kBf16>
+__device__ __forceinline__ float load_elem(const void* base, long long idx) {
+    if (kBf16) return __bfloat162float(((const __nv_bfloat16*)base)[idx]);
+    return ((const float*)base)[idx];
+}
+template <int D, bool kBf16>
 __global__ void __launch_bounds__(128)
-attn_simt_f32_kernel(const __grid_constant__ AttnParams p) {
+attn_simt_kernel(const __grid_constant__ AttnParams p) {
     constexpr int kPer = D / 32;
     pdl_launch_dependents();
     pdl_wait();
@@ -506,13 +512,11 @@ attn_simt_f32_kernel(const __grid_constant__ AttnParams p) {
     const int tok_begin = split * sp.split_tokens;
     const int tok_end = min(sp.prefix_len + i + 1, tok_begin + sp.split_tokens);  // causal limit for row i
     const int* pt_row = p.page_table + (long long)sp.seq_index * p.pt_stride;
-    const float* kp = (const float*)p.k_pool;
-    const float* vp = (const float*)p.v_pool;
 
     float qv[kPer], acc[kPer];
-    const float* qrow = (const float*)p.q + ((long long)(sp.q_row0 + i) * p.hq + h) * D;
+    const long long q0 = ((long long)(sp.q_row0 + i) * p.hq + h) * D;
 #pragma unroll
-    for (int c = 0; c < kPer; ++c) { qv[c] = qrow[lane + 32 * c] * p.scale_log2; acc[c] = 0.f; }
+    for (int c = 0; c < kPer; ++c) { qv[c] = load_elem<kBf16>(p.q, q0 + lane + 32 * c) * p.scale_log2; acc[c] = 0.f; }
     float m = -INFINITY, l = 0.f;
     for (int tok = tok_begin + warp; tok < tok_end; tok += 4) {
         long long page = __ldg(pt_row + (tok >> 4));
@@ -523,7 +527,7 @@ attn_simt_f32_kernel(const __grid_constant__ AttnParams p) {
         const long long base = ((page * p.hkv + g) * kPage + (tok & 15)) * (long long)D;
         float dot = 0.f;
 #pragma unroll
-        for (int c = 0; c < kPer; ++c) dot += qv[c] * kp[base + lane + 32 * c];
+        for (int c = 0; c < kPer; ++c) dot += qv[c] * load_elem<kBf16>(p.k_pool, base + lane + 32 * c);
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, off);
         const float m_new = fmaxf(m, dot);
@@ -531,7 +535,7 @@ attn_simt_f32_kernel(const __grid_constant__ AttnParams p) {
         const float w = exp2f(dot - m_new);
         l = l * corr + w;
 #pragma unroll
-        for (int c = 0; c < kPer; ++c) acc[c] = acc[c] * corr + w * vp[base + lane + 32 * c];
+        for (int c = 0; c < kPer; ++c) acc[c] = acc[c] * corr + w * load_elem<kBf16>(p.v_pool, base + lane + 32 * c);
         m = m_new;
     }
     __shared__ float sm_o[4][D];
@@ -552,7 +556,9 @@ attn_simt_f32_kernel(const __grid_constant__ AttnParams p) {
             a += sm_o[k][c] * w;
         }
         if (sp.nsplit == 1) {
-            ((float*)p.out)[((long long)(sp.q_row0 + i) * p.hq + h) * D + c] = a / l_all;
+            const long long o = ((long long)(sp.q_row0 + i) * p.hq + h) * D + c;
+            if (kBf16) ((__nv_bfloat16*)p.out)[o] = __float2bfloat16_rn(a / l_all);
+            else ((float*)p.out)[o] = a / l_all;
             if (p.lse && c == 0) p.lse[(long long)(sp.q_row0 + i) * p.hq + h] = (m_all + log2f(l_all)) * 0.6931471805599453f;
         } else {
             const long long e = (long long)sp.part_base + ((long long)i * p.hq + h) * sp.nsplit + split;
@@ -853,10 +859,11 @@ cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, int kw, const CU
     }
 }
 
-cudaError_t launch_attn_simt_f32(const AttnParams& p, cudaStream_t stream) {
+cudaError_t launch_attn_simt(const AttnParams& p, int dtype, cudaStream_t stream) {
     if (p.num_items == 0) return cudaSuccess;
-    if (p.head_dim == 64) return launch_chained(attn_simt_f32_kernel<64>, dim3(p.num_items), dim3(128), 0, stream, p);
-    if (p.head_dim == 128) return launch_chained(attn_simt_f32_kernel<128>, dim3(p.num_items), dim3(128), 0, stream, p);
+    if (dtype == AGX_F32 && p.head_dim == 64) return launch_chained(attn_simt_kernel<64, false>, dim3(p.num_items), dim3(128), 0, stream, p);
+    if (dtype == AGX_F32 && p.head_dim == 128) return launch_chained(attn_simt_kernel<128, false>, dim3(p.num_items), dim3(128), 0, stream, p);
+    if (dtype == AGX_BF16 && p.head_dim == 64) return launch_chained(attn_simt_kernel<64, true>, dim3(p.num_items), dim3(128), 0, stream, p);
     return cudaErrorInvalidValue;
 }
 

@@ -123,8 +123,8 @@ cudaError_t launch_kv_append(int dtype, void* k_pool, void* v_pool, long long nu
 int attn_small_max_clusters(int mt, int kw, int cluster);
 cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, int kw, const CUtensorMap& map_k, const CUtensorMap& map_v,
                                    cudaStream_t stream);
-// Scalar fp32-math kernel for AGX_F32 pools (any q, d in {64, 128}).
-cudaError_t launch_attn_simt_f32(const AttnParams& p, cudaStream_t stream);
+// Scalar fp32-math kernel for AGX_F32 pools (any q, d in {64, 128}) and for AGX_BF16 pools with d = 64.
+cudaError_t launch_attn_simt(const AttnParams& p, int dtype, cudaStream_t stream);
 // Merge of split partials into out / lse.
 cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, cudaStream_t stream);   // honours p.part_half
 

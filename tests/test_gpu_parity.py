@@ -88,6 +88,16 @@ def test_c1_tiny_verify_bf16_rounded_inputs_d128():
     run_and_check(w)
 
 
+def test_c1_tiny_verify_bf16_head_dim_64():
+    """The tiny configuration's own shape (4/2 heads, d = 64, P = 256, q = 4) with bf16 storage, and two more shapes of
+    the scalar kernel that serves bf16 pools with head_dim 64: every output row, both call forms."""
+    w = W.make_attn_workload("c1_bf16_d64", 1, "bf16", 4, 2, 64, [256], [4], spare_pages=47)
+    run_and_check(w, strict=True)
+    w2 = W.make_attn_workload("bf16_d64_ragged", 12, "bf16", 8, 2, 64, [1000, 37, 0], [5, 40, 17])
+    run_and_check(w2, poison=True)
+    run_and_check(w2, poison=True, fused=True)
+
+
 def test_c2_decode_verify():
     b, stats = run_and_check(W.c2_decode_verify(), strict=True)
     assert b.ws_bytes > 0  # the context is split over many CTAs
