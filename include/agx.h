@@ -16,10 +16,14 @@
  *     the call returns without synchronising (except agx_get_status and the *_host call).
  *   - "device" pointers are device memory owned by the caller; "host" pointers are ordinary host
  *     memory read during the call only (the caller may reuse it as soon as the call returns).
- *     The library never frees or retains caller memory.  The handle owns a few hundred bytes of
- *     device state (a status word and a ticket counter).
+ *     The library never frees or retains caller memory.
  *   - A handle must be used from one stream at a time: calls on the same handle that overlap on
- *     the GPU share that state and race.
+ *     the GPU share that state and race.  Host threads: a handle is not thread-safe (it caches the last
+ *     launch plan, the pools' tensor maps and the last error text); use it from one host thread at a
+ *     time, or one handle per thread.  Different handles may be used concurrently: the only
+ *     process-wide state is a per-device note that a kernel's launch attributes have been set, which
+ *     every thread writes with the same value.
+ *   - The handle owns 256 bytes of device memory (a status word and the accept step's ticket counter).
  *   - Ragged batches: B sequences; sequence s has a cached prefix of prefix_len[s] tokens and a
  *     block of q_len[s] >= 1 new tokens; cu_q[B+1] is the exclusive prefix sum of q_len and
  *     total_q = cu_q[B].  Rows of q_block, k_new, v_new, out and logits are sequence-major,
