@@ -23,7 +23,8 @@
  *     time, or one handle per thread.  Different handles may be used concurrently: the only
  *     process-wide state is a per-device note that a kernel's launch attributes have been set, which
  *     every thread writes with the same value.
- *   - The handle owns 256 bytes of device memory (a status word and the accept step's ticket counter).
+ *   - The handle owns 512 KB of device memory (a status word, the accept step's ticket counter and one
+ *     64-bit key per logits row it can take, 65535).
  *   - Ragged batches: B sequences; sequence s has a cached prefix of prefix_len[s] tokens and a
  *     block of q_len[s] >= 1 new tokens; cu_q[B+1] is the exclusive prefix sum of q_len and
  *     total_q = cu_q[B].  Rows of q_block, k_new, v_new, out and logits are sequence-major,
@@ -173,7 +174,7 @@ AGX_API agx_status agx_attn_prefixed_append(agx_handle* handle, const void* q_bl
                                             void* out, float* lse, void* workspace, size_t workspace_bytes,
                                             void* stream);
 
-/* Scratch bytes agx_accept_greedy needs for total_q logits rows. */
+/* Scratch bytes agx_accept_greedy needs for total_q logits rows (the rows' winners; a few KB). */
 AGX_API int64_t agx_accept_workspace_bytes(agx_handle* handle, int32_t total_q, int32_t vocab);
 
 /*
@@ -216,12 +217,11 @@ AGX_API agx_status agx_accept_greedy(agx_handle* handle, const void* logits, int
  * embedded or serving runtime with a fixed device-memory budget), or next to an allocator it does
  * not own, where a cudaMalloc may synchronise the whole device, fragment the pool or simply be
  * forbidden.  This call takes no handle and no workspace and performs no allocation of any kind;
- * it uses a fixed scratch array inside the library (about 73 KB of device memory on every GPU that
+ * it uses a fixed scratch array inside the library (about 16 KB of device memory on every GPU that
  * loads the library, held until the process exits).
  *
  * Limit: total_q <= 2048 logits rows per call; more rows return AGX_E_RANGE and should use
- * agx_accept_greedy with a workspace.  (Each row is scanned in as many vocabulary chunks as fit the
- * array's 8192 key slots, at most 8 CTAs per SM.)
+ * agx_accept_greedy with a workspace.  (The array holds one 64-bit key per row and a counter.)
  *
  * The first call on each device looks up the device address of the scratch array (that device
  * must be current); make that first call outside any stream capture.  The look-up is guarded, so

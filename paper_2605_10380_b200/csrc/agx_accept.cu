@@ -4,9 +4,11 @@
 //
 // HBM-bound scan: rows * vocab * elem bytes, read once with 128-bit loads.  Grid = (chunks, rows);
 // every block reduces its slice of one row to a packed 64-bit (ordered value, inverted index) key
-// whose unsigned maximum is "largest value, lowest index on ties".  The last block to finish
-// (ticket counter) folds the per-chunk keys, compares drafts and writes the results, so no second
-// launch and no host round trip is needed.
+// whose unsigned maximum is "largest value, lowest index on ties", and folds it into the row's key
+// with one 64-bit atomic maximum (order-independent, so the result is bit-reproducible).  The last
+// block to finish (ticket counter) reads the row keys back, leaves them and the ticket at zero for
+// the next launch, compares drafts and writes the results, so no second launch and no host round
+// trip is needed.
 #include "agx_internal.cuh"
 #include "agx_sm100.cuh"
 
@@ -44,14 +46,14 @@ __device__ __forceinline__ void scan_vec(const uint4 v, unsigned int base, unsig
     }
 }
 
-constexpr int kFoldKeys = 2048;              // 16 KB of shared memory for the final fold
+constexpr int kTokSmem = 2048;               // winners of up to this many rows stay in shared memory for the draft comparison
 
 template <bool kBf16, bool kVec>
 __global__ void __launch_bounds__(256)
-accept_kernel(const void* __restrict__ logits, long long row_stride, int vocab, int chunk_elems, int chunks,
+accept_kernel(const void* __restrict__ logits, long long row_stride, int vocab, int chunk_elems,
               const int* __restrict__ drafts, const int* __restrict__ cu_q, int B, int total_q,
               int* __restrict__ accept_len, int* __restrict__ next_token, int* __restrict__ argmax,
-              int* __restrict__ seq_lens, unsigned long long* partials, int* tokens, unsigned int* ticket) {
+              int* __restrict__ seq_lens, unsigned long long* row_keys, int* tokens_global, unsigned int* ticket) {
     constexpr int kVecElems = kBf16 ? 8 : 4;
     pdl_launch_dependents();
     pdl_wait();
@@ -116,7 +118,7 @@ accept_kernel(const void* __restrict__ logits, long long row_stride, int vocab, 
         unsigned long long b = warp_best[0];
 #pragma unroll
         for (int w = 1; w < 8; ++w) b = warp_best[w] > b ? warp_best[w] : b;
-        partials[(size_t)row * chunks + chunk] = b;
+        if (b) atomicMax(row_keys + row, b);   // (every key of a real element is non-zero: its low word is 2^32 - 1 - index)
         __threadfence();
         const unsigned int total = gridDim.x * gridDim.y;
         const unsigned int t = atomicAdd(ticket, 1u);
@@ -127,35 +129,20 @@ accept_kernel(const void* __restrict__ logits, long long row_stride, int vocab, 
     if (!is_last) return;
     __threadfence();
 
-    // final fold: one warp per row, the row's chunk keys spread over the lanes.  Up to kFoldKeys keys are first
-    // brought into shared memory by all threads at once (one memory round trip whatever the number of rows).
-    __shared__ unsigned long long keys[kFoldKeys];
-    const int n_keys = total_q * chunks;
-    const bool staged = n_keys <= kFoldKeys;
-    if (staged) {
-        for (int k = threadIdx.x; k < n_keys; k += 256) keys[k] = __ldcg(partials + k);
-        __syncthreads();
-    }
-    for (int r = threadIdx.x >> 5; r < total_q; r += 8) {
-        unsigned long long b = 0ull;
-        for (int c = threadIdx.x & 31; c < chunks; c += 32) {
-            const unsigned long long v = staged ? keys[r * chunks + c] : __ldcg(partials + (size_t)r * chunks + c);
-            b = v > b ? v : b;
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, b, off);
-            b = o > b ? o : b;
-        }
-        if ((threadIdx.x & 31) == 0) {
-            const int t = (int)(0xFFFFFFFFu - (unsigned int)(b & 0xFFFFFFFFull));
-            tokens[r] = t;
-            if (argmax) argmax[r] = t;
-        }
+    // the rows' winners: read the keys back past the L1, zero them for the next launch; up to kTokSmem winners stay in
+    // shared memory for the draft comparison, more go through global memory
+    __shared__ int tokens_smem[kTokSmem];
+    const bool in_smem = total_q <= kTokSmem;
+    int* tokens = in_smem ? tokens_smem : tokens_global;
+    for (int r = threadIdx.x; r < total_q; r += 256) {
+        const unsigned long long b = __ldcg(row_keys + r);
+        row_keys[r] = 0ull;
+        const int t = (int)(0xFFFFFFFFu - (unsigned int)(b & 0xFFFFFFFFull));
+        tokens[r] = t;
+        if (argmax) argmax[r] = t;
     }
     __syncthreads();
-    // draft comparison and commit: one warp per sequence, 32 drafts compared at a time (the winners are read back
-    // past the L1: other warps of this block wrote them a moment ago)
+    // draft comparison and commit: one warp per sequence, 32 drafts compared at a time
     for (int s = threadIdx.x >> 5; s < B; s += 8) {
         const int lane = threadIdx.x & 31;
         const int r0 = cu_q[s];
@@ -163,7 +150,7 @@ accept_kernel(const void* __restrict__ logits, long long row_stride, int vocab, 
         const int* dr = drafts + (r0 - s);
         int a = 0;
         while (a < k) {
-            const bool match = (a + lane < k) ? (dr[a + lane] == __ldcg(tokens + r0 + a + lane)) : false;
+            const bool match = (a + lane < k) ? (dr[a + lane] == (in_smem ? tokens[r0 + a + lane] : __ldcg(tokens + r0 + a + lane))) : false;
             const unsigned int m = __ballot_sync(0xFFFFFFFFu, match);
             const int run = (m == 0xFFFFFFFFu) ? 32 : __ffs(~m) - 1;   // leading matches of this group of 32
             a += run;
@@ -171,7 +158,7 @@ accept_kernel(const void* __restrict__ logits, long long row_stride, int vocab, 
         }
         if (lane == 0) {
             accept_len[s] = a;
-            next_token[s] = __ldcg(tokens + r0 + a);
+            next_token[s] = in_smem ? tokens[r0 + a] : __ldcg(tokens + r0 + a);
             if (seq_lens) seq_lens[s] = seq_lens[s] + a + 1;
         }
     }
@@ -179,7 +166,7 @@ accept_kernel(const void* __restrict__ logits, long long row_stride, int vocab, 
 
 cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_stride, int vocab, const int* drafts,
                           const int* cu_q, int B, int total_q, int* accept_len, int* next_token, int* argmax,
-                          int* seq_lens, unsigned long long* partials, int chunks, unsigned int* ticket,
+                          int* seq_lens, unsigned long long* row_keys, int* tokens_global, int chunks, unsigned int* ticket,
                           cudaStream_t stream) {
     const bool bf16 = logits_dtype == AGX_BF16;
     const int esz = bf16 ? 2 : 4;
@@ -187,12 +174,11 @@ cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_st
     int chunk_elems = (vocab + chunks - 1) / chunks;
     chunk_elems = (chunk_elems + vec_elems - 1) / vec_elems * vec_elems;  // chunk starts stay 16-byte aligned
     const bool vec = ((uintptr_t)logits % 16 == 0) && ((row_stride * esz) % 16 == 0);
-    int* tokens = (int*)(partials + (size_t)total_q * chunks);
     dim3 grid(chunks, total_q);
     cudaError_t err = cudaSuccess;
 #define AGX_LAUNCH_ACCEPT(BF, VEC)                                                                              \
     err = launch_chained(accept_kernel<BF, VEC>, grid, dim3(256), 0, stream, logits, row_stride, vocab, chunk_elems,  \
-                         chunks, drafts, cu_q, B, total_q, accept_len, next_token, argmax, seq_lens, partials, tokens, \
+                         drafts, cu_q, B, total_q, accept_len, next_token, argmax, seq_lens, row_keys, tokens_global, \
                          ticket)
     if (bf16) { if (vec) AGX_LAUNCH_ACCEPT(true, true); else AGX_LAUNCH_ACCEPT(true, false); }
     else      { if (vec) AGX_LAUNCH_ACCEPT(false, true); else AGX_LAUNCH_ACCEPT(false, false); }
@@ -210,19 +196,18 @@ cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_st
 // code that must not disturb a caching allocator owned by someone else (a cudaMalloc there can
 // synchronise the device or fail outright).  agx_accept_greedy needs a caller-provided workspace
 // and a handle whose creation allocates; the entry point below needs neither.  Its scratch (the
-// per-chunk argmax keys, the per-row winners and the ticket counter) lives in a fixed array that
-// is part of the loaded module, so every GPU that loads the library carries these 73 KB until the
-// process exits.
+// rows' argmax keys and the ticket counter) lives in a fixed array that is part of the loaded
+// module, so every GPU that loads the library carries these 16 KB until the process exits.
 #include <atomic>
 #include <mutex>
 
 namespace agx {
 namespace {
-constexpr int kStaticMaxRows = 2048;    // logits rows per call
-constexpr int kStaticMaxSlots = 8192;   // rows * chunks partial keys per call
+constexpr int kStaticMaxRows = 2048;    // logits rows per call (their winners fit the kernel's shared memory)
 constexpr int kStaticDevices = 64;
-// layout: [0, 256) ticket counter | partial keys (8 B each) | per-row winners (4 B each)
-constexpr size_t kStaticBytes = 256 + (size_t)kStaticMaxSlots * 8 + (size_t)kStaticMaxRows * 4;
+// layout: [0, 256) ticket counter | one 64-bit key per row
+constexpr size_t kStaticBytes = 256 + (size_t)kStaticMaxRows * 8;
+static_assert(kStaticMaxRows <= kTokSmem, "the allocation-free variant has no global buffer for the rows' winners");
 static __device__ __align__(256) unsigned char g_accept_scratch[kStaticBytes];
 
 struct StaticDeviceState {
@@ -274,10 +259,9 @@ extern "C" AGX_API agx_status agx_accept_greedy_static(const void* logits, int32
         }
     }
     // Chunks per row: enough CTAs that every thread needs a single trip of two 16-byte loads (8 per SM, as the workspace
-    // variant aims for), as far as the fixed number of key slots goes: rows * chunks <= target + rows <= kStaticMaxSlots.
+    // variant aims for).
     const int vec = logits_dtype == AGX_BF16 ? 8 : 4;
-    const int target = 8 * st.sm_count < kStaticMaxSlots - kStaticMaxRows ? 8 * st.sm_count : kStaticMaxSlots - kStaticMaxRows;
-    int want = (target + total_q - 1) / total_q;
+    int want = (8 * st.sm_count + total_q - 1) / total_q;
     const int max_chunks = (vocab + 256 * vec * 2 - 1) / (256 * vec * 2);   // >= 2 vectors per thread
     if (want > max_chunks) want = max_chunks;
     if (want < 1) want = 1;
@@ -286,11 +270,11 @@ extern "C" AGX_API agx_status agx_accept_greedy_static(const void* logits, int32
     const int chunks = (vocab + chunk_elems - 1) / chunk_elems;   // <= want
 
     unsigned char* base = (unsigned char*)scratch;
-    // the array keeps whatever the previous call left: the ticket counter must start at zero
-    if (cudaMemsetAsync(base, 0, 256, (cudaStream_t)stream) != cudaSuccess) return AGX_E_CUDA;
-    // launch_accept places the per-row winners right behind total_q * chunks keys
+    // the array keeps whatever the previous call left: the ticket counter and the rows' keys must start at zero (the
+    // kernel leaves them at zero itself; the clear makes the call independent of how an earlier one ended)
+    if (cudaMemsetAsync(base, 0, 256 + (size_t)total_q * 8, (cudaStream_t)stream) != cudaSuccess) return AGX_E_CUDA;
     cudaError_t e = launch_accept(logits, logits_dtype, row_stride, vocab, drafts, cu_q, B, total_q, accept_len,
-                                  next_token, argmax, seq_lens, (unsigned long long*)(base + 256), chunks,
+                                  next_token, argmax, seq_lens, (unsigned long long*)(base + 256), nullptr, chunks,
                                   (unsigned int*)base, (cudaStream_t)stream);
     return e == cudaSuccess ? AGX_OK : AGX_E_CUDA;
 }

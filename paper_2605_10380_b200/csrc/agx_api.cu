@@ -36,6 +36,7 @@ struct agx_handle {
     int sm_count;
     int* d_status;          // device status word
     unsigned int* d_ticket; // ticket counter of the accept kernel (self-resetting)
+    unsigned long long* d_row_keys;   // one argmax key per logits row of the accept kernel (all zero between launches)
     int last_launches;
     int small_min_split;    // tokens; tuning knob (env AGX_SMALL_MIN_SPLIT)
     int force_mma_sync;     // route large q through the mma.sync kernel (env AGX_FORCE_MMA_SYNC)
@@ -375,11 +376,13 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     int major = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, h->device);
     if (e == cudaSuccess && major != 10) { delete h; return AGX_E_UNSUPPORTED; }
-    if (e == cudaSuccess) e = cudaMalloc((void**)&h->d_status, 256);
+    constexpr size_t kStateBytes = 256 + 65536 * 8;   // status word and accept ticket | one key per logits row (at most 65535)
+    if (e == cudaSuccess) e = cudaMalloc((void**)&h->d_status, kStateBytes);
     if (e != cudaSuccess) { delete h; return e == cudaErrorMemoryAllocation ? AGX_E_NOMEM : AGX_E_CUDA; }
-    e = cudaMemset(h->d_status, 0, 256);
+    e = cudaMemset(h->d_status, 0, kStateBytes);
     if (e != cudaSuccess) { cudaFree(h->d_status); delete h; return AGX_E_CUDA; }
     h->d_ticket = (unsigned int*)(h->d_status + 16);
+    h->d_row_keys = (unsigned long long*)(h->d_status + 64);
     *out = h;
     return AGX_OK;
 }
@@ -551,10 +554,8 @@ static int accept_chunks(const agx_handle* h, int total_q, int vocab, int dtype)
 int64_t agx_accept_workspace_bytes(agx_handle* h, int32_t total_q, int32_t vocab) {
     if (!h) return AGX_E_INVAL;
     if (total_q < 0 || vocab < 1) return fail(h, AGX_E_RANGE, "total_q < 0 or vocab < 1");
-    // chunk count depends on the logits dtype; size for the larger of the two
-    const int chunks = std::max(accept_chunks(h, std::max(total_q, 1), vocab, AGX_BF16),
-                                accept_chunks(h, std::max(total_q, 1), vocab, AGX_F32));
-    return (int64_t)total_q * chunks * 8 + (int64_t)total_q * 4 + 256;
+    // the rows' winners when they do not fit the kernel's shared memory (more than 2048 rows); the rows' keys live in the handle
+    return (int64_t)total_q * 4 + 256;
 }
 
 agx_status agx_accept_greedy(agx_handle* h, const void* logits, int32_t logits_dtype, int64_t row_stride,
@@ -577,7 +578,7 @@ agx_status agx_accept_greedy(agx_handle* h, const void* logits, int32_t logits_d
         return fail(h, AGX_E_INVAL, "accept workspace missing, misaligned or too small (%lld needed)", (long long)need);
     const int chunks = accept_chunks(h, total_q, vocab, logits_dtype);
     cudaError_t e = launch_accept(logits, logits_dtype, row_stride, vocab, drafts, cu_q, B, total_q, accept_len,
-                                  next_token, argmax, seq_lens, (unsigned long long*)workspace, chunks, h->d_ticket,
+                                  next_token, argmax, seq_lens, h->d_row_keys, (int*)workspace, chunks, h->d_ticket,
                                   (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(h, e, "accept launch");
     h->last_launches = 1;

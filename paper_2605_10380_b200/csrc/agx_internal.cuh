@@ -136,7 +136,7 @@ cudaError_t launch_attn_tile_bf16(const AttnParams& p, bool streams, const CUten
 
 cudaError_t launch_accept(const void* logits, int logits_dtype, long long row_stride, int vocab, const int* drafts,
                           const int* cu_q, int B, int total_q, int* accept_len, int* next_token, int* argmax,
-                          int* seq_lens, unsigned long long* partials, int chunks, unsigned int* ticket,
+                          int* seq_lens, unsigned long long* row_keys, int* tokens_global, int chunks, unsigned int* ticket,
                           cudaStream_t stream);
 
 // Private copies of KV pages (a reused prefix that is cut inside a page, Sec. 4.2).
