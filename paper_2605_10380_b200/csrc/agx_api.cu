@@ -168,7 +168,7 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
         long long base_items = 0;  // items per split, summed over sequences
         std::vector<long long> per_seq_items(seqs.size());
         if (k == KIND_SIMT) { unit = 64; min_split = 256; target = h->sm_count * 16; }
-        else if (k == KIND_TILE || k == KIND_STREAM) { unit = 128; min_split = k == KIND_TILE ? 512 : 256; target = h->sm_count; }
+        else if (k == KIND_TILE || k == KIND_STREAM) { unit = 128; min_split = k == KIND_TILE ? 128 : 256; target = h->sm_count; }
         else { unit = 16; min_split = h->small_min_split; target = h->sm_count * ((k == KIND_SMALL4 || small_kw == 8) ? 1 : 2); }
         const int rows_per_chunk = (k == KIND_SMALL1) ? 16 : (k == KIND_SMALL2) ? 32 : (k == KIND_SMALL4) ? 64 : (k == KIND_STREAM) ? 128 : 256;
         long long work = 0;
@@ -198,8 +198,9 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
         if (k == KIND_TILE || k == KIND_STREAM) {
             // several waves are fine here: pick the split length with the smallest estimated makespan, in units of one KV
             // tile's time (~1.6 us): waves * (tiles per item + fixed per-CTA cost of ~3 tiles), plus what the split costs
-            // afterwards: the merge launch (~2 units) and the partial rows written and read back (~0.3 units per MB;
-            // measured on a ragged batch of eight suffix prefills: 95 MB of partials cost 60 us more than 22 MB)
+            // afterwards: the merge launch (~2 units) and the partial rows written and read back (~0.3 units per MB beyond the
+            // first 16 MB, which stay in L2; measured on a ragged batch of eight suffix prefills: 95 MB of partials cost 60 us
+            // more than 22 MB, while 9 MB in one-tile splits of a 128-token suffix over 1000 tokens cost nothing)
             int max_len = 0;
             for (int s : seqs) max_len = std::max(max_len, P[s] + Q[s]);
             const long long row_bytes = k == KIND_TILE ? 256 : 520;   // fp16 row | fp32 row + (m, l)
@@ -212,7 +213,7 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
                     if (ns > 1) part_bytes += (long long)Q[s] * c.num_q_heads * ns * row_bytes;
                 }
                 const long long cost = 16 * waves * (std::min(c_tokens, round_up(max_len, unit)) / unit + 3) +
-                                       (part_bytes ? 32 + 5 * (part_bytes >> 20) : 0);
+                                       (part_bytes ? 32 + 5 * std::max<long long>(0, (part_bytes >> 20) - 16) : 0);
                 if (best_cost < 0 || cost < best_cost) { best_cost = cost; C = c_tokens; }
             }
             if (const char* force = getenv("AGX_TILE_SPLIT_TOKENS")) { if (atoi(force) >= unit) C = atoi(force) / unit * unit; }
