@@ -43,6 +43,7 @@ struct agx_handle {
     int debug_plan;         // print launch plans to stderr (env AGX_DEBUG_PLAN)
     int small_kw;           // pages per pipeline stage of the warp-MMA kernel: 4, 8, or 0 = chosen per batch (env AGX_SMALL_KW)
     int batch_stream_tokens; // total tokens of a batch's small blocks from which they all take the stream schedule (env AGX_BATCH_STREAM_TOKENS)
+    bool merge_sms;         // one-wave small-q launches leave SMs free for their merge kernel (env AGX_MERGE_SMS=0 turns it off)
     bool cluster_merge;     // KV splits of the small-q kernel merged inside thread-block clusters where the batch allows (env AGX_CLUSTER_MERGE=0 turns it off)
     int zero_copy;          // host steps: bit 0 = kernels read small pinned inputs, bit 1 = kernels write `out` into a pinned buffer (env AGX_ZERO_COPY, default 3)
     int stream_max_rows;    // blocks of up to this many rows per KV head may take the one-Q-tile schedule in 128-row chunks (env AGX_STREAM_MAX_ROWS)
@@ -101,6 +102,7 @@ struct Launch {
     int num_items;
     int kw;          // small-q kernel: pages per pipeline stage (KV groups), 4 or 8
     int cluster;     // > 1: CTAs per cluster = KV splits of every sequence of the launch, merged in-kernel (no partials)
+    bool lean_merge; // small-q kernel: fp16 partials, merged by the two-warp merge kernel on SMs left out of the attention grid
     std::vector<SeqPlan> seqs;
 };
 
@@ -245,6 +247,29 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
                 if (h->debug_plan) fprintf(stderr, "agx plan: clusters of %d: %d fit the device, %lld needed\n", common, fit, base_items);
             }
         }
+        // ---- small-q kernel, one wave of one CTA per SM, splits merged by the merge kernel: leave that kernel SMs of its own.
+        //      An attention CTA takes a whole SM, so merge CTAs that find no free SM sit on SMs the next call's attention CTAs
+        //      need, and those CTAs then start (and fetch their K/V) only after the merge instead of under it.  With a few SMs
+        //      left out of the attention grid the merge CTAs are resident there from the start and the next call's grid
+        //      follows this one without a gap.  A two-warp merge CTA handles two (row, head) pairs; 12 (up to 20 splits) or 8
+        //      of them fit an SM.
+        bool lean_merge = false;   // fp16 partials and the two-warp merge kernel (slower than fp32 partials and the four-warp
+                                   // one where the attention grid fills every SM twice over, e.g. four verify blocks of 4096)
+        if (!cluster && (k == KIND_SMALL1 || k == KIND_SMALL2 || k == KIND_SMALL4) && (k == KIND_SMALL4 || small_kw == 8) &&
+            seqs.size() <= (size_t)kMaxSeqs && h->merge_sms) {
+            long long pairs = 0;
+            for (int s : seqs) pairs += (long long)Q[s] * c.num_q_heads;
+            for (;;) {
+                const long long items = count_items(C);
+                int ns_max = 1;
+                for (int s : seqs) ns_max = std::max(ns_max, (P[s] + Q[s] + C - 1) / C);
+                if (ns_max == 1 || items > h->sm_count) break;   // no merge, or more than one wave anyway
+                const long long reserve = (pairs + (ns_max <= 20 ? 24 : 16) - 1) / (ns_max <= 20 ? 24 : 16);
+                lean_merge = true;
+                if (reserve > h->sm_count / 8 || items <= h->sm_count - reserve || items <= base_items) break;
+                C += unit;
+            }
+        }
         // ---- emit launches of at most kMaxSeqs sequences
         for (size_t a = 0; a < seqs.size(); a += kMaxSeqs) {
             Launch ln;
@@ -252,6 +277,7 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
             ln.total_rows = 0;
             ln.num_items = 0;
             ln.cluster = cluster;
+            ln.lean_merge = lean_merge;
             ln.kw = (k == KIND_SMALL4) ? 4 : small_kw;
             for (size_t n = a; n < std::min(seqs.size(), a + kMaxSeqs); ++n) {
                 const int s = seqs[n];
@@ -360,6 +386,8 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     h->stream_max_rows = env ? atoi(env) : 384;
     env = getenv("AGX_CLUSTER_MERGE");
     h->cluster_merge = !(env && atoi(env) == 0);
+    env = getenv("AGX_MERGE_SMS");
+    h->merge_sms = !(env && atoi(env) == 0);
     env = getenv("AGX_ZERO_COPY");
     h->zero_copy = env ? atoi(env) : 3;
     env = getenv("AGX_SMALL_KW");
@@ -493,7 +521,7 @@ static agx_status attn_impl(agx_handle* h, const void* q_block, const void* k_ne
         }
         cudaError_t e;
         p.cluster_size = ln.cluster;
-        p.part_half = ln.kind == KIND_TILE;
+        p.part_half = ln.kind == KIND_TILE || ln.lean_merge;
         p.k_new = p.v_new = nullptr;
         if (k_new) {
             p.k_new = k_new; p.v_new = v_new;

@@ -149,67 +149,72 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     auto produce = [&](int stage) {   // called by all lanes of warp 0
         if (stage >= n_stages || !alive) return;
         const int slot = stage % NS;
-        alive = mbar_wait(empty_bar(slot), ((stage / NS) & 1) ^ 1, abort_flag, p.status, p.wait_limit_cycles);
-        if (!alive) return;
+        alive = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(slot), ((stage / NS) & 1) ^ 1, abort_flag, p.status, p.wait_limit_cycles));
+        if (!alive) return;   // (the same answer in every lane: the lanes stay together for the shuffles and copies below)
         const int pi0 = stage * kKW;
         if ((pi0 >> 5) != group_cur) { ids_cur = ids_next; group_cur = pi0 >> 5; ids_next = fetch_ids(group_cur + 1); }
         const int npg = min(kKW, n_pages - pi0);
-        int id[kKW];
-#pragma unroll
-        for (int pg = 0; pg < kKW; ++pg) id[pg] = __shfl_sync(0xFFFFFFFFu, ids_cur, (pi0 + pg) & 31);
+        const int my_id = __shfl_sync(0xFFFFFFFFu, ids_cur, (pi0 + lane) & 31);   // lane pg < npg: the id of the stage's page pg
         if (stage == p.drop_stage) return;   // test hook: this stage never arrives, its consumers' waits run out
         if (lane == 0) {
             mbar_arrive_expect_tx(full_bar(slot), npg * 8192u);
             last_armed = stage;
-            const uint32_t dst0 = smem_base + slot * kStageBytes;
-#pragma unroll
-            for (int pg = 0; pg < kKW; ++pg) {
-                if (pg < npg) {
-                    const int y = (id[pg] * p.hkv + g) * kPage;
-                    const uint32_t dk = dst0 + pg * 4096, dv = dk + kStageTokens * kRowBytes;
-                    tma_load_2d(dk, &map_k, 0, y, full_bar(slot));
-                    tma_load_2d(dk + 2048, &map_k, 64, y, full_bar(slot));
-                    tma_load_2d(dv, &map_v, 0, y, full_bar(slot));
-                    tma_load_2d(dv + 2048, &map_v, 64, y, full_bar(slot));
-                }
-            }
+        }
+        __syncwarp();   // the barrier is armed before any lane's copies can complete on it
+        // lane pg copies page pg: one lane issuing a stage's 32 boxes of 2 KB takes ~60 ns per box, eight lanes ~40 (measured)
+        if (lane < npg) {
+            const int y = (my_id * p.hkv + g) * kPage;
+            const uint32_t dk = smem_base + slot * kStageBytes + lane * 4096, dv = dk + kStageTokens * kRowBytes;
+            tma_load_2d(dk, &map_k, 0, y, full_bar(slot));
+            tma_load_2d(dk + 2048, &map_k, 64, y, full_bar(slot));
+            tma_load_2d(dv, &map_v, 0, y, full_bar(slot));
+            tma_load_2d(dv + 2048, &map_v, 64, y, full_bar(slot));
         }
     };
-    // The producer lane set the barriers up itself, so it needs nothing from the other warps: it fetches the page
+    // A CTA with block rows of its own stores them first (fused append, one row chunk per sequence); its producer warp
+    // waits on a named barrier until every thread's rows are in the pages, the other warps only arrive there and go on.
+    if (own_rows) {
+        append_rows_bf16(p, sp, g, tok_begin, tok_begin + sp.split_tokens, tid, kThreads);
+        if (warp != 0) asm volatile("bar.arrive 8, %0;\n" ::"n"(kThreads) : "memory");
+    }
+    // The producer lane set the barriers up itself, so it needs nothing else from the other warps: it fetches the page
     // ids and issues the first copies at once, while the others bring the Q tile in.
     if (warp == 0) {
         __syncwarp();   // lane 0's barrier initialisation, before the other lanes poll those barriers
         ids_cur = fetch_ids(0);
         ids_next = fetch_ids(1);
         bool waited = !pre;
-        if (!own_rows) {
-            const int stable_end = P & ~(kPage - 1);   // tokens below this sit in pages no append of this block touches
-#pragma unroll
-            for (int s = 0; s < NS - 1; ++s) {
-                if (!waited && tok_begin + (s + 1) * kStageTokens > stable_end) { pdl_wait(); waited = true; }
-                produce(s);
-            }
+        if (own_rows) asm volatile("bar.sync 8, %0;\n" ::"n"(kThreads) : "memory");
+        const int stable_end = P & ~(kPage - 1);   // tokens below this sit in pages no append of this block touches
+#pragma unroll 1
+        for (int s = 0; s < NS - 1; ++s) {
+            if (!waited && tok_begin + (s + 1) * kStageTokens > stable_end) { pdl_wait(); waited = true; }
+            produce(s);
         }
         if (!waited) pdl_wait();
     }
-    if (own_rows) append_rows_bf16(p, sp, g, tok_begin, tok_begin + sp.split_tokens, tid, kThreads);   // fused append (row_chunks == 1)
     // ---- Q tile -> shared (rows beyond q*G are zero), by the warps other than the producer's
-    for (int c = tid - 32; c >= 0 && c < MT * 16 * 16; c += kThreads - 32) {
-        const int r = c >> 4, ch = c & 15;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (row0 + r < rows) {
-            const int i = (row0 + r) / G, hg = (row0 + r) - i * G;
-            const long long off = ((long long)(sp.q_row0 + i) * p.hq + g * G + hg) * kRowBytes + ch * 16;
-            v = __ldg((const uint4*)((const unsigned char*)p.q + off));
+    //      (a thread's loads are all issued before its first store: one trip to memory, not one per 16-byte unit)
+    if (tid >= 32) {
+        constexpr int kUnits = MT * 16 * 16, kLoaders = kThreads - 32, kPer = (kUnits + kLoaders - 1) / kLoaders;
+        uint4 v[kPer];
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const int c = tid - 32 + j * kLoaders, r = c >> 4, ch = c & 15;
+            v[j] = make_uint4(0, 0, 0, 0);
+            if (c < kUnits && row0 + r < rows) {
+                const int i = (row0 + r) / G, hg = (row0 + r) - i * G;
+                const long long off = ((long long)(sp.q_row0 + i) * p.hq + g * G + hg) * kRowBytes + ch * 16;
+                v[j] = __ldg((const uint4*)((const unsigned char*)p.q + off));
+            }
         }
-        *(uint4*)(q_smem + swz(r, ch)) = v;
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const int c = tid - 32 + j * kLoaders;
+            if (c < kUnits) *(uint4*)(q_smem + swz(c >> 4, c & 15)) = v[j];
+        }
     }
     __syncthreads();  // barriers initialised, Q tile visible
-    if (warp == 0 && own_rows) {
-#pragma unroll
-        for (int s = 0; s < NS - 1; ++s) produce(s);
-    }
-
 
     uint32_t qa[8][4];
     {
@@ -255,6 +260,7 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     auto group_sync = [&]() { asm volatile("bar.sync %0, %1;\n" ::"r"(1 + mt), "n"(32 * KW) : "memory"); };
 
     bool live = true;   // a warp whose wait gave up keeps meeting the others at the group barriers
+#pragma unroll 1
     for (int stage = 0; stage < n_stages; ++stage) {
         const int slot = stage % NS;
         if (warp == 0) produce(stage + NS - 1);
@@ -410,6 +416,7 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int r = mt * 16 + rg + 8 * h;                  // row of the CTA's chunk
+        const unsigned int row_lanes = __ballot_sync(0xFFFFFFFFu, row0 + r < rows);   // (the four lanes of a row go together)
         if (row0 + r >= rows) continue;
         float l_all = 0.f;
 #pragma unroll
@@ -429,19 +436,43 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
                 *(uint32_t*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)) = pack_bf16(o[n][2 * h] * inv, o[n][2 * h + 1] * inv);
             if (p.lse && first) p.lse[(long long)(sp.q_row0 + i) * p.hq + hd] = (m_all + log2f(l_all)) * 0.6931471805599453f;
         } else {
-            float* orow;
             if (in_cluster) {
-                orow = cl_o + r * kD;
+                float* orow = cl_o + r * kD;
                 if (first) cl_ml[r] = make_float2(m_all, l_all);
-            } else {
-                const long long e = (long long)sp.part_base + ((long long)i * p.hq + hd) * sp.nsplit + split;
-                orow = p.part_o + e * kD;
-                if (first) p.part_ml[e] = make_float2(m_all, l_all);
-            }
 #pragma unroll
-            for (int n = 0; n < 2 * kCG; ++n)
-                if (in_cluster) *(float2*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)) = make_float2(o[n][2 * h], o[n][2 * h + 1]);
-                else __stcg((float2*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)), make_float2(o[n][2 * h], o[n][2 * h + 1]));   // read next by other SMs
+                for (int n = 0; n < 2 * kCG; ++n)
+                    *(float2*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)) = make_float2(o[n][2 * h], o[n][2 * h + 1]);
+            } else {
+                // split partial for the merge kernel, written past the L1 (read next by other SMs)
+                const long long e = (long long)sp.part_base + ((long long)i * p.hq + hd) * sp.nsplit + split;
+                if (first) p.part_ml[e] = make_float2(m_all, l_all);
+                if (p.part_half) {
+                    // the row divided by its own sum, as fp16 in the first 256 bytes of the entry's 512-byte slot (the merge
+                    // weighs split k by l_k 2^(m_k - m)).  A lane holds two columns of each of two neighbouring 8-column
+                    // tiles: lane pairs swap one pair each, so that every lane stores four consecutive columns (8 bytes) and
+                    // the four lanes of a row write a whole 32-byte sector
+                    const float inv = (l_all > 0.f) ? 1.f / l_all : 0.f;
+                    unsigned char* orow = (unsigned char*)p.part_o + e * 512;
+#pragma unroll
+                    for (int c = 0; c < kCG; ++c) {
+                        const __half2 lo = __floats2half2_rn(o[2 * c][2 * h] * inv, o[2 * c][2 * h + 1] * inv);
+                        const __half2 hi = __floats2half2_rn(o[2 * c + 1][2 * h] * inv, o[2 * c + 1][2 * h + 1] * inv);
+                        const unsigned int mine_lo = *reinterpret_cast<const unsigned int*>(&lo);
+                        const unsigned int mine_hi = *reinterpret_cast<const unsigned int*>(&hi);
+                        const bool odd = lane & 1;
+                        const unsigned int got = __shfl_xor_sync(row_lanes, odd ? mine_lo : mine_hi, 1);
+                        // even lane: its own columns of the first tile, then its partner's; odd lane: the same in the second tile
+                        const uint2 pk = odd ? make_uint2(got, mine_hi) : make_uint2(mine_lo, got);
+                        const int col = (kg * kCG + c) * 16 + (odd ? 8 : 0) + 4 * ((lane & 3) >> 1);
+                        __stcg((uint2*)(orow + col * 2), pk);
+                    }
+                } else {   // the un-normalised fp32 row
+                    float* orow = p.part_o + e * kD;
+#pragma unroll
+                    for (int n = 0; n < 2 * kCG; ++n)
+                        __stcg((float2*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)), make_float2(o[n][2 * h], o[n][2 * h + 1]));
+                }
+            }
         }
     }
     if (in_cluster && sp.nsplit > 1) {   // (uniform over the cluster: all its CTAs belong to one sequence)
@@ -778,6 +809,62 @@ attn_combine_half4_kernel(const __grid_constant__ AttnParams p, int total_rows) 
     }
 }
 
+// The same merge for the fp16 partials of the small-q kernel (5 to 32 KV splits): one (row, head) pair per warp, lane k
+// holding split k's (m, l) and every lane four columns of every split's row, all loads in flight at once.  CTAs of two
+// warps with few registers (12 or 8 CTAs per SM), so that the merge of a one-wave launch fits the few SMs the planner
+// leaves out of the attention grid for it.
+template <int kNsMax>
+__global__ void __launch_bounds__(64, kNsMax <= 20 ? 12 : 8)
+attn_combine_half32_kernel(const __grid_constant__ AttnParams p, int total_rows) {
+    pdl_launch_dependents();
+    const int lane = threadIdx.x & 31;
+    const int rh = blockIdx.x * 2 + (threadIdx.x >> 5);
+    if (rh >= total_rows * p.hq) return;
+    const int lrow = rh / p.hq, h = rh - lrow * p.hq;
+    int si = 0, acc_rows = 0;
+#pragma unroll 1
+    for (int s = 0; s < p.num_seqs; ++s) {
+        if (lrow >= acc_rows && lrow < acc_rows + p.seq[s].q_len) { si = s; break; }
+        acc_rows += p.seq[s].q_len;
+    }
+    const SeqPlan& sp = p.seq[si];
+    const int ns = sp.nsplit;
+    if (ns == 1) return;   // written directly by the attention kernel
+    const int i = lrow - acc_rows;
+    const long long e0 = (long long)sp.part_base + ((long long)i * p.hq + h) * ns;
+    const long long out_off = (long long)(sp.q_row0 + i) * p.hq + h;
+    const unsigned char* rows = (const unsigned char*)p.part_o + e0 * 512 + lane * 8;
+    pdl_wait();   // the partials are complete
+    const float2 ml = (lane < ns) ? __ldcg(p.part_ml + e0 + lane) : make_float2(-INFINITY, 0.f);
+    // no branch between the loads: slots past the last split repeat its row, and weigh nothing below
+    uint2 v[kNsMax];
+#pragma unroll
+    for (int k = 0; k < kNsMax; ++k) v[k] = __ldcg((const uint2*)(rows + min(k, ns - 1) * 512));
+    float m_all = ml.x;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, off));
+    const float w_mine = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m_all) * ml.y;   // 0 in lanes past the last split
+    float l_all = w_mine;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xFFFFFFFFu, l_all, off);   // (a fixed order: reproducible)
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int k = 0; k < kNsMax; ++k) {
+        const float w = __shfl_sync(0xFFFFFFFFu, w_mine, k);
+        // a split that saw no token for this row publishes only (m, l) = (-inf, 0): its row may hold anything, NaN included
+        const bool use = w != 0.f;
+        const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&v[k].x));
+        const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&v[k].y));
+        acc.x += use ? a.x * w : 0.f; acc.y += use ? a.y * w : 0.f; acc.z += use ? b.x * w : 0.f; acc.w += use ? b.y * w : 0.f;
+    }
+    const float inv = 1.f / l_all;
+    uint2 packed;
+    packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+    packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+    *(uint2*)((__nv_bfloat16*)p.out + out_off * kD + lane * 4) = packed;
+    if (p.lse && lane == 0) p.lse[out_off] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+}
+
 // --------------------------------------------------------------------------------------------
 namespace {
 template <int MT, int KW, int NS>
@@ -882,7 +969,12 @@ cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, 
             const int want = (int)((n + 4 * kCombineRows - 1) / (4 * kCombineRows));   // CTAs whose warps take kCombineRows pairs each
             return launch_chained(attn_combine_half4_kernel, dim3(want > one_wave ? blocks : (want > 0 ? want : 1)), dim3(128), 0, stream, p, total_rows);
         }
-        if (ns_max <= 16) return launch_chained(attn_combine_kernel<true, 16, true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
+        if (ns_max <= 32) {
+            if (ns_max <= 8) return launch_chained(attn_combine_half32_kernel<8>, dim3((int)((n + 1) / 2)), dim3(64), 0, stream, p, total_rows);
+            if (ns_max <= 12) return launch_chained(attn_combine_half32_kernel<12>, dim3((int)((n + 1) / 2)), dim3(64), 0, stream, p, total_rows);
+            if (ns_max <= 20) return launch_chained(attn_combine_half32_kernel<20>, dim3((int)((n + 1) / 2)), dim3(64), 0, stream, p, total_rows);
+            return launch_chained(attn_combine_half32_kernel<32>, dim3((int)((n + 1) / 2)), dim3(64), 0, stream, p, total_rows);
+        }
         return launch_chained(attn_combine_kernel<true, 1 << 30, true>, dim3(blocks), dim3(128), 0, stream, p, total_rows);
     }
     if (dtype == AGX_BF16) {
