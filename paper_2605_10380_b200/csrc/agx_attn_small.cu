@@ -53,6 +53,23 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
 // byte offset of 16-byte chunk `ch` (0..15) of row `r` in a [rows][256 B] tile, XOR-swizzled
 __device__ __forceinline__ uint32_t swz(int r, int ch) { return (uint32_t)(r * kRowBytes + ((ch ^ (r & 7)) << 4)); }
 
+// Loads the compiler keeps where they are written (and that go to L2: the data was just written by other SMs).
+__device__ __forceinline__ uint2 ld_volatile_u2(const void* p) {
+    uint2 v;
+    asm volatile("ld.volatile.global.v2.u32 {%0, %1}, [%2];\n" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 ld_volatile_f4(const void* p) {
+    float4 v;
+    asm volatile("ld.volatile.global.v4.f32 {%0, %1, %2, %3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ float2 ld_volatile_f2(const void* p) {
+    float2 v;
+    asm volatile("ld.volatile.global.v2.f32 {%0, %1}, [%2];\n" : "=f"(v.x), "=f"(v.y) : "l"(p) : "memory");
+    return v;
+}
+
 // Locate the work item: sequence plan + (kv head, split).
 __device__ __forceinline__ int find_seq(const AttnParams& p, int item) {
     int s = 0;
@@ -609,12 +626,12 @@ attn_simt_kernel(const __grid_constant__ AttnParams p) {
 template <bool kHalfPart>
 __device__ __forceinline__ float4 load_part4(const AttnParams& p, long long entry, int c4) {
     if (kHalfPart) {
-        const uint2 raw = __ldcg((const uint2*)((const unsigned char*)p.part_o + entry * 512 + c4 * 2));   // written by other SMs just before: past the L1
+        const uint2 raw = ld_volatile_u2((const unsigned char*)p.part_o + entry * 512 + c4 * 2);   // written by other SMs just before: past the L1
         const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
         const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
         return make_float4(a.x, a.y, b.x, b.y);
     }
-    return __ldcg((const float4*)(p.part_o + entry * p.head_dim + c4));
+    return ld_volatile_f4(p.part_o + entry * p.head_dim + c4);
 }
 template <bool kBf16Out, int kMaxNs, bool kHalfPart>
 __global__ void __launch_bounds__(128, kMaxNs <= 4 ? 10 : kMaxNs <= 16 ? 5 : 3)
@@ -647,7 +664,9 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
     if (kMaxNs <= 32 || ns <= 32) {
         // One round trip to memory: lane k fetches (m, l) of split k while every lane already fetches its
         // columns of every split's O row; the weights then travel by shuffle, splits in index order.
-        const float2 ml = (lane < ns) ? __ldcg(p.part_ml + e0 + lane) : make_float2(-INFINITY, 0.f);
+        // (volatile loads: the compiler leaves them in this order, ahead of the first use of any of them)
+        float2 ml = make_float2(-INFINITY, 0.f);
+        if (lane < ns) ml = ld_volatile_f2(p.part_ml + e0 + lane);
         float4 v[kInFlight], v2[kFew ? 1 : 16];
 #pragma unroll
         for (int j = 0; j < kInFlight; ++j)
@@ -773,10 +792,11 @@ attn_combine_half4_kernel(const __grid_constant__ AttnParams p, int total_rows) 
     uint2 v[kCombineRows][4];
 #pragma unroll
     for (int j = 0; j < kCombineRows; ++j) {
-        ml[j] = (lane < ns[j]) ? __ldcg(p.part_ml + e0[j] + lane) : make_float2(-INFINITY, 0.f);
+        ml[j] = make_float2(-INFINITY, 0.f);
+        if (lane < ns[j]) ml[j] = ld_volatile_f2(p.part_ml + e0[j] + lane);
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-            if (k < ns[j]) v[j][k] = __ldcg((const uint2*)((const unsigned char*)p.part_o + (e0[j] + k) * 512 + lane * 8));
+            if (k < ns[j]) v[j][k] = ld_volatile_u2((const unsigned char*)p.part_o + (e0[j] + k) * 512 + lane * 8);
     }
 #pragma unroll
     for (int j = 0; j < kCombineRows; ++j) {
@@ -819,50 +839,56 @@ attn_combine_half32_kernel(const __grid_constant__ AttnParams p, int total_rows)
     pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
     const int rh = blockIdx.x * 2 + (threadIdx.x >> 5);
-    if (rh >= total_rows * p.hq) return;
-    const int lrow = rh / p.hq, h = rh - lrow * p.hq;
-    int si = 0, acc_rows = 0;
+    int ns = 1, si = 0, acc_rows = 0, lrow = 0, h = 0;
+    if (rh < total_rows * p.hq) {
+        lrow = rh / p.hq; h = rh - lrow * p.hq;
 #pragma unroll 1
-    for (int s = 0; s < p.num_seqs; ++s) {
-        if (lrow >= acc_rows && lrow < acc_rows + p.seq[s].q_len) { si = s; break; }
-        acc_rows += p.seq[s].q_len;
+        for (int s = 0; s < p.num_seqs; ++s) {
+            if (lrow >= acc_rows && lrow < acc_rows + p.seq[s].q_len) { si = s; break; }
+            acc_rows += p.seq[s].q_len;
+        }
+        ns = p.seq[si].nsplit;
     }
-    const SeqPlan& sp = p.seq[si];
-    const int ns = sp.nsplit;
-    if (ns == 1) return;   // written directly by the attention kernel
-    const int i = lrow - acc_rows;
-    const long long e0 = (long long)sp.part_base + ((long long)i * p.hq + h) * ns;
-    const long long out_off = (long long)(sp.q_row0 + i) * p.hq + h;
-    const unsigned char* rows = (const unsigned char*)p.part_o + e0 * 512 + lane * 8;
-    pdl_wait();   // the partials are complete
-    const float2 ml = (lane < ns) ? __ldcg(p.part_ml + e0 + lane) : make_float2(-INFINITY, 0.f);
-    // no branch between the loads: slots past the last split repeat its row, and weigh nothing below
-    uint2 v[kNsMax];
+    if (ns > 1) {   // (a single split was written directly by the attention kernel)
+        const SeqPlan& sp = p.seq[si];
+        const int i = lrow - acc_rows;
+        const long long e0 = (long long)sp.part_base + ((long long)i * p.hq + h) * ns;
+        const long long out_off = (long long)(sp.q_row0 + i) * p.hq + h;
+        const unsigned char* rows = (const unsigned char*)p.part_o + e0 * 512 + lane * 8;
+        pdl_wait();   // the partials are complete
+        // Every load is issued before the first use of any of them: volatile loads keep their place in the instruction stream
+        // (left to itself the compiler moved the row loads behind the reduction of the maxima, i.e. behind a first trip to
+        // memory: 0.6 us on decode verify).  No branch between the loads: slots past the last split repeat its row, and weigh
+        // nothing below.
+        uint2 v[kNsMax];
 #pragma unroll
-    for (int k = 0; k < kNsMax; ++k) v[k] = __ldcg((const uint2*)(rows + min(k, ns - 1) * 512));
-    float m_all = ml.x;
+        for (int k = 0; k < kNsMax; ++k) v[k] = ld_volatile_u2(rows + min(k, ns - 1) * 512);
+        float2 ml = make_float2(-INFINITY, 0.f);
+        if (lane < ns) ml = ld_volatile_f2(p.part_ml + e0 + lane);
+        float m_all = ml.x;
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, off));
-    const float w_mine = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m_all) * ml.y;   // 0 in lanes past the last split
-    float l_all = w_mine;
+        for (int off = 16; off > 0; off >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xFFFFFFFFu, m_all, off));
+        const float w_mine = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m_all) * ml.y;   // 0 in lanes past the last split
+        float l_all = w_mine;
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xFFFFFFFFu, l_all, off);   // (a fixed order: reproducible)
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int off = 16; off > 0; off >>= 1) l_all += __shfl_xor_sync(0xFFFFFFFFu, l_all, off);   // (a fixed order: reproducible)
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int k = 0; k < kNsMax; ++k) {
-        const float w = __shfl_sync(0xFFFFFFFFu, w_mine, k);
-        // a split that saw no token for this row publishes only (m, l) = (-inf, 0): its row may hold anything, NaN included
-        const bool use = w != 0.f;
-        const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&v[k].x));
-        const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&v[k].y));
-        acc.x += use ? a.x * w : 0.f; acc.y += use ? a.y * w : 0.f; acc.z += use ? b.x * w : 0.f; acc.w += use ? b.y * w : 0.f;
+        for (int k = 0; k < kNsMax; ++k) {
+            const float w = __shfl_sync(0xFFFFFFFFu, w_mine, k);
+            // a split that saw no token for this row publishes only (m, l) = (-inf, 0): its row may hold anything, NaN included
+            const bool use = w != 0.f;
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&v[k].x));
+            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&v[k].y));
+            acc.x += use ? a.x * w : 0.f; acc.y += use ? a.y * w : 0.f; acc.z += use ? b.x * w : 0.f; acc.w += use ? b.y * w : 0.f;
+        }
+        const float inv = 1.f / l_all;
+        uint2 packed;
+        packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+        packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+        *(uint2*)((__nv_bfloat16*)p.out + out_off * kD + lane * 4) = packed;
+        if (p.lse && lane == 0) p.lse[out_off] = (m_all + log2f(l_all)) * 0.6931471805599453f;
     }
-    const float inv = 1.f / l_all;
-    uint2 packed;
-    packed.x = pack_bf16(acc.x * inv, acc.y * inv);
-    packed.y = pack_bf16(acc.z * inv, acc.w * inv);
-    *(uint2*)((__nv_bfloat16*)p.out + out_off * kD + lane * 4) = packed;
-    if (p.lse && lane == 0) p.lse[out_off] = (m_all + log2f(l_all)) * 0.6931471805599453f;
 }
 
 // --------------------------------------------------------------------------------------------
