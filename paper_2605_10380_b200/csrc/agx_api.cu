@@ -162,6 +162,12 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
         groups[k].push_back(s);
     }
     const int small_kw = h->small_kw ? h->small_kw : (warp_mma_seqs >= 2 && warp_mma_tokens * c.num_kv_heads / 8 >= 8192) ? 4 : 8;
+    // Work items are handed to the SMs in launch order: the sequences with the longest contexts go first, so that the
+    // longest items of a ragged batch are not the ones left over for the last wave (env AGX_LONGEST_FIRST=0 keeps the batch order).
+    static const bool longest_first = !(getenv("AGX_LONGEST_FIRST") && atoi(getenv("AGX_LONGEST_FIRST")) == 0);
+    if (longest_first)
+        for (int k : {(int)KIND_TILE, (int)KIND_STREAM})
+            std::stable_sort(groups[k].begin(), groups[k].end(), [&](int a, int b) { return P[a] + Q[a] > P[b] + Q[b]; });
     for (int k = 0; k < KIND_COUNT; ++k) {
         const std::vector<int>& seqs = groups[k];
         if (seqs.empty()) continue;
