@@ -196,6 +196,7 @@ struct TileItem {
 struct EpiCtx {
     TileItem it;
     int part_base, hq;
+    int part_half;   // split partials leave as fp16 rows divided by their own sums (always so on the 256-row schedule)
     void* out;
     float* part_o;
     float2* part_ml;
@@ -313,7 +314,8 @@ __device__ __noinline__ void tile_epilogue(unsigned char* smem, uint32_t tO, flo
                     oreg[4 * v + 3] = __float_as_uint(__uint_as_float(oreg[4 * v + 3]) * w_own + (w_other != 0.f ? o1.w * w_other : 0.f));
                 }
             }
-            if (single || !kStreams) {   // (the 256-row schedule normalises its split partials too: they leave as fp16)
+            const bool half_part = kStreams && !single && cx.part_half;
+            if (single || !kStreams || half_part) {   // (the 256-row schedule normalises its split partials too: they leave as fp16)
 #pragma unroll
                 for (int c = 0; c < 64; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * inv);
             }
@@ -328,6 +330,11 @@ __device__ __noinline__ void tile_epilogue(unsigned char* smem, uint32_t tO, flo
                             pk.x = pack_bf16(__uint_as_float(oreg[4 * v]), __uint_as_float(oreg[4 * v + 1]));
                             pk.y = pack_bf16(__uint_as_float(oreg[4 * v + 2]), __uint_as_float(oreg[4 * v + 3]));
                             *(uint2*)((unsigned char*)row_dst + (c8 * 8 + v) * 8) = pk;
+                        } else if (half_part) {
+                            uint2 pk;
+                            pk.x = pack_f16(__uint_as_float(oreg[4 * v]), __uint_as_float(oreg[4 * v + 1]));
+                            pk.y = pack_f16(__uint_as_float(oreg[4 * v + 2]), __uint_as_float(oreg[4 * v + 3]));
+                            __stcg((uint2*)((unsigned char*)row_dst + (c8 * 8 + v) * 8), pk);
                         } else {
                             __stcg((uint4*)((unsigned char*)row_dst + (c8 * 8 + v) * 16),
                                    make_uint4(oreg[4 * v], oreg[4 * v + 1], oreg[4 * v + 2], oreg[4 * v + 3]));
@@ -667,6 +674,7 @@ attn_tile_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constan
         cx->part_base = sp.part_base; cx->hq = p.hq;
         cx->out = p.out; cx->part_o = p.part_o; cx->part_ml = p.part_ml; cx->lse = p.lse;
         cx->magic = p.row_div_magic;
+        cx->part_half = p.part_half;
         mbar_arrive(bar(BAR_CTX));   // (release) the epilogue waits on this before it reads the context
     }
     } else {
