@@ -267,7 +267,15 @@ AGX_API agx_status agx_get_status(agx_handle* handle, void* stream, int32_t* dev
  *   h_accept_len, h_next_token, h_seq_lens : host int32 [B]; h_seq_lens receives
  *                                prefix_len + accept_len + 1
  *   vocab == 0                 : attention only (a middle layer of a model): the logits, drafts
- *                                and accept outputs are ignored and may be NULL
+ *                                and accept outputs are ignored and may be NULL.  Such a step that moves
+ *                                4 MiB or more runs as chunked prefill: every block is cut into chunks of 384
+ *                                rows (environment variable AGX_HOST_PIPELINE_ROWS, 0 = never), rows
+ *                                [r0, r1) of a block being a block of their own behind a prefix longer by r0;
+ *                                the uploads of a chunk, the attention calls of the chunks before it and the
+ *                                downloads of their rows overlap on two streams the handle owns, which start
+ *                                behind the work already on `stream` and which `stream` waits for at the end
+ *                                of the call.  Results are those of the single call; on an error in the middle
+ *                                the chunks already enqueued still run.
  *   workspace                  : device, >= agx_verify_step_host_workspace_bytes(...) bytes,
  *                                256-byte aligned; holds the staged copies and both scratch areas
  * Errors: as the three calls; nothing is launched when a check fails.

@@ -53,6 +53,11 @@ struct agx_handle {
     int drop_stage;         // AGX_OPT_TEST_DROP_STAGE (-1 = none)
     std::unordered_map<const void*, PoolMap> pool_maps;
     std::vector<int32_t> cu_host;  // staging for agx_verify_step_host (lives until its final sync)
+    // Large attention-only host steps run as a pipeline of row chunks: uploads on one stream of the handle's own, the
+    // attention calls on the caller's stream, downloads on a third (env AGX_HOST_PIPELINE_ROWS: rows per chunk, 0 = off).
+    int pipe_rows;
+    cudaStream_t pipe_in, pipe_out;
+    std::vector<cudaEvent_t> pipe_events;
     // the launch plan of the last batch seen: the layers of a model step all ask for the same one
     Plan* plan_cache;
     std::vector<int32_t> plan_P, plan_Q;
@@ -395,6 +400,9 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     h->stream_max_rows = env ? atoi(env) : 384;
     env = getenv("AGX_CLUSTER_MERGE");
     h->cluster_merge = !(env && atoi(env) == 0);
+    env = getenv("AGX_HOST_PIPELINE_ROWS");
+    h->pipe_rows = env ? std::max(0, atoi(env)) : 384;   // measured on the long-context step: 256 / 384 / 512 / 768 / 1024 rows -> 1.54 / 1.43 / 1.57 / 1.56 / 1.72 ms
+    h->pipe_in = h->pipe_out = nullptr;
     env = getenv("AGX_MERGE_SMS");
     h->merge_sms = !(env && atoi(env) == 0);
     env = getenv("AGX_ZERO_COPY");
@@ -428,6 +436,9 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
 agx_status agx_destroy(agx_handle* h) {
     if (!h) return AGX_E_INVAL;
     cudaFree(h->d_status);
+    if (h->pipe_in) cudaStreamDestroy(h->pipe_in);
+    if (h->pipe_out) cudaStreamDestroy(h->pipe_out);
+    for (cudaEvent_t ev : h->pipe_events) cudaEventDestroy(ev);
     delete h->plan_cache;
     delete h;
     return AGX_OK;
@@ -677,6 +688,17 @@ void* mapped_alias(const void* host) {
     return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
 }
 
+// Attention-only host steps that move a few megabytes or more are cut into row chunks whose transfers overlap the
+// attention calls of the other chunks (chunked prefill: rows [r0, r1) of a block are a block of their own behind a prefix
+// longer by r0, since the chunks before them have appended their K/V by then).
+bool host_step_pipelined(const agx_handle* h, int B, const int32_t* Q, int vocab) {
+    if (vocab > 0 || h->pipe_rows <= 0) return false;
+    long long tq = 0;
+    for (int s = 0; s < B; ++s) tq += Q[s];
+    const long long in_bytes = tq * (h->cfg.num_q_heads + 2 * h->cfg.num_kv_heads) * h->cfg.head_dim * elem_size(h->cfg.dtype);
+    return in_bytes >= (4ll << 20) && tq > h->pipe_rows;
+}
+
 struct HostStepLayout {
     size_t q, k, v, out, logits, drafts, prefix, cu, acc, next, seqlen, attn_ws, accept_ws, total;
     size_t q_bytes, kv_bytes, logits_bytes, attn_ws_bytes, accept_ws_bytes;
@@ -698,8 +720,20 @@ agx_status host_step_layout(agx_handle* h, int B, const int32_t* P, const int32_
         tq += Q[s];
     }
     if (tq > 65535) return fail(h, AGX_E_RANGE, "more than 65535 rows in one host step");
-    const int64_t aws = agx_attn_workspace_bytes(h, B, P, Q);
-    if (aws < 0) return (agx_status)aws;
+    int64_t aws = 0;
+    if (host_step_pipelined(h, B, Q, vocab)) {
+        // one attention call per (sequence, row chunk), one after the other on the caller's stream: the largest workspace of them
+        for (int s = 0; s < B; ++s)
+            for (int r0 = 0; r0 < Q[s]; r0 += h->pipe_rows) {
+                const int32_t pc = P[s] + r0, qc = std::min(h->pipe_rows, Q[s] - r0);
+                const int64_t w = agx_attn_workspace_bytes(h, 1, &pc, &qc);
+                if (w < 0) return (agx_status)w;
+                aws = std::max(aws, w);
+            }
+    } else {
+        aws = agx_attn_workspace_bytes(h, B, P, Q);
+        if (aws < 0) return (agx_status)aws;
+    }
     const int64_t cws = with_accept ? agx_accept_workspace_bytes(h, (int)tq, vocab) : 0;
     if (cws < 0) return (agx_status)cws;
     const size_t es = elem_size(h->cfg.dtype);
@@ -750,6 +784,60 @@ static agx_status verify_step_host_impl(agx_handle* h, void* k_pool, void* v_poo
         return fail(h, AGX_E_INVAL, "host-step workspace missing, misaligned or too small (%zu needed)", L.total);
     cudaStream_t stream = (cudaStream_t)stream_v;
     char* ws = (char*)workspace;
+    if (host_step_pipelined(h, B, Q, vocab)) {
+        cudaError_t pe = cudaSuccess;
+        if (!h->pipe_in) pe = cudaStreamCreateWithFlags(&h->pipe_in, cudaStreamNonBlocking);
+        if (pe == cudaSuccess && !h->pipe_out) pe = cudaStreamCreateWithFlags(&h->pipe_out, cudaStreamNonBlocking);
+        size_t chunks = 0;
+        for (int s = 0; s < B; ++s) chunks += (size_t)(Q[s] + h->pipe_rows - 1) / h->pipe_rows;
+        while (pe == cudaSuccess && h->pipe_events.size() < 2 * chunks + 2) {
+            cudaEvent_t ev;
+            pe = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+            if (pe == cudaSuccess) h->pipe_events.push_back(ev);
+        }
+        if (pe != cudaSuccess) return cuda_fail(h, pe, "host step: pipeline set-up");
+        const size_t es = elem_size(h->cfg.dtype);
+        const size_t q_row = (size_t)h->cfg.num_q_heads * h->cfg.head_dim * es, kv_row = (size_t)h->cfg.num_kv_heads * h->cfg.head_dim * es;
+        cudaEvent_t fork = h->pipe_events[2 * chunks], join = h->pipe_events[2 * chunks + 1];
+        // the side streams start behind whatever the caller has already put on its stream ...
+        pe = cudaEventRecord(fork, stream);
+        if (pe == cudaSuccess) pe = cudaStreamWaitEvent(h->pipe_in, fork, 0);
+        if (pe == cudaSuccess) pe = cudaStreamWaitEvent(h->pipe_out, fork, 0);
+        int launches = 0;
+        size_t i = 0, row0 = 0;
+        for (int s = 0; s < B && pe == cudaSuccess; ++s) {
+            for (int r0 = 0; r0 < Q[s] && pe == cudaSuccess; r0 += h->pipe_rows, ++i) {
+                const int32_t pc = P[s] + r0, qc = std::min(h->pipe_rows, Q[s] - r0);
+                const size_t r = row0 + r0;
+                cudaEvent_t in_done = h->pipe_events[2 * i], out_ready = h->pipe_events[2 * i + 1];
+                pe = cudaMemcpyAsync(ws + L.q + r * q_row, (const char*)h_q + r * q_row, qc * q_row, cudaMemcpyHostToDevice, h->pipe_in);
+                if (pe == cudaSuccess) pe = cudaMemcpyAsync(ws + L.k + r * kv_row, (const char*)h_k + r * kv_row, qc * kv_row, cudaMemcpyHostToDevice, h->pipe_in);
+                if (pe == cudaSuccess) pe = cudaMemcpyAsync(ws + L.v + r * kv_row, (const char*)h_v + r * kv_row, qc * kv_row, cudaMemcpyHostToDevice, h->pipe_in);
+                if (pe == cudaSuccess) pe = cudaEventRecord(in_done, h->pipe_in);
+                if (pe == cudaSuccess) pe = cudaStreamWaitEvent(stream, in_done, 0);
+                if (pe != cudaSuccess) break;
+                st = agx_attn_prefixed_append(h, ws + L.q + r * q_row, ws + L.k + r * kv_row, ws + L.v + r * kv_row, k_pool, v_pool,
+                                              num_pages, page_table + (size_t)s * pt_stride, pt_stride, &pc, &qc, 1, ws + L.out + r * q_row,
+                                              nullptr, L.attn_ws_bytes ? ws + L.attn_ws : nullptr, L.attn_ws_bytes, stream);
+                if (st != AGX_OK) break;
+                launches += h->last_launches;
+                pe = cudaEventRecord(out_ready, stream);
+                if (pe == cudaSuccess) pe = cudaStreamWaitEvent(h->pipe_out, out_ready, 0);
+                if (pe == cudaSuccess) pe = cudaMemcpyAsync((char*)h_out + r * q_row, ws + L.out + r * q_row, qc * q_row, cudaMemcpyDeviceToHost, h->pipe_out);
+            }
+            row0 += Q[s];
+        }
+        // ... and the caller's stream ends behind the last download (also when a call in the middle failed: the join still
+        // has to bring the side streams back, or a stream capture of the caller's would be left forked)
+        cudaError_t je = cudaEventRecord(join, h->pipe_out);
+        if (je == cudaSuccess) je = cudaStreamWaitEvent(stream, join, 0);
+        if (st != AGX_OK) return st;
+        if (pe == cudaSuccess) pe = je;
+        if (pe == cudaSuccess && sync) pe = cudaStreamSynchronize(stream);
+        if (pe != cudaSuccess) return cuda_fail(h, pe, "host step: pipelined transfers");
+        h->last_launches = launches;
+        return AGX_OK;
+    }
     std::vector<int32_t>& cu = h->cu_host;  // outlives the asynchronous copy (the call ends with a sync)
     cu.assign(B + 1, 0);
     for (int s = 0; s < B; ++s) cu[s + 1] = cu[s] + Q[s];

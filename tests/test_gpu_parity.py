@@ -553,6 +553,32 @@ def test_verify_step_host_matches_oracle(enqueue_only, memory, monkeypatch):
     assert np.array_equal(h_acc.numpy(), al) and np.array_equal(h_nxt.numpy(), nt) and np.array_equal(h_sl.numpy(), sl)
 
 
+@pytest.mark.parametrize("enqueue_only,rows", [(False, None), (True, None), (True, "200"), (True, "0")])
+def test_attention_only_host_step_in_row_chunks_matches_oracle(enqueue_only, rows, monkeypatch):
+    """A host step that moves several megabytes and has no accept part runs as a pipeline of row chunks (chunked
+    prefill: uploads, attention calls and downloads of different chunks overlap on streams of the handle's own).  Two
+    ragged blocks whose last chunks are short, default chunk length, a shorter one and the pipeline switched off: the
+    pools and every output row against the oracle, and a second step on the same handle right behind the first."""
+    if rows is not None:
+        monkeypatch.setenv("AGX_HOST_PIPELINE_ROWS", rows)
+    w = W.make_attn_workload("host_chunks", 91, "bf16", 32, 8, 128, [1000, 333], [700, 600], spare_pages=2)
+    b = DeviceBatch(w)
+    to_t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).view(torch.bfloat16).pin_memory()
+    hq, hk, hv = to_t(w.q_block), to_t(w.k_new), to_t(w.v_new)
+    n = b.h.verify_step_host_workspace_bytes(w.prefix_len, w.q_len, "bf16", 0, 0)
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+    kp, vp = oracle_pools_after_append(w)
+    ref, _ = oracle.attn_paged_batch(w.q_block, kp, vp, w.page_table, "bf16", w.prefix_len, w.q_len, w.cu_q)
+    for step in range(2):
+        h_out = torch.zeros((w.total_q, 32, 128), dtype=torch.bfloat16).pin_memory()
+        b.h.verify_step_host(b.k_pool, b.v_pool, b.page_table, w.prefix_len, w.q_len, hq, hk, hv, None, "bf16", 0, 0,
+                             None, h_out, None, None, None, ws, enqueue_only=enqueue_only)
+        torch.cuda.synchronize()
+        assert b.status() == 0
+        assert np.array_equal(host_storage(b.k_pool, "bf16"), kp) and np.array_equal(host_storage(b.v_pool, "bf16"), vp)
+        check_attention(h_out.to(torch.float64).numpy(), ref, f"host step in row chunks, step {step}")
+
+
 def test_verify_step_host_with_more_sequences_than_one_launch_holds():
     """60 sequences through the host-buffer step: lengths travel by copy instead of kernel arguments, attention takes
     several launches."""
