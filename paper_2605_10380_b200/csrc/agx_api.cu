@@ -866,7 +866,24 @@ static agx_status verify_step_host_impl(agx_handle* h, void* k_pool, void* v_poo
     } else {
         h2d(L.q, h_q, L.q_bytes); h2d(L.k, h_k, L.kv_bytes); h2d(L.v, h_v, L.kv_bytes);
     }
-    if (with_accept) {
+    // The logits are needed by the accept step only: a megabyte or more of them crosses on a stream of the handle's own,
+    // beside the attention kernels, and the caller's stream waits for that copy just before the accept launch.
+    cudaEvent_t logits_done = nullptr;
+    if (with_accept && L.logits_bytes >= (1u << 20) && h->pipe_rows > 0 && e == cudaSuccess) {
+        if (!h->pipe_in) e = cudaStreamCreateWithFlags(&h->pipe_in, cudaStreamNonBlocking);
+        while (e == cudaSuccess && h->pipe_events.size() < 2) {
+            cudaEvent_t ev;
+            e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+            if (e == cudaSuccess) h->pipe_events.push_back(ev);
+        }
+        if (e == cudaSuccess) e = cudaEventRecord(h->pipe_events[0], stream);   // behind whatever last used the workspace
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(h->pipe_in, h->pipe_events[0], 0);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(ws + L.logits, h_logits, L.logits_bytes, cudaMemcpyHostToDevice, h->pipe_in);
+        if (e == cudaSuccess && L.total_q > B)
+            e = cudaMemcpyAsync(ws + L.drafts, h_drafts, (size_t)(L.total_q - B) * 4, cudaMemcpyHostToDevice, h->pipe_in);
+        if (e == cudaSuccess) e = cudaEventRecord(h->pipe_events[1], h->pipe_in);
+        if (e == cudaSuccess) logits_done = h->pipe_events[1];
+    } else if (with_accept) {
         h2d(L.logits, h_logits, L.logits_bytes);
         h2d(L.drafts, h_drafts, (size_t)(L.total_q - B) * 4);
     }
@@ -889,8 +906,12 @@ static agx_status verify_step_host_impl(agx_handle* h, void* k_pool, void* v_poo
     st = agx_attn_prefixed_append(h, ws + L.q, ws + L.k, ws + L.v, k_pool, v_pool, num_pages, page_table, pt_stride, P, Q,
                                   B, out_dev, nullptr, L.attn_ws_bytes ? ws + L.attn_ws : nullptr, L.attn_ws_bytes,
                                   stream);
+    if (st == AGX_OK) launches += h->last_launches;
+    if (logits_done) {   // (also when the attention call failed: the side stream is brought back before the call returns)
+        e = cudaStreamWaitEvent(stream, logits_done, 0);
+        if (e != cudaSuccess) return cuda_fail(h, e, "host step: logits upload");
+    }
     if (st != AGX_OK) return st;
-    launches += h->last_launches;
     if (with_accept) {
         st = agx_accept_greedy(h, ws + L.logits, logits_dtype, row_stride, vocab, (const int32_t*)(ws + L.drafts),
                                (const int32_t*)(ws + L.cu), B, L.total_q, (int32_t*)(ws + L.acc),
