@@ -261,7 +261,10 @@ AGX_API agx_status agx_get_status(agx_handle* handle, void* stream, int32_t* dev
  *                                kernel reads them across the bus instead of three transfers; a
  *                                pinned, mapped h_out of at most 1 MiB is written by the attention
  *                                kernels directly.  Results are the same either way.
- *   h_logits                   : host, [total_q][row_stride] of logits_dtype
+ *   h_logits                   : host, [total_q][row_stride] of logits_dtype; a megabyte or more of them is
+ *                                uploaded on a stream the handle owns, beside the attention kernels (it starts
+ *                                behind the work already on `stream`, and `stream` waits for it before the
+ *                                accept step)
  *   h_drafts                   : host int32 [total_q - B] (may be NULL when total_q == B)
  *   h_out                      : host, [total_q][num_q_heads][head_dim]
  *   h_accept_len, h_next_token, h_seq_lens : host int32 [B]; h_seq_lens receives
