@@ -753,9 +753,9 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
 }
 
 // The same merge for the partials of the 256-row tensor-core schedule (fp16 rows divided by their own sums, at most 4
-// splits): one wave of CTAs, each warp taking up to three (row, head) pairs with all their loads in flight at once, so
-// that the merge of a split prefill (12288 pairs, 9 MB of partials) is one memory round trip per warp instead of
-// several waves of short-lived CTAs.
+// splits): each warp takes up to three (row, head) pairs with all their loads in flight at once, so that the merge of
+// a split prefill (12288 pairs, 9 MB of partials) is one wave of CTAs and one memory round trip per warp instead of
+// several waves of short-lived CTAs, and a larger merge has a third of the CTAs with three times the bytes in flight each.
 constexpr int kCombineRows = 3;
 __global__ void __launch_bounds__(128, 8)
 attn_combine_half4_kernel(const __grid_constant__ AttnParams p, int total_rows) {
@@ -988,12 +988,10 @@ cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, 
     for (int i = 0; i < p.num_seqs; ++i) ns_max = p.seq[i].nsplit > ns_max ? p.seq[i].nsplit : ns_max;
     if (dtype == AGX_BF16 && p.part_half) {
         if (ns_max <= 4) {
-            int device = 0, sms = 0;
-            if (cudaGetDevice(&device) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
-                return cudaErrorInvalidDevice;
-            const int one_wave = sms * 8;
-            const int want = (int)((n + 4 * kCombineRows - 1) / (4 * kCombineRows));   // CTAs whose warps take kCombineRows pairs each
-            return launch_chained(attn_combine_half4_kernel, dim3(want > one_wave ? blocks : (want > 0 ? want : 1)), dim3(128), 0, stream, p, total_rows);
+            // CTAs whose warps take kCombineRows pairs each (under ncu on the long prefill, 65536 pairs: 20.5-21.6 us against 29.1 us
+            // for four times as many CTAs of one pair per warp)
+            const int want = (int)((n + 4 * kCombineRows - 1) / (4 * kCombineRows));
+            return launch_chained(attn_combine_half4_kernel, dim3(want > 0 ? want : 1), dim3(128), 0, stream, p, total_rows);
         }
         if (ns_max <= 32) {
             if (ns_max <= 8) return launch_chained(attn_combine_half32_kernel<8>, dim3((int)((n + 1) / 2)), dim3(64), 0, stream, p, total_rows);
