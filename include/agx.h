@@ -271,11 +271,13 @@ AGX_API agx_status agx_get_status(agx_handle* handle, void* stream, int32_t* dev
  *                                prefix_len + accept_len + 1
  *   vocab == 0                 : attention only (a middle layer of a model): the logits, drafts
  *                                and accept outputs are ignored and may be NULL.  Such a step that moves
- *                                4 MiB or more runs as chunked prefill: every block is cut into chunks of 384
- *                                rows (environment variable AGX_HOST_PIPELINE_ROWS, 0 = never), rows
- *                                [r0, r1) of a block being a block of their own behind a prefix longer by r0;
- *                                the uploads of a chunk, the attention calls of the chunks before it and the
- *                                downloads of their rows overlap on two streams the handle owns, which start
+ *                                4 MiB or more is cut into several attention calls: runs of whole blocks of
+ *                                about a thousand rows, or, where that gives fewer than three calls, chunks of
+ *                                384 rows of a block (environment variable AGX_HOST_PIPELINE_ROWS, 0 = never
+ *                                cut), rows [r0, r1) of a block being a block of their own behind a prefix longer
+ *                                by r0 (chunked prefill); the uploads of a chunk, the attention calls of the chunks
+ *                                before it and the downloads of their rows overlap on two streams the handle owns,
+ *                                which start
  *                                behind the work already on `stream` and which `stream` waits for at the end
  *                                of the call.  Results are those of the single call; on an error in the middle
  *                                the chunks already enqueued still run.

@@ -699,6 +699,40 @@ bool host_step_pipelined(const agx_handle* h, int B, const int32_t* Q, int vocab
     return in_bytes >= (4ll << 20) && tq > h->pipe_rows;
 }
 
+// The attention calls of a pipelined host step: runs of whole blocks that together have about a thousand rows, and
+// blocks longer than that in row chunks of pipe_rows rows.
+struct HostChunk {
+    int s0, nseq;      // sequences [s0, s0 + nseq)
+    int r0, rows;      // nseq == 1: rows [r0, r0 + rows) of the block; otherwise r0 = 0 and rows = all rows of the run
+    size_t row_begin;  // first row of the chunk in the step's row order
+};
+void host_step_chunks(const agx_handle* h, int B, const int32_t* Q, std::vector<HostChunk>& out) {
+    // Runs of whole blocks of about a thousand rows (measured on the ragged prefill blocks of c4, runs of 384 / 512 / 768 / 1024 rows:
+    // 1.94 / 1.97 / 1.81 / 1.77 ms per step).  When that gives fewer than three calls there is nothing to overlap: blocks on their
+    // own are then cut into row chunks (the 512-row block of c3 as one call 1.68 ms per 8 layers, as 384 + 128 rows 1.54 ms; with
+    // many runs the cut only adds calls: c4 1.93 ms).
+    const int run_rows = std::max(1024, 2 * h->pipe_rows);
+    std::vector<HostChunk> runs;
+    size_t row = 0;
+    int s = 0;
+    while (s < B) {
+        HostChunk c = {s, 0, 0, 0, row};
+        while (s < B && c.nseq < kMaxSeqs && (c.nseq == 0 || c.rows + Q[s] <= run_rows)) {
+            c.rows += Q[s]; row += Q[s]; ++c.nseq; ++s;
+        }
+        runs.push_back(c);
+    }
+    out.clear();
+    for (const HostChunk& c : runs) {
+        if (runs.size() < 3 && c.nseq == 1 && c.rows > h->pipe_rows) {
+            for (int r0 = 0; r0 < c.rows; r0 += h->pipe_rows)
+                out.push_back({c.s0, 1, r0, std::min(h->pipe_rows, c.rows - r0), c.row_begin + (size_t)r0});
+        } else {
+            out.push_back(c);
+        }
+    }
+}
+
 struct HostStepLayout {
     size_t q, k, v, out, logits, drafts, prefix, cu, acc, next, seqlen, attn_ws, accept_ws, total;
     size_t q_bytes, kv_bytes, logits_bytes, attn_ws_bytes, accept_ws_bytes;
@@ -722,14 +756,15 @@ agx_status host_step_layout(agx_handle* h, int B, const int32_t* P, const int32_
     if (tq > 65535) return fail(h, AGX_E_RANGE, "more than 65535 rows in one host step");
     int64_t aws = 0;
     if (host_step_pipelined(h, B, Q, vocab)) {
-        // one attention call per (sequence, row chunk), one after the other on the caller's stream: the largest workspace of them
-        for (int s = 0; s < B; ++s)
-            for (int r0 = 0; r0 < Q[s]; r0 += h->pipe_rows) {
-                const int32_t pc = P[s] + r0, qc = std::min(h->pipe_rows, Q[s] - r0);
-                const int64_t w = agx_attn_workspace_bytes(h, 1, &pc, &qc);
-                if (w < 0) return (agx_status)w;
-                aws = std::max(aws, w);
-            }
+        // one attention call per chunk, one after the other on the caller's stream: the largest workspace of them
+        std::vector<HostChunk> chunks;
+        host_step_chunks(h, B, Q, chunks);
+        for (const HostChunk& c : chunks) {
+            const int32_t pc = P[c.s0] + c.r0, qc = c.rows;
+            const int64_t w = c.nseq == 1 ? agx_attn_workspace_bytes(h, 1, &pc, &qc) : agx_attn_workspace_bytes(h, c.nseq, P + c.s0, Q + c.s0);
+            if (w < 0) return (agx_status)w;
+            aws = std::max(aws, w);
+        }
     } else {
         aws = agx_attn_workspace_bytes(h, B, P, Q);
         if (aws < 0) return (agx_status)aws;
@@ -788,8 +823,9 @@ static agx_status verify_step_host_impl(agx_handle* h, void* k_pool, void* v_poo
         cudaError_t pe = cudaSuccess;
         if (!h->pipe_in) pe = cudaStreamCreateWithFlags(&h->pipe_in, cudaStreamNonBlocking);
         if (pe == cudaSuccess && !h->pipe_out) pe = cudaStreamCreateWithFlags(&h->pipe_out, cudaStreamNonBlocking);
-        size_t chunks = 0;
-        for (int s = 0; s < B; ++s) chunks += (size_t)(Q[s] + h->pipe_rows - 1) / h->pipe_rows;
+        std::vector<HostChunk> list;
+        host_step_chunks(h, B, Q, list);
+        const size_t chunks = list.size();
         while (pe == cudaSuccess && h->pipe_events.size() < 2 * chunks + 2) {
             cudaEvent_t ev;
             pe = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
@@ -804,28 +840,26 @@ static agx_status verify_step_host_impl(agx_handle* h, void* k_pool, void* v_poo
         if (pe == cudaSuccess) pe = cudaStreamWaitEvent(h->pipe_in, fork, 0);
         if (pe == cudaSuccess) pe = cudaStreamWaitEvent(h->pipe_out, fork, 0);
         int launches = 0;
-        size_t i = 0, row0 = 0;
-        for (int s = 0; s < B && pe == cudaSuccess; ++s) {
-            for (int r0 = 0; r0 < Q[s] && pe == cudaSuccess; r0 += h->pipe_rows, ++i) {
-                const int32_t pc = P[s] + r0, qc = std::min(h->pipe_rows, Q[s] - r0);
-                const size_t r = row0 + r0;
-                cudaEvent_t in_done = h->pipe_events[2 * i], out_ready = h->pipe_events[2 * i + 1];
-                pe = cudaMemcpyAsync(ws + L.q + r * q_row, (const char*)h_q + r * q_row, qc * q_row, cudaMemcpyHostToDevice, h->pipe_in);
-                if (pe == cudaSuccess) pe = cudaMemcpyAsync(ws + L.k + r * kv_row, (const char*)h_k + r * kv_row, qc * kv_row, cudaMemcpyHostToDevice, h->pipe_in);
-                if (pe == cudaSuccess) pe = cudaMemcpyAsync(ws + L.v + r * kv_row, (const char*)h_v + r * kv_row, qc * kv_row, cudaMemcpyHostToDevice, h->pipe_in);
-                if (pe == cudaSuccess) pe = cudaEventRecord(in_done, h->pipe_in);
-                if (pe == cudaSuccess) pe = cudaStreamWaitEvent(stream, in_done, 0);
-                if (pe != cudaSuccess) break;
-                st = agx_attn_prefixed_append(h, ws + L.q + r * q_row, ws + L.k + r * kv_row, ws + L.v + r * kv_row, k_pool, v_pool,
-                                              num_pages, page_table + (size_t)s * pt_stride, pt_stride, &pc, &qc, 1, ws + L.out + r * q_row,
-                                              nullptr, L.attn_ws_bytes ? ws + L.attn_ws : nullptr, L.attn_ws_bytes, stream);
-                if (st != AGX_OK) break;
-                launches += h->last_launches;
-                pe = cudaEventRecord(out_ready, stream);
-                if (pe == cudaSuccess) pe = cudaStreamWaitEvent(h->pipe_out, out_ready, 0);
-                if (pe == cudaSuccess) pe = cudaMemcpyAsync((char*)h_out + r * q_row, ws + L.out + r * q_row, qc * q_row, cudaMemcpyDeviceToHost, h->pipe_out);
-            }
-            row0 += Q[s];
+        for (size_t i = 0; i < chunks && pe == cudaSuccess; ++i) {
+            const HostChunk& c = list[i];
+            const int32_t pc = P[c.s0] + c.r0, qc = c.rows;
+            const size_t r = c.row_begin, n = (size_t)c.rows;
+            cudaEvent_t in_done = h->pipe_events[2 * i], out_ready = h->pipe_events[2 * i + 1];
+            pe = cudaMemcpyAsync(ws + L.q + r * q_row, (const char*)h_q + r * q_row, n * q_row, cudaMemcpyHostToDevice, h->pipe_in);
+            if (pe == cudaSuccess) pe = cudaMemcpyAsync(ws + L.k + r * kv_row, (const char*)h_k + r * kv_row, n * kv_row, cudaMemcpyHostToDevice, h->pipe_in);
+            if (pe == cudaSuccess) pe = cudaMemcpyAsync(ws + L.v + r * kv_row, (const char*)h_v + r * kv_row, n * kv_row, cudaMemcpyHostToDevice, h->pipe_in);
+            if (pe == cudaSuccess) pe = cudaEventRecord(in_done, h->pipe_in);
+            if (pe == cudaSuccess) pe = cudaStreamWaitEvent(stream, in_done, 0);
+            if (pe != cudaSuccess) break;
+            st = agx_attn_prefixed_append(h, ws + L.q + r * q_row, ws + L.k + r * kv_row, ws + L.v + r * kv_row, k_pool, v_pool, num_pages,
+                                          page_table + (size_t)c.s0 * pt_stride, pt_stride, c.nseq == 1 ? &pc : P + c.s0,
+                                          c.nseq == 1 ? &qc : Q + c.s0, c.nseq, ws + L.out + r * q_row, nullptr,
+                                          L.attn_ws_bytes ? ws + L.attn_ws : nullptr, L.attn_ws_bytes, stream);
+            if (st != AGX_OK) break;
+            launches += h->last_launches;
+            pe = cudaEventRecord(out_ready, stream);
+            if (pe == cudaSuccess) pe = cudaStreamWaitEvent(h->pipe_out, out_ready, 0);
+            if (pe == cudaSuccess) pe = cudaMemcpyAsync((char*)h_out + r * q_row, ws + L.out + r * q_row, n * q_row, cudaMemcpyDeviceToHost, h->pipe_out);
         }
         // ... and the caller's stream ends behind the last download (also when a call in the middle failed: the join still
         // has to bring the side streams back, or a stream capture of the caller's would be left forked)

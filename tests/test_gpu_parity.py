@@ -556,12 +556,13 @@ def test_verify_step_host_matches_oracle(enqueue_only, memory, monkeypatch):
 @pytest.mark.parametrize("enqueue_only,rows", [(False, None), (True, None), (True, "200"), (True, "0")])
 def test_attention_only_host_step_in_row_chunks_matches_oracle(enqueue_only, rows, monkeypatch):
     """A host step that moves several megabytes and has no accept part runs as a pipeline of row chunks (chunked
-    prefill: uploads, attention calls and downloads of different chunks overlap on streams of the handle's own).  Two
-    ragged blocks whose last chunks are short, default chunk length, a shorter one and the pipeline switched off: the
-    pools and every output row against the oracle, and a second step on the same handle right behind the first."""
+    prefill: uploads, attention calls and downloads of different chunks overlap on streams of the handle's own).  A
+    block long enough to be cut into row chunks with a short last one, a run of two short blocks that share a call and
+    a block on its own; default chunk length, a shorter one and the pipeline switched off: the pools and every output
+    row against the oracle, and a second step on the same handle right behind the first."""
     if rows is not None:
         monkeypatch.setenv("AGX_HOST_PIPELINE_ROWS", rows)
-    w = W.make_attn_workload("host_chunks", 91, "bf16", 32, 8, 128, [1000, 333], [700, 600], spare_pages=2)
+    w = W.make_attn_workload("host_chunks", 91, "bf16", 32, 8, 128, [600, 333, 50, 700], [1300, 200, 150, 900], spare_pages=2)
     b = DeviceBatch(w)
     to_t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).view(torch.bfloat16).pin_memory()
     hq, hk, hv = to_t(w.q_block), to_t(w.k_new), to_t(w.v_new)
