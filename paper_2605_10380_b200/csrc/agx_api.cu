@@ -267,8 +267,7 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
         bool lean_merge = false;   // fp16 partials and the two-warp merge kernel (slower than fp32 partials and the four-warp
                                    // one where the attention grid fills every SM twice over, e.g. four verify blocks of 4096)
         const bool small_one_per_sm = (k == KIND_SMALL1 || k == KIND_SMALL2 || k == KIND_SMALL4) && (k == KIND_SMALL4 || small_kw == 8);
-        // (the one-Q-tile tensor-core schedule as well: a single long sequence is one wave of whole-SM CTAs too; there the
-        //  fp16 partials are taken only together with the free SMs)
+        // (the one-Q-tile tensor-core schedule as well: a single long sequence is one wave of whole-SM CTAs too)
         if (!cluster && (small_one_per_sm || k == KIND_STREAM) && seqs.size() <= (size_t)kMaxSeqs && h->merge_sms) {
             long long pairs = 0;
             for (int s : seqs) pairs += (long long)Q[s] * c.num_q_heads;
@@ -278,9 +277,9 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
                 for (int s : seqs) ns_max = std::max(ns_max, (P[s] + Q[s] + C - 1) / C);
                 if (ns_max == 1 || items > h->sm_count) break;   // no merge, or more than one wave anyway
                 const long long reserve = (pairs + (ns_max <= 20 ? 24 : 16) - 1) / (ns_max <= 20 ? 24 : 16);
-                if (k == KIND_STREAM && reserve > h->sm_count / 8) break;
+                if (reserve > h->sm_count / 8) break;   // a merge that large needs the whole device anyway
                 lean_merge = true;
-                if (reserve > h->sm_count / 8 || items <= h->sm_count - reserve || items <= base_items) break;
+                if (items <= h->sm_count - reserve || items <= base_items) break;
                 C += unit;
             }
         }
