@@ -81,16 +81,18 @@ __device__ __forceinline__ int find_seq(const AttnParams& p, int item) {
 
 }  // namespace
 
-template <int MT, int KW, int NS>
-__global__ void __launch_bounds__(32 * MT * KW, (MT * KW <= 8) ? 2 : 1)
+// MW = m-tiles per warp: with MW = 2 a warp scores its page against both 16-row tiles of a 32-row block and accumulates
+// both tiles' output columns, so every K and V fragment is read from shared memory once instead of twice.
+template <int MT, int KW, int NS, int MW>
+__global__ void __launch_bounds__(32 * (MT / MW) * KW, ((MT / MW) * KW <= 8 && MW == 1) ? 2 : 1)
 attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtensorMap map_k,
                        const __grid_constant__ CUtensorMap map_v) {
     extern __shared__ unsigned char smem_raw[];
     constexpr int kKW = KW;
     constexpr int kStageTokens = kKW * kPage;
     constexpr int kStageBytes = 2 * kStageTokens * kRowBytes;
-    constexpr int kThreads = 32 * MT * KW;
-    constexpr int kWarps = MT * KW;
+    constexpr int kThreads = 32 * (MT / MW) * KW;
+    constexpr int kWarps = (MT / MW) * KW;
     constexpr int kRingBytes = NS * kStageBytes;
     constexpr int kClusterBytes = MT * 16 * (kD * 4 + 8);   // this CTA's (O, m, l) rows, read by the cluster's other CTAs (in the dead ring)
     constexpr int kRegion = kRingBytes > kClusterBytes ? kRingBytes : kClusterBytes;
@@ -109,8 +111,8 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
-    const int mt = warp % MT;
-    const int kg = warp / MT;
+    const int mt0 = (warp % (MT / MW)) * MW;   // first of this warp's MW m-tiles
+    const int kg = warp / (MT / MW);
 
     const int si = find_seq(p, blockIdx.x);
     const SeqPlan sp = p.seq[si];
@@ -233,32 +235,33 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     }
     __syncthreads();  // barriers initialised, Q tile visible
 
-    uint32_t qa[8][4];
-    {
-        const int r = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+    uint32_t qa[MW][8][4];
+#pragma unroll
+    for (int w = 0; w < MW; ++w) {
+        const int r = (mt0 + w) * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             const int ch = ks * 2 + (lane >> 4);
-            ldmatrix_x4(qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], smem_u32(q_smem) + swz(r, ch));
+            ldmatrix_x4(qa[w][ks][0], qa[w][ks][1], qa[w][ks][2], qa[w][ks][3], smem_u32(q_smem) + swz(r, ch));
         }
     }
 
-    // Warp (mt, kg) scores page kg of every stage against its 16 rows, but accumulates O only for the kCG * 16
+    // Warp (mt, kg) scores page kg of every stage against its 16 rows (per m-tile), but accumulates O only for the kCG * 16
     // output columns it owns, over ALL pages of the stage: the P fragments of the stage's pages travel through shared
     // memory and the KV groups of an m-tile share one running maximum, so nothing has to be merged at the end.
     constexpr int kCG = 8 / KW;                    // 16-column groups of O per warp
-    float o[2 * kCG][4];
+    float o[MW][2 * kCG][4];
+    float m_run[MW][2], l_run[MW][2];              // running maximum of rows g and g + 8 (log2 units) | this lane's share of the row sums
+    int limit[MW][2];                              // last visible token of the two rows this thread holds
 #pragma unroll
-    for (int n = 0; n < 2 * kCG; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
-    float m_run[2] = {-INFINITY, -INFINITY};       // the m-tile's running maximum of rows g and g + 8 (log2 units)
-    float l_run[2] = {0.f, 0.f};                   // this lane's share of this KV group's row sums
-
-    // row limits (last visible token) for the two rows this thread holds
-    int limit[2];
-    {
-        const int rA = row0 + mt * 16 + (lane >> 2);
-        limit[0] = P + min(rA / G, q - 1);
-        limit[1] = P + min((rA + 8) / G, q - 1);
+    for (int w = 0; w < MW; ++w) {
+#pragma unroll
+        for (int n = 0; n < 2 * kCG; ++n) { o[w][n][0] = o[w][n][1] = o[w][n][2] = o[w][n][3] = 0.f; }
+        m_run[w][0] = m_run[w][1] = -INFINITY;
+        l_run[w][0] = l_run[w][1] = 0.f;
+        const int rA = row0 + (mt0 + w) * 16 + (lane >> 2);
+        limit[w][0] = P + min(rA / G, q - 1);
+        limit[w][1] = P + min((rA + 8) / G, q - 1);
     }
     // Per-lane ldmatrix offsets inside one page of the TMA layout [half 2][16 rows][128 B], where the
     // 16-byte unit u of row r sits at ((u ^ (r & 7)) << 4).  K (x4): row = nt*8 + lane%8, unit = (kp&1)*4 + lane/8.
@@ -271,10 +274,10 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
 #pragma unroll
     for (int j = 0; j < 4; ++j) v_off[j] = v_row * 128 + ((v_x ^ (uint32_t)(j << 1)) << 4);
 
-    const int rg = lane >> 2;                      // this lane's rows in the m-tile: rg and rg + 8
-    float* my_max = x_max + (mt * 16 + rg) * KW;   // x_max[mt][row][kg]
-    uint4* my_p = x_p + (mt * KW) * 32 + lane;     // x_p[mt][kg][lane]: page kg's P as the lanes' MMA A fragments
-    auto group_sync = [&]() { asm volatile("bar.sync %0, %1;\n" ::"r"(1 + mt), "n"(32 * KW) : "memory"); };
+    const int rg = lane >> 2;                      // this lane's rows in an m-tile: rg and rg + 8
+    float* my_max = x_max + (mt0 * 16 + rg) * KW;  // x_max[mt][row][kg]; m-tile mt0 + w: + w * 16 * KW
+    uint4* my_p = x_p + (mt0 * KW) * 32 + lane;    // x_p[mt][kg][lane]: page kg's P as the lanes' MMA A fragments; + w * KW * 32
+    auto group_sync = [&]() { asm volatile("bar.sync %0, %1;\n" ::"r"(1 + mt0 / MW), "n"(32 * KW) : "memory"); };
 
     bool live = true;   // a warp whose wait gave up keeps meeting the others at the group barriers
 #pragma unroll 1
@@ -288,8 +291,10 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
         const int tok0 = stage_tok0 + kg * kPage;
         const bool has_page = kg < npg;
         const uint32_t stage_base = smem_base + slot * kStageBytes;
-        float s[2][4];
-        float mx[2] = {-INFINITY, -INFINITY};
+        float s[MW][2][4];
+        float mx[MW][2];
+#pragma unroll
+        for (int w = 0; w < MW; ++w) mx[w][0] = mx[w][1] = -INFINITY;
         if (has_page) {
             const uint32_t k_base = stage_base + kg * 4096;
             const uint32_t v_base = k_base + kStageTokens * kRowBytes;
@@ -303,13 +308,16 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
                 }
                 __syncwarp();
             }
-            // S = Q K^T for 16 tokens: two n-tiles of 8 tokens, as four accumulation chains of four MMAs each
-            // (even and odd k-steps of both n-tiles): a dependent mma.sync is slow to issue
-            float s_odd[2][4];
+            // S = Q K^T for 16 tokens: two n-tiles of 8 tokens, as four accumulation chains of four MMAs each per m-tile
+            // (even and odd k-steps of both n-tiles): a dependent mma.sync is slow to issue.  A K fragment serves every m-tile.
+            float s_odd[MW][2][4];
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt) {
-                s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-                s_odd[nt][0] = s_odd[nt][1] = s_odd[nt][2] = s_odd[nt][3] = 0.f;
+            for (int w = 0; w < MW; ++w) {
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) {
+                    s[w][nt][0] = s[w][nt][1] = s[w][nt][2] = s[w][nt][3] = 0.f;
+                    s_odd[w][nt][0] = s_odd[w][nt][1] = s_odd[w][nt][2] = s_odd[w][nt][3] = 0.f;
+                }
             }
 #pragma unroll
             for (int kp = 0; kp < 4; ++kp) {
@@ -317,92 +325,109 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
                 for (int nt = 0; nt < 2; ++nt) {
                     uint32_t b0, b1, b2, b3;
                     ldmatrix_x4(b0, b1, b2, b3, k_base + (kp >> 1) * 2048 + nt * 1024 + k_off[kp & 1]);
-                    mma_bf16(s[nt], qa[2 * kp], b0, b1);
-                    mma_bf16(s_odd[nt], qa[2 * kp + 1], b2, b3);
-                }
-            }
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) s[nt][e] += s_odd[nt][e];
-            }
-            // mask the causal edge / the end of the split (raw scores; the scale is folded into the exp)
-            if ((tok0 + kPage - 1 > P) || (tok0 + kPage > tok_end)) {
-#pragma unroll
-                for (int nt = 0; nt < 2; ++nt) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int tok = tok0 + nt * 8 + 2 * (lane & 3) + (e & 1);
-                        if (tok > limit[e >> 1] || tok >= tok_end) s[nt][e] = -INFINITY;
+                    for (int w = 0; w < MW; ++w) {
+                        mma_bf16(s[w][nt], qa[w][2 * kp], b0, b1);
+                        mma_bf16(s_odd[w][nt], qa[w][2 * kp + 1], b2, b3);
                     }
                 }
             }
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                float v = fmaxf(fmaxf(s[0][2 * h], s[0][2 * h + 1]), fmaxf(s[1][2 * h], s[1][2 * h + 1]));
-                v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, 1));
-                v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, 2));
-                mx[h] = v * p.scale_log2;
-            }
-        }
-        if ((lane & 3) == 0) { my_max[kg] = mx[0]; my_max[8 * KW + kg] = mx[1]; }
-        group_sync();   // the stage's page maxima of this m-tile are in place
-
-        // one running maximum per row for the whole m-tile; P of this warp's page against it
-        float corr[2];
-        uint32_t pa[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            float m_new = m_run[h];
-#pragma unroll
-            for (int k4 = 0; k4 < KW; k4 += 4) {
-                const float4 v = *(const float4*)(my_max + h * 8 * KW + k4);
-                m_new = fmaxf(fmaxf(m_new, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
-            }
-            const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
-            corr[h] = ex2(m_run[h] - m_ref);
-            m_run[h] = m_new;
-            float sum = 0.f;
-            if (has_page) {
+            for (int w = 0; w < MW; ++w) {
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt) {
-                    s[nt][2 * h] = ex2(fmaf(s[nt][2 * h], p.scale_log2, -m_ref));
-                    s[nt][2 * h + 1] = ex2(fmaf(s[nt][2 * h + 1], p.scale_log2, -m_ref));
-                    sum += s[nt][2 * h] + s[nt][2 * h + 1];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) s[w][nt][e] += s_odd[w][nt][e];
+                }
+                // mask the causal edge / the end of the split (raw scores; the scale is folded into the exp)
+                if ((tok0 + kPage - 1 > P) || (tok0 + kPage > tok_end)) {
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int tok = tok0 + nt * 8 + 2 * (lane & 3) + (e & 1);
+                            if (tok > limit[w][e >> 1] || tok >= tok_end) s[w][nt][e] = -INFINITY;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    float v = fmaxf(fmaxf(s[w][0][2 * h], s[w][0][2 * h + 1]), fmaxf(s[w][1][2 * h], s[w][1][2 * h + 1]));
+                    v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, 1));
+                    v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, 2));
+                    mx[w][h] = v * p.scale_log2;
                 }
             }
-            l_run[h] = l_run[h] * corr[h] + sum;
         }
-        if (has_page) {
-            pa[0] = pack_bf16(s[0][0], s[0][1]);
-            pa[1] = pack_bf16(s[0][2], s[0][3]);
-            pa[2] = pack_bf16(s[1][0], s[1][1]);
-            pa[3] = pack_bf16(s[1][2], s[1][3]);
-        }
-        my_p[kg * 32] = make_uint4(pa[0], pa[1], pa[2], pa[3]);
-        if (__any_sync(0xFFFFFFFFu, corr[0] != 1.f || corr[1] != 1.f)) {
+        if ((lane & 3) == 0) {
 #pragma unroll
-            for (int n = 0; n < 2 * kCG; ++n) {
-                o[n][0] *= corr[0]; o[n][1] *= corr[0];
-                o[n][2] *= corr[1]; o[n][3] *= corr[1];
+            for (int w = 0; w < MW; ++w) { my_max[w * 16 * KW + kg] = mx[w][0]; my_max[w * 16 * KW + 8 * KW + kg] = mx[w][1]; }
+        }
+        group_sync();   // the stage's page maxima of this warp's m-tiles are in place
+
+        // one running maximum per row for a whole m-tile; P of this warp's page against it
+#pragma unroll
+        for (int w = 0; w < MW; ++w) {
+            float corr[2];
+            uint32_t pa[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                float m_new = m_run[w][h];
+#pragma unroll
+                for (int k4 = 0; k4 < KW; k4 += 4) {
+                    const float4 v = *(const float4*)(my_max + w * 16 * KW + h * 8 * KW + k4);
+                    m_new = fmaxf(fmaxf(m_new, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+                }
+                const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
+                corr[h] = ex2(m_run[w][h] - m_ref);
+                m_run[w][h] = m_new;
+                float sum = 0.f;
+                if (has_page) {
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt) {
+                        s[w][nt][2 * h] = ex2(fmaf(s[w][nt][2 * h], p.scale_log2, -m_ref));
+                        s[w][nt][2 * h + 1] = ex2(fmaf(s[w][nt][2 * h + 1], p.scale_log2, -m_ref));
+                        sum += s[w][nt][2 * h] + s[w][nt][2 * h + 1];
+                    }
+                }
+                l_run[w][h] = l_run[w][h] * corr[h] + sum;
+            }
+            if (has_page) {
+                pa[0] = pack_bf16(s[w][0][0], s[w][0][1]);
+                pa[1] = pack_bf16(s[w][0][2], s[w][0][3]);
+                pa[2] = pack_bf16(s[w][1][0], s[w][1][1]);
+                pa[3] = pack_bf16(s[w][1][2], s[w][1][3]);
+            }
+            my_p[(w * KW + kg) * 32] = make_uint4(pa[0], pa[1], pa[2], pa[3]);
+            if (__any_sync(0xFFFFFFFFu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+                for (int n = 0; n < 2 * kCG; ++n) {
+                    o[w][n][0] *= corr[0]; o[w][n][1] *= corr[0];
+                    o[w][n][2] *= corr[1]; o[w][n][3] *= corr[1];
+                }
             }
         }
         group_sync();   // every page's P fragments (and zeroed V rows) are in place
 
-        // O[:, this warp's columns] += P V over the stage's pages
+        // O[:, this warp's columns] += P V over the stage's pages (a V fragment serves every m-tile)
 #pragma unroll
         for (int k = 0; k < kKW; ++k) {
             if (k < npg) {
-                const uint4 pk = my_p[k * 32];
-                const uint32_t a[4] = {pk.x, pk.y, pk.z, pk.w};
+                uint4 pk[MW];
+#pragma unroll
+                for (int w = 0; w < MW; ++w) pk[w] = my_p[(w * KW + k) * 32];
                 const uint32_t v_base = stage_base + kStageTokens * kRowBytes + k * 4096;
 #pragma unroll
                 for (int c = 0; c < kCG; ++c) {
                     const int cp = kg * kCG + c;
                     uint32_t b0, b1, b2, b3;
                     ldmatrix_x4_trans(b0, b1, b2, b3, v_base + (cp >> 2) * 2048 + v_off[cp & 3]);
-                    mma_bf16(o[2 * c], a, b0, b1);
-                    mma_bf16(o[2 * c + 1], a, b2, b3);
+#pragma unroll
+                    for (int w = 0; w < MW; ++w) {
+                        const uint32_t a[4] = {pk[w].x, pk[w].y, pk[w].z, pk[w].w};
+                        mma_bf16(o[w][2 * c], a, b0, b1);
+                        mma_bf16(o[w][2 * c + 1], a, b2, b3);
+                    }
                 }
             }
         }
@@ -412,11 +437,17 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
 
     // ---- row sums of the m-tile: each KV group's share through shared memory
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 1);
-        l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 2);
+    for (int w = 0; w < MW; ++w) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            l_run[w][h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[w][h], 1);
+            l_run[w][h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[w][h], 2);
+        }
+        if ((lane & 3) == 0) {
+            x_l[((mt0 + w) * 16 + rg) * KW + kg] = l_run[w][0];
+            x_l[((mt0 + w) * 16 + rg + 8) * KW + kg] = l_run[w][1];
+        }
     }
-    if ((lane & 3) == 0) { x_l[(mt * 16 + rg) * KW + kg] = l_run[0]; x_l[(mt * 16 + rg + 8) * KW + kg] = l_run[1]; }
     // After a wait gave up, copies armed by the producer lane may still be on their way into the ring: it waits for
     // them (bounded by the clock alone) before the CTA reuses or releases that shared memory.
     if (tid == 0 && *abort_flag) {
@@ -431,8 +462,9 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
     float* cl_o = (float*)ring;                              // [MT*16][kD]
     float2* cl_ml = (float2*)(ring + MT * 16 * kD * 4);      // [MT*16]
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        const int r = mt * 16 + rg + 8 * h;                  // row of the CTA's chunk
+    for (int wh = 0; wh < 2 * MW; ++wh) {
+        const int w = wh >> 1, h = wh & 1;
+        const int r = (mt0 + w) * 16 + rg + 8 * h;           // row of the CTA's chunk
         const unsigned int row_lanes = __ballot_sync(0xFFFFFFFFu, row0 + r < rows);   // (the four lanes of a row go together)
         if (row0 + r >= rows) continue;
         float l_all = 0.f;
@@ -441,7 +473,7 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
             const float4 v = *(const float4*)(x_l + r * KW + k4);
             l_all += (v.x + v.y) + (v.z + v.w);
         }
-        const float m_all = m_run[h];
+        const float m_all = m_run[w][h];
         const int i = (row0 + r) / G, hg = (row0 + r) - i * G;
         const int hd = g * G + hg;
         const bool first = kg == 0 && (lane & 3) == 0;       // one lane per row writes the row's (m, l)
@@ -450,7 +482,7 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
             __nv_bfloat16* orow = (__nv_bfloat16*)p.out + ((long long)(sp.q_row0 + i) * p.hq + hd) * kD;
 #pragma unroll
             for (int n = 0; n < 2 * kCG; ++n)
-                *(uint32_t*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)) = pack_bf16(o[n][2 * h] * inv, o[n][2 * h + 1] * inv);
+                *(uint32_t*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)) = pack_bf16(o[w][n][2 * h] * inv, o[w][n][2 * h + 1] * inv);
             if (p.lse && first) p.lse[(long long)(sp.q_row0 + i) * p.hq + hd] = (m_all + log2f(l_all)) * 0.6931471805599453f;
         } else {
             if (in_cluster) {
@@ -458,7 +490,7 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
                 if (first) cl_ml[r] = make_float2(m_all, l_all);
 #pragma unroll
                 for (int n = 0; n < 2 * kCG; ++n)
-                    *(float2*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)) = make_float2(o[n][2 * h], o[n][2 * h + 1]);
+                    *(float2*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)) = make_float2(o[w][n][2 * h], o[w][n][2 * h + 1]);
             } else {
                 // split partial for the merge kernel, written past the L1 (read next by other SMs)
                 const long long e = (long long)sp.part_base + ((long long)i * p.hq + hd) * sp.nsplit + split;
@@ -472,8 +504,8 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
                     unsigned char* orow = (unsigned char*)p.part_o + e * 512;
 #pragma unroll
                     for (int c = 0; c < kCG; ++c) {
-                        const __half2 lo = __floats2half2_rn(o[2 * c][2 * h] * inv, o[2 * c][2 * h + 1] * inv);
-                        const __half2 hi = __floats2half2_rn(o[2 * c + 1][2 * h] * inv, o[2 * c + 1][2 * h + 1] * inv);
+                        const __half2 lo = __floats2half2_rn(o[w][2 * c][2 * h] * inv, o[w][2 * c][2 * h + 1] * inv);
+                        const __half2 hi = __floats2half2_rn(o[w][2 * c + 1][2 * h] * inv, o[w][2 * c + 1][2 * h + 1] * inv);
                         const unsigned int mine_lo = *reinterpret_cast<const unsigned int*>(&lo);
                         const unsigned int mine_hi = *reinterpret_cast<const unsigned int*>(&hi);
                         const bool odd = lane & 1;
@@ -487,7 +519,7 @@ attn_small_bf16_kernel(const __grid_constant__ AttnParams p, const __grid_consta
                     float* orow = p.part_o + e * kD;
 #pragma unroll
                     for (int n = 0; n < 2 * kCG; ++n)
-                        __stcg((float2*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)), make_float2(o[n][2 * h], o[n][2 * h + 1]));
+                        __stcg((float2*)(orow + (kg * kCG * 2 + n) * 8 + 2 * (lane & 3)), make_float2(o[w][n][2 * h], o[w][n][2 * h + 1]));
                 }
             }
         }
@@ -902,7 +934,7 @@ constexpr int small_smem_bytes() {
     return (kRing > kClusterBytes ? kRing : kClusterBytes) + MT * 16 * kRowBytes + 2 * NS * 8 + 16 + kExchange + 1024;
 }
 
-template <int MT, int KW, int NS>
+template <int MT, int KW, int NS, int MW = 1>
 cudaError_t launch_small(const AttnParams& p, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
     constexpr int kSmem = small_smem_bytes<MT, KW, NS>();
     // the attribute is per device: remember which devices have it (a process normally drives one GPU)
@@ -911,19 +943,19 @@ cudaError_t launch_small(const AttnParams& p, const CUtensorMap& map_k, const CU
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return cudaErrorInvalidDevice;
     bool& configured = configured_on[device];
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+        cudaError_t e = cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS, MW>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);   // clusters of up to 16
+        e = cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS, MW>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);   // clusters of up to 16
         if (e != cudaSuccess) return e;
         configured = true;
     }
     if (p.cluster_size > 1)
-        return launch_chained_cluster(attn_small_bf16_kernel<MT, KW, NS>, dim3(p.num_items), dim3(32 * MT * KW), kSmem,
+        return launch_chained_cluster(attn_small_bf16_kernel<MT, KW, NS, MW>, dim3(p.num_items), dim3(32 * (MT / MW) * KW), kSmem,
                                       (unsigned)p.cluster_size, stream, p, map_k, map_v);
-    return launch_chained(attn_small_bf16_kernel<MT, KW, NS>, dim3(p.num_items), dim3(32 * MT * KW), kSmem, stream, p, map_k, map_v);
+    return launch_chained(attn_small_bf16_kernel<MT, KW, NS, MW>, dim3(p.num_items), dim3(32 * (MT / MW) * KW), kSmem, stream, p, map_k, map_v);
 }
 
-template <int MT, int KW, int NS>
+template <int MT, int KW, int NS, int MW = 1>
 int max_clusters(int cluster) {
     static int cached[64][17];   // 0 = not asked yet, else 1 + answer
     int device = 0;
@@ -931,15 +963,15 @@ int max_clusters(int cluster) {
     if (cached[device][cluster]) return cached[device][cluster] - 1;
     constexpr int kSmem = small_smem_bytes<MT, KW, NS>();
     int n = 0;
-    if (cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) == cudaSuccess &&
-        cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+    if (cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS, MW>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) == cudaSuccess &&
+        cudaFuncSetAttribute(attn_small_bf16_kernel<MT, KW, NS, MW>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(cluster * 64); cfg.blockDim = dim3(32 * MT * KW); cfg.dynamicSmemBytes = kSmem;
+        cfg.gridDim = dim3(cluster * 64); cfg.blockDim = dim3(32 * (MT / MW) * KW); cfg.dynamicSmemBytes = kSmem;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr; cfg.numAttrs = 1;
-        if (cudaOccupancyMaxActiveClusters(&n, attn_small_bf16_kernel<MT, KW, NS>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+        if (cudaOccupancyMaxActiveClusters(&n, attn_small_bf16_kernel<MT, KW, NS, MW>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
     } else {
         (void)cudaGetLastError();
     }
@@ -948,7 +980,15 @@ int max_clusters(int cluster) {
 }
 }  // namespace
 
+// 32-row blocks on 8-page stages: both m-tiles in every warp (8 warps; decode verify 9.84 -> 9.42 us) or, with AGX_SMALL_MW=1,
+// one m-tile per warp (16 warps).  On 4-page stages two tiles per warp are slower (4 x 4096 verify 20.1 -> 20.3 us).
+static bool two_tiles_per_warp() {
+    static const bool on = !(getenv("AGX_SMALL_MW") && atoi(getenv("AGX_SMALL_MW")) == 1);
+    return on;
+}
+
 int attn_small_max_clusters(int mt, int kw, int cluster) {
+    if (mt == 2 && kw == 8 && two_tiles_per_warp()) return max_clusters<2, 8, 3, 2>(cluster);
     switch (mt * 16 + kw) {
         case 1 * 16 + 4: return max_clusters<1, 4, 3>(cluster);
         case 2 * 16 + 4: return max_clusters<2, 4, 3>(cluster);
@@ -962,6 +1002,7 @@ int attn_small_max_clusters(int mt, int kw, int cluster) {
 cudaError_t launch_attn_small_bf16(const AttnParams& p, int mt, int kw, const CUtensorMap& map_k, const CUtensorMap& map_v,
                                    cudaStream_t stream) {
     if (p.num_items == 0) return cudaSuccess;
+    if (mt == 2 && kw == 8 && two_tiles_per_warp()) return launch_small<2, 8, 3, 2>(p, map_k, map_v, stream);
     switch (mt * 16 + kw) {
         case 1 * 16 + 4: return launch_small<1, 4, 3>(p, map_k, map_v, stream);
         case 2 * 16 + 4: return launch_small<2, 4, 3>(p, map_k, map_v, stream);
