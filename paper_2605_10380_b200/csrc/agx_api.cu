@@ -43,6 +43,7 @@ struct agx_handle {
     int debug_plan;         // print launch plans to stderr (env AGX_DEBUG_PLAN)
     int small_kw;           // pages per pipeline stage of the warp-MMA kernel: 4, 8, or 0 = chosen per batch (env AGX_SMALL_KW)
     int batch_stream_tokens; // total tokens of a batch's small blocks from which they all take the stream schedule (env AGX_BATCH_STREAM_TOKENS)
+    bool longest_first;     // sequences of a launch ordered by decreasing context length (env AGX_LONGEST_FIRST=0: batch order)
     bool merge_sms;         // one-wave small-q launches leave SMs free for their merge kernel (env AGX_MERGE_SMS=0 turns it off)
     bool cluster_merge;     // KV splits of the small-q kernel merged inside thread-block clusters where the batch allows (env AGX_CLUSTER_MERGE=0 turns it off)
     int zero_copy;          // host steps: bit 0 = kernels read small pinned inputs, bit 1 = kernels write `out` into a pinned buffer (env AGX_ZERO_COPY, default 3)
@@ -169,8 +170,7 @@ agx_status build_plan(agx_handle* h, int B, const int32_t* P, const int32_t* Q, 
     const int small_kw = h->small_kw ? h->small_kw : (warp_mma_seqs >= 2 && warp_mma_tokens * c.num_kv_heads / 8 >= 8192) ? 4 : 8;
     // Work items are handed to the SMs in launch order: the sequences with the longest contexts go first, so that the
     // longest items of a ragged batch are not the ones left over for the last wave (env AGX_LONGEST_FIRST=0 keeps the batch order).
-    static const bool longest_first = !(getenv("AGX_LONGEST_FIRST") && atoi(getenv("AGX_LONGEST_FIRST")) == 0);
-    if (longest_first)
+    if (h->longest_first)
         for (int k : {(int)KIND_TILE, (int)KIND_STREAM})
             std::stable_sort(groups[k].begin(), groups[k].end(), [&](int a, int b) { return P[a] + Q[a] > P[b] + Q[b]; });
     for (int k = 0; k < KIND_COUNT; ++k) {
@@ -402,6 +402,8 @@ agx_status agx_create(const agx_config* cfg, agx_handle** out) {
     env = getenv("AGX_HOST_PIPELINE_ROWS");
     h->pipe_rows = env ? std::max(0, atoi(env)) : 384;   // measured on the long-context step: 256 / 384 / 512 / 768 / 1024 rows -> 1.54 / 1.43 / 1.57 / 1.56 / 1.72 ms
     h->pipe_in = h->pipe_out = nullptr;
+    env = getenv("AGX_LONGEST_FIRST");
+    h->longest_first = !(env && atoi(env) == 0);
     env = getenv("AGX_MERGE_SMS");
     h->merge_sms = !(env && atoi(env) == 0);
     env = getenv("AGX_ZERO_COPY");

@@ -833,6 +833,30 @@ def test_c3_prefix_cached_prefill_and_full_prefill_rows():
     check_attention(out[si, sh], full, "c3 vs full prefill rows", strict=True)
 
 
+def test_order_of_sequences_inside_a_launch_changes_no_bit(monkeypatch):
+    """The planner puts the longest contexts first in the launches of the tensor-core schedules; with
+    AGX_LONGEST_FIRST=0 they stay in batch order.  Work items do not depend on one another, so the two orders must
+    give the same bits (ragged prefill blocks and verify blocks in one batch, shortest context first in the batch)."""
+    w = W.make_attn_workload("order", 4242, "bf16", 32, 8, 128, [300, 9000, 1500, 12000, 4000, 700], [200, 8, 500, 4, 300, 130],
+                             spare_pages=2)
+    outs = []
+    for flag in ("1", "0"):
+        monkeypatch.setenv("AGX_LONGEST_FIRST", flag)
+        b = DeviceBatch(w)
+        out, lse = b.attend_append()
+        assert b.status() == 0
+        outs.append((host_storage(b.out, "bf16").copy(), lse.copy()))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    kp, vp = oracle_pools_after_append(w)
+    rng = np.random.default_rng(7)
+    for s in range(w.batch):
+        q = int(w.q_len[s]); r0 = int(w.cu_q[s])
+        si = rng.integers(0, q, 8).astype(np.int32); sh = rng.integers(0, 32, 8).astype(np.int32)
+        ref, _, _ = oracle.attn_paged(w.q_block[r0:r0 + q], kp, vp, w.page_table[s], "bf16", int(w.prefix_len[s]), select=(si, sh))
+        got = torch.from_numpy(outs[0][0].view(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
+        check_attention(got[r0 + si, sh], ref, "order of sequences")
+
+
 def test_tile_and_small_kernels_in_one_ragged_batch():
     P = [2048, 2300, 2048 + 7, 4000, 2600, 3000]
     q = [8, 200, 1, 130, 16, 513]
