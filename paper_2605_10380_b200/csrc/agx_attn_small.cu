@@ -785,10 +785,12 @@ attn_combine_kernel(const __grid_constant__ AttnParams p, int total_rows) {
 }
 
 // The same merge for the partials of the 256-row tensor-core schedule (fp16 rows divided by their own sums, at most 4
-// splits): each warp takes up to three (row, head) pairs with all their loads in flight at once, so that the merge of
-// a split prefill (12288 pairs, 9 MB of partials) is one wave of CTAs and one memory round trip per warp instead of
-// several waves of short-lived CTAs, and a larger merge has a third of the CTAs with three times the bytes in flight each.
-constexpr int kCombineRows = 3;
+// splits): each warp takes two (row, head) pairs with all their loads in flight at once, so that the merge of a split
+// prefill (12288 pairs, 9 MB of partials) is about one wave of CTAs and one memory round trip per warp instead of several
+// waves of short-lived CTAs, and a larger merge has half the CTAs with twice the bytes in flight each.  (Measured: one /
+// two / three / four pairs per warp give 29.1 / 19.8 / 20.5-21.6 / - us for the 65536 pairs of the long prefill under
+// ncu; c3 29.9 / 29.9 / 31.0 us and (1500, 200) 17.8 / 18.3 / 19.3 us per call for two / three / four.)
+constexpr int kCombineRows = 2;
 __global__ void __launch_bounds__(128, 8)
 attn_combine_half4_kernel(const __grid_constant__ AttnParams p, int total_rows) {
     pdl_launch_dependents();
@@ -1029,8 +1031,7 @@ cudaError_t launch_attn_combine(const AttnParams& p, int dtype, int total_rows, 
     for (int i = 0; i < p.num_seqs; ++i) ns_max = p.seq[i].nsplit > ns_max ? p.seq[i].nsplit : ns_max;
     if (dtype == AGX_BF16 && p.part_half) {
         if (ns_max <= 4) {
-            // CTAs whose warps take kCombineRows pairs each (under ncu on the long prefill, 65536 pairs: 20.5-21.6 us against 29.1 us
-            // for four times as many CTAs of one pair per warp)
+            // CTAs whose warps take kCombineRows pairs each
             const int want = (int)((n + 4 * kCombineRows - 1) / (4 * kCombineRows));
             return launch_chained(attn_combine_half4_kernel, dim3(want > 0 ? want : 1), dim3(128), 0, stream, p, total_rows);
         }
